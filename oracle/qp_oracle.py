@@ -1,0 +1,182 @@
+"""ctypes front end of the CPU oracle (``qp_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The GPU library never imports this module and this
+module never imports the GPU library.
+
+All arrays are numpy.  bf16 and fp16 tensors travel as ``uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "qp_oracle.c")
+_LIB = os.path.join(_HERE, "libqp_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+               "-fno-fast-math", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        i, i64, p = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p
+        L.qpo_n_keep.restype = i64
+        L.qpo_n_keep.argtypes = [i64, i, i, i, i]
+        L.qpo_scores.restype = None
+        L.qpo_scores.argtypes = [p, p, i, i, i, i, i, i, i, p, p]
+        L.qpo_select.restype = None
+        L.qpo_select.argtypes = [p, i, i, i, i, i, p]
+        L.qpo_quantize.restype = None
+        L.qpo_quantize.argtypes = [p, p, p, i, i, i, i, i, i, i, p, p, p, p, p, p]
+        L.qpo_dequantize.restype = None
+        L.qpo_dequantize.argtypes = [p, p, p, p, p, p, i, i, i, i, i, i, p, p]
+        L.qpo_decode.restype = None
+        L.qpo_decode.argtypes = [p, p, p, i, i, i, i, i, p]
+        L.qpo_f32_to_f16_down.restype = ctypes.c_uint16
+        L.qpo_f32_to_f16_down.argtypes = [ctypes.c_float]
+        L.qpo_f32_to_f16_up.restype = ctypes.c_uint16
+        L.qpo_f32_to_f16_up.argtypes = [ctypes.c_float]
+        L.qpo_f16_to_f32.restype = ctypes.c_float
+        L.qpo_f16_to_f32.argtypes = [ctypes.c_uint16]
+        L.qpo_num_threads.restype = i
+        L.qpo_num_threads.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray | None):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a: np.ndarray, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == dtype, (a.dtype, dtype)
+    return a
+
+
+def num_threads() -> int:
+    return int(lib().qpo_num_threads())
+
+
+def n_keep(budget_bits: int, bits: int, group: int, L: int, w: int) -> int:
+    return int(lib().qpo_n_keep(budget_bits, bits, group, L, w))
+
+
+def f32_to_f16_down(x: float) -> int:
+    return int(lib().qpo_f32_to_f16_down(x))
+
+
+def f32_to_f16_up(x: float) -> int:
+    return int(lib().qpo_f32_to_f16_up(x))
+
+
+def f16_to_f32(h: int) -> float:
+    return float(lib().qpo_f16_to_f32(h))
+
+
+def scores(q_win: np.ndarray, k: np.ndarray, pool: int = 7, want_votes: bool = False):
+    """q_win [Bt,Hq,w,D], k [Bt,Hkv,L,D] uint16(bf16) -> pooled [Bt,Hkv,P] fp64."""
+    q_win, k = _c(q_win, np.uint16), _c(k, np.uint16)
+    Bt, Hq, w, D = q_win.shape
+    _, Hkv, L, _ = k.shape
+    P = L - w
+    pooled = np.empty((Bt, Hkv, P), np.float64)
+    votes = np.empty((Bt, Hkv, P), np.float64) if want_votes else None
+    lib().qpo_scores(_p(q_win), _p(k), Bt, Hq, Hkv, D, L, w, pool, _p(pooled), _p(votes))
+    return (pooled, votes) if want_votes else pooled
+
+
+def select(pooled: np.ndarray, L: int, w: int, n: int) -> np.ndarray:
+    """pooled [Bt,Hkv,P] fp64 -> kept [Bt,Hkv,n] int32 ascending."""
+    pooled = _c(pooled, np.float64)
+    Bt, Hkv, P = pooled.shape
+    assert P == L - w
+    kept = np.empty((Bt, Hkv, n), np.int32)
+    lib().qpo_select(_p(pooled), Bt, Hkv, L, w, n, _p(kept))
+    return kept
+
+
+@dataclass
+class Packed:
+    """The packed pruned cache of one layer, in the library's documented layout."""
+    bits: int
+    group: int
+    n: int
+    k_codes: np.ndarray   # u32 [Bt,Hkv,n/g,D,wpg]   (bits 16: u16 [Bt,Hkv,n,D])
+    v_codes: np.ndarray   # u32 [Bt,Hkv,n,D/g,wpg]   (bits 16: u16 [Bt,Hkv,n,D])
+    k_scale: np.ndarray | None  # u16(fp16) [Bt,Hkv,n/g,D]
+    k_zero: np.ndarray | None
+    v_scale: np.ndarray | None  # u16(fp16) [Bt,Hkv,n,D/g]
+    v_zero: np.ndarray | None
+
+
+def quantize(k: np.ndarray, v: np.ndarray, kept: np.ndarray, bits: int, group: int) -> Packed:
+    k, v, kept = _c(k, np.uint16), _c(v, np.uint16), _c(kept, np.int32)
+    Bt, Hkv, L, D = k.shape
+    n = kept.shape[-1]
+    if bits == 16:
+        kc = np.empty((Bt, Hkv, n, D), np.uint16)
+        vc = np.empty((Bt, Hkv, n, D), np.uint16)
+        lib().qpo_quantize(_p(k), _p(v), _p(kept), Bt, Hkv, D, L, n, bits, group,
+                           _p(kc), None, None, _p(vc), None, None)
+        return Packed(bits, group, n, kc, vc, None, None, None, None)
+    assert n % group == 0 and D % group == 0
+    wpg = group * bits // 32
+    kc = np.empty((Bt, Hkv, n // group, D, wpg), np.uint32)
+    ks = np.empty((Bt, Hkv, n // group, D), np.uint16)
+    kz = np.empty_like(ks)
+    vc = np.empty((Bt, Hkv, n, D // group, wpg), np.uint32)
+    vs = np.empty((Bt, Hkv, n, D // group), np.uint16)
+    vz = np.empty_like(vs)
+    lib().qpo_quantize(_p(k), _p(v), _p(kept), Bt, Hkv, D, L, n, bits, group,
+                       _p(kc), _p(ks), _p(kz), _p(vc), _p(vs), _p(vz))
+    return Packed(bits, group, n, kc, vc, ks, kz, vs, vz)
+
+
+def dequantize(pk: Packed, D: int):
+    """-> (K', V') fp64 [Bt,Hkv,n,D]  (Eq. 5)."""
+    Bt, Hkv = pk.k_codes.shape[:2]
+    kd = np.empty((Bt, Hkv, pk.n, D), np.float64)
+    vd = np.empty_like(kd)
+    lib().qpo_dequantize(_p(pk.k_codes), _p(pk.k_scale), _p(pk.k_zero), _p(pk.v_codes),
+                         _p(pk.v_scale), _p(pk.v_zero), Bt, Hkv, D, pk.n, pk.bits, pk.group,
+                         _p(kd), _p(vd))
+    return kd, vd
+
+
+def decode(q: np.ndarray, kd: np.ndarray, vd: np.ndarray) -> np.ndarray:
+    """q [Bt,Hq,D] uint16(bf16); kd, vd fp64 [Bt,Hkv,n,D] -> out fp64 [Bt,Hq,D]  (Eq. 3)."""
+    q, kd, vd = _c(q, np.uint16), _c(kd, np.float64), _c(vd, np.float64)
+    Bt, Hq, D = q.shape
+    _, Hkv, n, _ = kd.shape
+    out = np.empty((Bt, Hq, D), np.float64)
+    lib().qpo_decode(_p(q), _p(kd), _p(vd), Bt, Hq, Hkv, D, n, _p(out))
+    return out
+
+
+def compress_layer(k, v, q_win, budget_bits: int, bits: int, group: int = 32, pool: int = 7):
+    """The whole prefill-side path on the CPU: scores -> select -> gather+quantize."""
+    L, w = k.shape[2], q_win.shape[2]
+    n = n_keep(budget_bits, bits, group, L, w)
+    if n < 0:
+        raise ValueError("budget cannot be met")
+    pooled = scores(q_win, k, pool)
+    kept = select(pooled, L, w, n)
+    return quantize(k, v, kept, bits, group), kept, pooled
