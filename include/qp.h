@@ -1,0 +1,172 @@
+/*
+ * qp.h — C ABI of the quantized-pruning KV-cache library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel hot path of "quantized pruning"
+ * (arXiv 2412.12706, Sec. 3 "Methods", paragraph "Quantized Pruning"): at the end
+ * of prefill each layer's KV cache is pruned to a fixed number of tokens per KV
+ * head and the kept keys/values are quantized; every decode step then attends
+ * over the dequantized packed cache.
+ *
+ * Conventions for every call
+ *   - "device" pointers are CUDA device memory of the current device, "host"
+ *     pointers ordinary host memory.  The caller owns every buffer; the library
+ *     never allocates, frees, synchronises or copies to the host.  All work is
+ *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and buffers must stay alive until the stream has passed that point.
+ *   - bf16 / fp16 tensors are raw 16-bit patterns, row-major and contiguous, base
+ *     addresses 16-byte aligned.  Inputs must be finite with |x| <= 65504.
+ *   - Host-checkable errors are returned before anything is launched and leave
+ *     the outputs untouched.  Launch failures are reported as QP_ERR_CUDA from
+ *     cudaGetLastError() without synchronising.
+ *   - Results are deterministic: same inputs, same bits.
+ *
+ * Notation (the paper's where it has one): Bt batch, Hq query heads, Hkv KV heads,
+ * G = Hq/Hkv, D head dimension, L prompt length, w observation window,
+ * P = L - w, B = bits in {2,4,8,16}, g = quantization group size,
+ * n = n_keep = tokens kept per KV head (the w window tokens included).
+ */
+#ifndef QP_H_
+#define QP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QP_OK = 0,
+  QP_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, Hq % Hkv != 0, w >= L, even pool ... */
+  QP_ERR_UNSUPPORTED = 2, /* bits not in {2,4,8,16}, group not in {32,64,128}, D not in {64,128}, G > 8, w > 64 */
+  QP_ERR_BUDGET = 3,      /* budget gives n <= w, or n is not a whole number of groups */
+  QP_ERR_WORKSPACE = 4,   /* workspace too small */
+  QP_ERR_ALIGNMENT = 5,   /* a base pointer is not 16-byte aligned */
+  QP_ERR_CUDA = 6         /* a launch failed */
+} qp_status;
+
+#define QP_MAX_LAYERS 128
+
+/*
+ * Packed pruned cache of one layer: a plain descriptor (host memory) of
+ * caller-allocated device buffers.  It may be copied freely; the library keeps no
+ * reference to it.  Layout of the buffers (wpg = g*B/32 words per group):
+ *
+ *   k_codes  uint32 [Bt, Hkv, n/g, D, wpg]   key groups: one channel, g consecutive KEPT tokens
+ *   k_scale  fp16   [Bt, Hkv, n/g, D]        (per-channel quantization, KIVI; Sec. 2 and 5.3)
+ *   k_zero   fp16   [Bt, Hkv, n/g, D]
+ *   v_codes  uint32 [Bt, Hkv, n, D/g, wpg]   value groups: one kept token, g consecutive channels
+ *   v_scale  fp16   [Bt, Hkv, n, D/g]        (per-token quantization)
+ *   v_zero   fp16   [Bt, Hkv, n, D/g]
+ *
+ * Element e of a group sits in word e / (32/B) at bit offset (e mod (32/B)) * B.
+ * A stored value is reconstructed as code * scale + zero (Eq. 5).
+ * B = 16: k_codes / v_codes hold the gathered bf16 rows [Bt, Hkv, n, D] and the four
+ * scale/zero pointers are unused (sizes 0).
+ * Kept tokens are stored in ascending order of their position in the prompt.
+ */
+typedef struct qp_cache {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep, reserved_;
+  size_t k_codes_bytes, v_codes_bytes;
+  size_t k_meta_bytes; /* bytes of k_scale; k_zero has the same size */
+  size_t v_meta_bytes; /* bytes of v_scale; v_zero has the same size */
+  void *k_codes, *v_codes, *k_scale, *k_zero, *v_scale, *v_zero; /* device */
+} qp_cache;
+
+/* Text for a status code (static storage, never NULL). */
+const char* qp_status_string(qp_status s);
+
+/*
+ * Token budget (Appendix B "Memory Budgets"; Fig. 2: tokens x bits is held
+ * constant).  budget_bits is the token-bit product per (KV head, channel), e.g.
+ * 512 tokens at 16 bit = 8192.  *n_keep = min(budget_bits / bits, L); scale/zero
+ * metadata is not counted.  QP_ERR_BUDGET if n_keep <= w or (bits < 16 and n_keep
+ * is not a multiple of group).  Host only.
+ */
+qp_status qp_n_keep(int64_t budget_bits, int bits, int group, int L, int w, int32_t* n_keep /* host, out */);
+
+/*
+ * Fills the shape fields and the four byte sizes of *out for the layout above and
+ * sets the six pointers to NULL.  Host only.
+ */
+qp_status qp_cache_layout(int batch, int n_q_heads, int n_kv_heads, int head_dim, int bits, int group,
+                          int n_keep, qp_cache* out /* host, out */);
+
+/* Bytes of device scratch that qp_compress_layer / qp_window_scores need (0 on invalid shapes). */
+size_t qp_compress_workspace_bytes(int batch, int n_q_heads, int n_kv_heads, int head_dim, int L, int w);
+
+/* Bytes of device scratch that qp_decode_attn needs for this cache (0 on an invalid descriptor).
+ * For qp_decode_attn_layers pass the sum over the layers. */
+size_t qp_decode_workspace_bytes(const qp_cache* cache /* host */);
+
+/*
+ * S1, observation-window scores.  The paper names its pruning method (SnapKV,
+ * Sec. 4 "Setup", Appendix B: the last 32 tokens are always retained) without
+ * defining it; this is the rule implemented.  For each KV head and each of its G
+ * query heads h and window rows i (position p = P + i):
+ *   S[j] = q[h,i].k[j] / sqrt(D) for j <= p;  Pr = softmax_j(S)
+ *   vote[j] = sum_h sum_i Pr_{h,i}[j]                          j < P
+ *   scores[j] = (sum_{|t| <= (pool-1)/2} vote[j+t], zero outside [0,P)) / pool
+ * Q_win bf16 [Bt,Hq,w,D], K bf16 [Bt,Hkv,L,D] (device) -> scores fp32 [Bt,Hkv,P] (device).
+ * pool must be odd (1 = no pooling).
+ */
+qp_status qp_window_scores(const void* Q_win, const void* K, int batch, int n_q_heads, int n_kv_heads,
+                           int head_dim, int L, int w, int pool, float* scores, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
+/*
+ * S2, per-head top-k (Sec. 3 "KV Pruning": keep s < n tokens).  Of the P prefix
+ * positions of each (batch, KV head) the n_keep - w with the largest score are
+ * kept, equal scores resolved toward the lower position; the w window positions
+ * P..L-1 are always kept.  scores fp32 [Bt,Hkv,P] (device, no NaN) ->
+ * kept_idx int32 [Bt,Hkv,n_keep] (device), ascending.
+ */
+qp_status qp_select_topk(const float* scores, int batch, int n_kv_heads, int L, int w, int n_keep,
+                         int32_t* kept_idx, void* stream);
+
+/*
+ * S3, gather + quantize + pack (Eq. 4: Q(G) = round((G - z)/s), s = (m - z)/(2^B - 1),
+ * z = min, m = max of the group).  Stored precision: z is rounded down and s rounded
+ * up to fp16, and the codes are computed in fp32 from the STORED z and s as
+ * clamp(rint((x - z)/s), 0, 2^B - 1) (true division, ties to even); s = 0 gives codes 0.
+ * K, V bf16 [Bt,Hkv,L,D], kept_idx int32 [Bt,Hkv,n_keep] ascending, each < L (device).
+ * cache: shape fields as from qp_cache_layout, pointers set by the caller.
+ */
+qp_status qp_gather_quantize(const void* K, const void* V, const int32_t* kept_idx, int L,
+                             const qp_cache* cache /* host */, void* stream);
+
+/*
+ * Prefill-side path of one layer: S1 -> S2 -> S3 ("Quantized Pruning": prune first,
+ * then quantize the preserved states).  n_keep follows qp_n_keep(budget_bits, bits,
+ * group, L, w); cache->n_keep etc. must agree with it (QP_ERR_BUDGET otherwise).
+ * Outputs: the cache buffers and kept_idx int32 [Bt,Hkv,n_keep] (device).
+ */
+qp_status qp_compress_layer(const void* K, const void* V, const void* Q_win, int batch, int n_q_heads,
+                            int n_kv_heads, int head_dim, int L, int w, int64_t budget_bits, int bits,
+                            int group, int pool, const qp_cache* cache /* host */,
+                            int32_t* kept_idx /* device */, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+/*
+ * S4 + S5, decode-step attention over the packed cache (Eq. 3 on the dequantized
+ * cache of Eq. 5): out[b,h,:] = softmax_t(q[b,h].K'[t] / sqrt(D)) V' over the n kept
+ * tokens of KV head h / G, no mask.  q, out bf16 [Bt,Hq,D] (device).  The token
+ * range is split across thread blocks and the partial results merged; workspace
+ * holds the partials.
+ */
+qp_status qp_decode_attn(const void* q, const qp_cache* cache /* host */, void* out, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
+/*
+ * The same decode attention for n_layers independent layers in one pair of
+ * launches (1 <= n_layers <= QP_MAX_LAYERS).  q, caches, out are HOST arrays of
+ * length n_layers; q[l], out[l] are device pointers.  All caches must agree in
+ * batch, heads, head_dim, bits and group; n_keep may differ per layer.
+ */
+qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches,
+                                void* const* out, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QP_H_ */

@@ -1,0 +1,223 @@
+// C ABI of the library: argument checks, workspace carving and launches.  No allocation,
+// no synchronisation, no host copies.
+#include <cstring>
+
+#include "qp_common.cuh"
+
+using namespace qp;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool pow2_bits(int b) { return b == 2 || b == 4 || b == 8 || b == 16; }
+inline bool ok_group(int g) { return g == 32 || g == 64 || g == 128; }
+
+qp_status check_shape(int batch, int Hq, int Hkv, int D) {
+  if (batch < 1 || Hq < 1 || Hkv < 1 || D < 1 || Hq % Hkv != 0) return QP_ERR_INVALID_ARG;
+  if ((D != 64 && D != 128) || Hq / Hkv > 8) return QP_ERR_UNSUPPORTED;
+  return QP_OK;
+}
+
+qp_status check_cache(const qp_cache* c, bool need_ptrs) {
+  if (!c) return QP_ERR_INVALID_ARG;
+  qp_status s = check_shape(c->batch, c->n_q_heads, c->n_kv_heads, c->head_dim);
+  if (s != QP_OK) return s;
+  if (!pow2_bits(c->bits) || !ok_group(c->group) || c->head_dim % c->group != 0) return QP_ERR_UNSUPPORTED;
+  if (c->n_keep < 1) return QP_ERR_INVALID_ARG;
+  if (c->bits < 16 && c->n_keep % c->group != 0) return QP_ERR_BUDGET;
+  if (need_ptrs) {
+    if (!c->k_codes || !c->v_codes) return QP_ERR_INVALID_ARG;
+    if (!aligned16(c->k_codes) || !aligned16(c->v_codes)) return QP_ERR_ALIGNMENT;
+    if (c->bits < 16) {
+      if (!c->k_scale || !c->k_zero || !c->v_scale || !c->v_zero) return QP_ERR_INVALID_ARG;
+      if (!aligned16(c->k_scale) || !aligned16(c->k_zero) || !aligned16(c->v_scale) || !aligned16(c->v_zero))
+        return QP_ERR_ALIGNMENT;
+    }
+  }
+  return QP_OK;
+}
+
+size_t decode_ws_bytes_for(const qp_cache& c, int chunk) {
+  const size_t splits = (size_t)(c.n_keep + chunk - 1) / chunk;
+  const size_t G = (size_t)(c.n_q_heads / c.n_kv_heads);
+  return (size_t)c.batch * c.n_kv_heads * splits * G * (size_t)(c.head_dim + 2) * sizeof(float);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* qp_status_string(qp_status s) {
+  switch (s) {
+    case QP_OK: return "ok";
+    case QP_ERR_INVALID_ARG: return "invalid argument";
+    case QP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case QP_ERR_BUDGET: return "budget cannot be met";
+    case QP_ERR_WORKSPACE: return "workspace too small";
+    case QP_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case QP_ERR_CUDA: return "CUDA launch failed";
+  }
+  return "unknown status";
+}
+
+qp_status qp_n_keep(int64_t budget_bits, int bits, int group, int L, int w, int32_t* n_keep) {
+  if (!n_keep || L < 2 || w < 1 || w >= L || budget_bits < 1) return QP_ERR_INVALID_ARG;
+  if (!pow2_bits(bits) || !ok_group(group)) return QP_ERR_UNSUPPORTED;
+  int64_t n = budget_bits / bits;
+  if (n > L) n = L;
+  if (n <= w) return QP_ERR_BUDGET;
+  if (bits < 16 && n % group != 0) return QP_ERR_BUDGET;
+  *n_keep = (int32_t)n;
+  return QP_OK;
+}
+
+qp_status qp_cache_layout(int batch, int n_q_heads, int n_kv_heads, int head_dim, int bits, int group, int n_keep,
+                          qp_cache* out) {
+  if (!out) return QP_ERR_INVALID_ARG;
+  qp_cache c;
+  std::memset(&c, 0, sizeof(c));
+  c.batch = batch; c.n_q_heads = n_q_heads; c.n_kv_heads = n_kv_heads; c.head_dim = head_dim;
+  c.bits = bits; c.group = group; c.n_keep = n_keep;
+  const qp_status s = check_cache(&c, false);
+  if (s != QP_OK) return s;
+  const size_t elems = (size_t)batch * n_kv_heads * n_keep * head_dim;
+  if (bits == 16) {
+    c.k_codes_bytes = c.v_codes_bytes = elems * 2;
+  } else {
+    c.k_codes_bytes = c.v_codes_bytes = elems * bits / 8;
+    c.k_meta_bytes = c.v_meta_bytes = elems / group * 2;
+  }
+  *out = c;
+  return QP_OK;
+}
+
+size_t qp_compress_workspace_bytes(int batch, int n_q_heads, int n_kv_heads, int head_dim, int L, int w) {
+  if (check_shape(batch, n_q_heads, n_kv_heads, head_dim) != QP_OK || w < 1 || w >= L) return 0;
+  return score_workspace(batch, n_q_heads, n_kv_heads, L, w).total;
+}
+
+size_t qp_decode_workspace_bytes(const qp_cache* cache) {
+  if (check_cache(cache, false) != QP_OK) return 0;
+  return decode_ws_bytes_for(*cache, 128);   // 128 tokens is the smallest split any launch uses
+}
+
+static qp_status check_score_args(const void* Q_win, const void* K, int batch, int Hq, int Hkv, int D, int L, int w,
+                                  int pool) {
+  if (!Q_win || !K) return QP_ERR_INVALID_ARG;
+  qp_status s = check_shape(batch, Hq, Hkv, D);
+  if (s != QP_OK) return s;
+  if (w < 1 || w >= L || pool < 1 || pool % 2 == 0) return QP_ERR_INVALID_ARG;
+  if (w > 64) return QP_ERR_UNSUPPORTED;
+  if (!aligned16(Q_win) || !aligned16(K)) return QP_ERR_ALIGNMENT;
+  return QP_OK;
+}
+
+qp_status qp_window_scores(const void* Q_win, const void* K, int batch, int n_q_heads, int n_kv_heads, int head_dim,
+                           int L, int w, int pool, float* scores, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+  qp_status s = check_score_args(Q_win, K, batch, n_q_heads, n_kv_heads, head_dim, L, w, pool);
+  if (s != QP_OK) return s;
+  if (!scores || !workspace) return QP_ERR_INVALID_ARG;
+  if (!aligned16(scores) || !aligned16(workspace)) return QP_ERR_ALIGNMENT;
+  if (workspace_bytes < qp_compress_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim, L, w))
+    return QP_ERR_WORKSPACE;
+  const ScoreDims d{batch, n_q_heads, n_kv_heads, head_dim, L, w, pool};
+  return launch_window_scores(Q_win, K, d, scores, workspace, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_select_topk(const float* scores, int batch, int n_kv_heads, int L, int w, int n_keep, int32_t* kept_idx,
+                         void* stream) {
+  if (!scores || !kept_idx || batch < 1 || n_kv_heads < 1 || w < 1 || w >= L) return QP_ERR_INVALID_ARG;
+  if (n_keep <= w || n_keep > L) return QP_ERR_BUDGET;
+  return launch_select_topk(scores, batch * n_kv_heads, L, w, n_keep, kept_idx,
+                            static_cast<cudaStream_t>(stream)) == cudaSuccess ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_gather_quantize(const void* K, const void* V, const int32_t* kept_idx, int L, const qp_cache* cache,
+                             void* stream) {
+  if (!K || !V || !kept_idx || L < 1) return QP_ERR_INVALID_ARG;
+  const qp_status s = check_cache(cache, true);
+  if (s != QP_OK) return s;
+  if (cache->n_keep > L) return QP_ERR_BUDGET;
+  if (!aligned16(K) || !aligned16(V)) return QP_ERR_ALIGNMENT;
+  return launch_gather_quantize(K, V, kept_idx, L, *cache, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_compress_layer(const void* K, const void* V, const void* Q_win, int batch, int n_q_heads, int n_kv_heads,
+                            int head_dim, int L, int w, int64_t budget_bits, int bits, int group, int pool,
+                            const qp_cache* cache, int32_t* kept_idx, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+  if (!V || !kept_idx || !workspace) return QP_ERR_INVALID_ARG;
+  qp_status s = check_score_args(Q_win, K, batch, n_q_heads, n_kv_heads, head_dim, L, w, pool);
+  if (s != QP_OK) return s;
+  int32_t n = 0;
+  s = qp_n_keep(budget_bits, bits, group, L, w, &n);
+  if (s != QP_OK) return s;
+  s = check_cache(cache, true);
+  if (s != QP_OK) return s;
+  if (cache->batch != batch || cache->n_q_heads != n_q_heads || cache->n_kv_heads != n_kv_heads ||
+      cache->head_dim != head_dim || cache->bits != bits || cache->group != group)
+    return QP_ERR_INVALID_ARG;
+  if (cache->n_keep != n) return QP_ERR_BUDGET;
+  if (!aligned16(V) || !aligned16(workspace)) return QP_ERR_ALIGNMENT;
+  const ScoreWorkspace sw = score_workspace(batch, n_q_heads, n_kv_heads, L, w);
+  if (workspace_bytes < sw.total) return QP_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* pooled = reinterpret_cast<float*>(static_cast<char*>(workspace) + sw.pooled);
+  const ScoreDims d{batch, n_q_heads, n_kv_heads, head_dim, L, w, pool};
+  if (launch_window_scores(Q_win, K, d, pooled, workspace, st) != cudaSuccess) return QP_ERR_CUDA;
+  if (launch_select_topk(pooled, batch * n_kv_heads, L, w, n, kept_idx, st) != cudaSuccess) return QP_ERR_CUDA;
+  if (launch_gather_quantize(K, V, kept_idx, L, *cache, st) != cudaSuccess) return QP_ERR_CUDA;
+  return QP_OK;
+}
+
+qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches, void* const* out,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !q || !caches || !out || !workspace) return QP_ERR_INVALID_ARG;
+  if (!aligned16(workspace)) return QP_ERR_ALIGNMENT;
+  const qp_cache& c0 = caches[0];
+  long long total_tokens = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const qp_status s = check_cache(&caches[l], true);
+    if (s != QP_OK) return s;
+    const qp_cache& c = caches[l];
+    if (c.batch != c0.batch || c.n_q_heads != c0.n_q_heads || c.n_kv_heads != c0.n_kv_heads ||
+        c.head_dim != c0.head_dim || c.bits != c0.bits || c.group != c0.group)
+      return QP_ERR_INVALID_ARG;
+    if (!q[l] || !out[l]) return QP_ERR_INVALID_ARG;
+    if (!aligned16(q[l]) || !aligned16(out[l])) return QP_ERR_ALIGNMENT;
+    total_tokens += (long long)c.batch * c.n_kv_heads * c.n_keep;
+  }
+  const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
+  DecTable tab;
+  tab.n_layers = n_layers;
+  tab.chunk = decode_chunk_tokens(d, total_tokens);
+  size_t need = 0;
+  int max_splits = 0, slot = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const qp_cache& c = caches[l];
+    const int splits = (c.n_keep + tab.chunk - 1) / tab.chunk;
+    tab.l[l] = DecLayer{c.k_codes, c.v_codes,
+                        static_cast<const __half*>(c.k_scale), static_cast<const __half*>(c.k_zero),
+                        static_cast<const __half*>(c.v_scale), static_cast<const __half*>(c.v_zero),
+                        q[l], out[l], c.n_keep, slot};
+    slot += c.batch * c.n_kv_heads * splits;
+    need += decode_ws_bytes_for(c, tab.chunk);
+    if (splits > max_splits) max_splits = splits;
+  }
+  if (workspace_bytes < need) return QP_ERR_WORKSPACE;
+  return launch_decode(tab, d, max_splits, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_decode_attn(const void* q, const qp_cache* cache, void* out, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+  if (!cache) return QP_ERR_INVALID_ARG;
+  const void* qs[1] = {q};
+  void* os[1] = {out};
+  return qp_decode_attn_layers(1, qs, cache, os, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,220 @@
+// S4 + S5: split-K decode attention over the packed pruned cache.
+//
+// Grid = (token splits, batch x KV heads, layers).  A thread block streams its token range
+// of one KV head once; the G query heads of that KV head share the stream.  Dequantisation
+// (code * scale + zero) happens in registers, the softmax is the usual running (max, sum)
+// form in the log2 domain, and each block leaves one partial (m, l, acc[D]) per query head.
+// A second kernel merges the partials of a (batch, query head) in a fixed order.
+// No block ever waits for another one.
+#include "qp_common.cuh"
+
+namespace qp {
+
+namespace {
+
+constexpr int DG_THREADS = 128;
+constexpr int DG_WARPS = 4;
+constexpr int MAXG = 8;
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Reference-shaped kernel: any supported (B, g, D, G).  One lane per token on the key side,
+// one lane per channel (stride 32) on the value side.
+template <int BITS>
+__global__ void __launch_bounds__(DG_THREADS)
+decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials) {
+  constexpr int PER = BITS < 16 ? 32 / BITS : 1;
+  constexpr uint32_t QMAX = BITS < 16 ? (1u << BITS) - 1u : 0u;
+  const int layer = blockIdx.z, bh = blockIdx.y, split = blockIdx.x;
+  const DecLayer& ly = tab.l[layer];
+  const int n = ly.n, t_begin = split * tab.chunk;
+  if (t_begin >= n) return;
+  const int t_end = min(n, t_begin + tab.chunk);
+  const int D = dm.D, G = dm.Hq / dm.Hkv, g = dm.group, wpg = g * BITS / 32, ngv = D / g;
+  const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_splits = (n + tab.chunk - 1) / tab.chunk;
+
+  __shared__ float sq[MAXG][128];
+  __shared__ float s_m[DG_WARPS][MAXG], s_l[DG_WARPS][MAXG];
+  __shared__ float s_acc[DG_WARPS][MAXG][128];
+
+  const float scale_log2 = 1.4426950408889634f * rsqrtf((float)D);
+  const uint16_t* q = static_cast<const uint16_t*>(ly.q) + (size_t)(b * dm.Hq + hk * G) * D;
+  for (int i = tid; i < G * D; i += DG_THREADS) sq[i / D][i % D] = bf16_bits_to_f32(q[i]) * scale_log2;
+  __syncthreads();
+
+  float m[MAXG], l[MAXG], acc[MAXG][4];
+#pragma unroll
+  for (int h = 0; h < MAXG; ++h) {
+    m[h] = -INFINITY;
+    l[h] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[h][i] = 0.f;
+  }
+
+  const uint32_t* kc = static_cast<const uint32_t*>(ly.kc);
+  const uint32_t* vc = static_cast<const uint32_t*>(ly.vc);
+  const uint16_t* k16 = static_cast<const uint16_t*>(ly.kc);
+  const uint16_t* v16 = static_cast<const uint16_t*>(ly.vc);
+
+  for (int tile = t_begin + warp * 32; tile < t_end; tile += DG_WARPS * 32) {
+    const int tok = tile + lane;
+    const bool valid = tok < t_end;
+    const int tk = valid ? tok : t_end - 1;
+    float lg[MAXG];
+#pragma unroll
+    for (int h = 0; h < MAXG; ++h) lg[h] = 0.f;
+    if constexpr (BITS < 16) {
+      const int u = tk / g, e = tk % g;
+      const size_t base = ((size_t)bh * (n / g) + u) * D;
+      const int wsel = e / PER, sh = (e % PER) * BITS;
+      for (int d = 0; d < D; ++d) {
+        const uint32_t c = (kc[(base + d) * wpg + wsel] >> sh) & QMAX;
+        const float kf = fmaf((float)c, __half2float(ly.ks[base + d]), __half2float(ly.kz[base + d]));
+#pragma unroll
+        for (int h = 0; h < MAXG; ++h)
+          if (h < G) lg[h] = fmaf(sq[h][d], kf, lg[h]);
+      }
+    } else {
+      const uint16_t* row = k16 + ((size_t)bh * n + tk) * D;
+      for (int d = 0; d < D; ++d) {
+        const float kf = bf16_bits_to_f32(row[d]);
+#pragma unroll
+        for (int h = 0; h < MAXG; ++h)
+          if (h < G) lg[h] = fmaf(sq[h][d], kf, lg[h]);
+      }
+    }
+    float p[MAXG];
+#pragma unroll
+    for (int h = 0; h < MAXG; ++h) {
+      p[h] = 0.f;
+      if (h < G) {
+        const float v = valid ? lg[h] : -INFINITY;
+        const float mnew = fmaxf(m[h], warp_max(v));      // finite: lane 0 of a tile is always valid
+        p[h] = valid ? exp2f(v - mnew) : 0.f;
+        const float corr = exp2f(m[h] - mnew);             // 0 on the first tile (m = -inf)
+        l[h] = l[h] * corr + warp_sum(p[h]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[h][i] *= corr;
+        m[h] = mnew;
+      }
+    }
+    const int nt = min(32, t_end - tile);
+    for (int tt = 0; tt < nt; ++tt) {
+      const int tok2 = tile + tt;
+      float vf[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int d = lane + 32 * i;
+        vf[i] = 0.f;
+        if (d < D) {
+          if constexpr (BITS < 16) {
+            const int e2 = d % g;
+            const size_t gi = ((size_t)bh * n + tok2) * ngv + d / g;
+            const uint32_t c = (vc[gi * wpg + e2 / PER] >> ((e2 % PER) * BITS)) & QMAX;
+            vf[i] = fmaf((float)c, __half2float(ly.vs[gi]), __half2float(ly.vz[gi]));
+          } else {
+            vf[i] = bf16_bits_to_f32(v16[((size_t)bh * n + tok2) * D + d]);
+          }
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < MAXG; ++h)
+        if (h < G) {
+          const float ph = __shfl_sync(0xffffffffu, p[h], tt);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) acc[h][i] = fmaf(ph, vf[i], acc[h][i]);
+        }
+    }
+  }
+
+  // combine the four warps, fixed order
+#pragma unroll
+  for (int h = 0; h < MAXG; ++h)
+    if (h < G) {
+      if (lane == 0) { s_m[warp][h] = m[h]; s_l[warp][h] = l[h]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (lane + 32 * i < D) s_acc[warp][h][lane + 32 * i] = acc[h][i];
+    }
+  __syncthreads();
+  const size_t slot = (size_t)ly.part_base + (size_t)bh * n_splits + split;
+  for (int idx = tid; idx < G * D; idx += DG_THREADS) {
+    const int h = idx / D, d = idx % D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int wp = 0; wp < DG_WARPS; ++wp) M = fmaxf(M, s_m[wp][h]);
+    float Ls = 0.f, A = 0.f;
+#pragma unroll
+    for (int wp = 0; wp < DG_WARPS; ++wp)
+      if (s_m[wp][h] != -INFINITY) {
+        const float f = exp2f(s_m[wp][h] - M);
+        Ls = fmaf(s_l[wp][h], f, Ls);
+        A = fmaf(s_acc[wp][h][d], f, A);
+      }
+    float* o = partials + (slot * G + h) * (size_t)(D + 2);
+    if (d == 0) { o[0] = M; o[1] = Ls; }
+    o[2 + d] = A;
+  }
+}
+
+// S5: log-sum-exp merge of the split partials of one (layer, batch, query head)
+__global__ void __launch_bounds__(128)
+decode_merge_kernel(const __grid_constant__ DecTable tab, const DecDims dm, const float* __restrict__ partials) {
+  const int layer = blockIdx.y, bq = blockIdx.x, d = threadIdx.x;
+  const DecLayer& ly = tab.l[layer];
+  const int D = dm.D, G = dm.Hq / dm.Hkv;
+  if (d >= D) return;
+  const int b = bq / dm.Hq, h = bq % dm.Hq, bh = b * dm.Hkv + h / G, hl = h % G;
+  const int n_splits = (ly.n + tab.chunk - 1) / tab.chunk;
+  const float* base = partials + (((size_t)ly.part_base + (size_t)bh * n_splits) * G + hl) * (size_t)(D + 2);
+  const size_t stride = (size_t)G * (D + 2);
+  float M = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) M = fmaxf(M, base[s * stride]);
+  float Ls = 0.f, A = 0.f;
+  for (int s = 0; s < n_splits; ++s) {
+    const float f = exp2f(base[s * stride] - M);
+    Ls = fmaf(base[s * stride + 1], f, Ls);
+    A = fmaf(base[s * stride + 2 + d], f, A);
+  }
+  static_cast<bf16*>(ly.out)[(size_t)bq * D + d] = __float2bfloat16_rn(__fdiv_rn(A, Ls));
+}
+
+}  // namespace
+
+int decode_chunk_tokens(const DecDims& d, long long total_tokens) {
+  // aim at about eight blocks per SM, in whole 128-token units
+  long long c = (total_tokens + 148 * 8 - 1) / (148 * 8);
+  c = (c + 127) / 128 * 128;
+  if (c < 128) c = 128;
+  if (c > 4096) c = 4096;
+  (void)d;
+  return (int)c;
+}
+
+cudaError_t launch_decode(const DecTable& tab, const DecDims& d, int max_splits, float* partials, cudaStream_t st) {
+  const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
+  switch (d.bits) {
+    case 2: decode_generic_kernel<2><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
+    case 4: decode_generic_kernel<4><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
+    case 8: decode_generic_kernel<8><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
+    case 16: decode_generic_kernel<16><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
+    default: return cudaErrorInvalidValue;
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  decode_merge_kernel<<<dim3(d.Bt * d.Hq, tab.n_layers), 128, 0, st>>>(tab, d, partials);
+  return cudaGetLastError();
+}
+
+}  // namespace qp

@@ -1,0 +1,275 @@
+"""Thin binding over the C-ABI CUDA library (``libqp.so``): argument marshalling only.
+
+Every function has the name and the meaning of the C entry point it forwards to
+(see ``include/qp.h``).  torch is used for device memory, pointers and the current
+stream; no step of the path runs in Python or on the CPU.  Loading fails loudly
+when the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqp.so")
+
+QP_OK = 0
+QP_MAX_LAYERS = 128
+STATUS_NAMES = {0: "QP_OK", 1: "QP_ERR_INVALID_ARG", 2: "QP_ERR_UNSUPPORTED", 3: "QP_ERR_BUDGET",
+                4: "QP_ERR_WORKSPACE", 5: "QP_ERR_ALIGNMENT", 6: "QP_ERR_CUDA"}
+
+EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_workspace_bytes",
+           "qp_decode_workspace_bytes", "qp_window_scores", "qp_select_topk", "qp_gather_quantize",
+           "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers"]
+
+
+class QpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({status_string(status)})")
+
+
+class qp_cache(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("bits", ctypes.c_int32), ("group", ctypes.c_int32),
+                ("n_keep", ctypes.c_int32), ("reserved_", ctypes.c_int32),
+                ("k_codes_bytes", ctypes.c_size_t), ("v_codes_bytes", ctypes.c_size_t),
+                ("k_meta_bytes", ctypes.c_size_t), ("v_meta_bytes", ctypes.c_size_t),
+                ("k_codes", ctypes.c_void_p), ("v_codes", ctypes.c_void_p),
+                ("k_scale", ctypes.c_void_p), ("k_zero", ctypes.c_void_p),
+                ("v_scale", ctypes.c_void_p), ("v_zero", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded CUDA library.  Raises if it is missing: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2412_12706_b200.build` (needs nvcc, sm_100a)")
+        L = ctypes.CDLL(LIB_PATH)
+        i, i64, p, sz = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
+        cp = ctypes.POINTER(qp_cache)
+        L.qp_status_string.restype = ctypes.c_char_p
+        L.qp_status_string.argtypes = [i]
+        L.qp_n_keep.restype = i
+        L.qp_n_keep.argtypes = [i64, i, i, i, i, ctypes.POINTER(ctypes.c_int32)]
+        L.qp_cache_layout.restype = i
+        L.qp_cache_layout.argtypes = [i, i, i, i, i, i, i, cp]
+        L.qp_compress_workspace_bytes.restype = sz
+        L.qp_compress_workspace_bytes.argtypes = [i, i, i, i, i, i]
+        L.qp_decode_workspace_bytes.restype = sz
+        L.qp_decode_workspace_bytes.argtypes = [cp]
+        L.qp_window_scores.restype = i
+        L.qp_window_scores.argtypes = [p, p, i, i, i, i, i, i, i, p, p, sz, p]
+        L.qp_select_topk.restype = i
+        L.qp_select_topk.argtypes = [p, i, i, i, i, i, p, p]
+        L.qp_gather_quantize.restype = i
+        L.qp_gather_quantize.argtypes = [p, p, p, i, cp, p]
+        L.qp_compress_layer.restype = i
+        L.qp_compress_layer.argtypes = [p, p, p, i, i, i, i, i, i, i64, i, i, i, cp, p, p, sz, p]
+        L.qp_decode_attn.restype = i
+        L.qp_decode_attn.argtypes = [p, cp, p, p, sz, p]
+        L.qp_decode_attn_layers.restype = i
+        L.qp_decode_attn_layers.argtypes = [i, ctypes.POINTER(p), cp, ctypes.POINTER(p), p, sz, p]
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != QP_OK:
+        raise QpError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: torch.Tensor | None) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def status_string(status: int) -> str:
+    return lib().qp_status_string(status).decode()
+
+
+def n_keep(budget_bits: int, bits: int, group: int, L: int, w: int) -> int:
+    out = ctypes.c_int32(0)
+    _check(lib().qp_n_keep(budget_bits, bits, group, L, w, ctypes.byref(out)), "qp_n_keep")
+    return out.value
+
+
+def cache_layout(batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, bits: int, group: int,
+                 n_keep_: int) -> qp_cache:
+    c = qp_cache()
+    _check(lib().qp_cache_layout(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_,
+                                 ctypes.byref(c)), "qp_cache_layout")
+    return c
+
+
+def compress_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim, L, w) -> int:
+    return int(lib().qp_compress_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim, L, w))
+
+
+def decode_workspace_bytes(cache: "Cache | qp_cache") -> int:
+    c = cache.desc if isinstance(cache, Cache) else cache
+    return int(lib().qp_decode_workspace_bytes(ctypes.byref(c)))
+
+
+@dataclass
+class Cache:
+    """Device buffers of one layer's packed cache plus the C descriptor that points at them."""
+    desc: qp_cache
+    k_codes: torch.Tensor
+    v_codes: torch.Tensor
+    k_scale: torch.Tensor | None
+    k_zero: torch.Tensor | None
+    v_scale: torch.Tensor | None
+    v_zero: torch.Tensor | None
+
+    @property
+    def nbytes(self) -> int:
+        d = self.desc
+        return d.k_codes_bytes + d.v_codes_bytes + 2 * d.k_meta_bytes + 2 * d.v_meta_bytes
+
+
+def alloc_cache(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_, device="cuda") -> Cache:
+    """Allocates the buffers of ``qp_cache_layout`` with torch and fills in the pointers."""
+    d = cache_layout(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_)
+    n, D, g = n_keep_, head_dim, group
+    if bits == 16:
+        kc = torch.empty((batch, n_kv_heads, n, D), dtype=torch.bfloat16, device=device)
+        vc = torch.empty_like(kc)
+        ks = kz = vs = vz = None
+    else:
+        wpg = g * bits // 32
+        kc = torch.empty((batch, n_kv_heads, n // g, D, wpg), dtype=torch.int32, device=device)
+        vc = torch.empty((batch, n_kv_heads, n, D // g, wpg), dtype=torch.int32, device=device)
+        ks = torch.empty((batch, n_kv_heads, n // g, D), dtype=torch.float16, device=device)
+        kz = torch.empty_like(ks)
+        vs = torch.empty((batch, n_kv_heads, n, D // g), dtype=torch.float16, device=device)
+        vz = torch.empty_like(vs)
+    assert kc.numel() * kc.element_size() == d.k_codes_bytes and vc.numel() * vc.element_size() == d.v_codes_bytes
+    d.k_codes, d.v_codes = _ptr(kc), _ptr(vc)
+    d.k_scale, d.k_zero, d.v_scale, d.v_zero = _ptr(ks), _ptr(kz), _ptr(vs), _ptr(vz)
+    return Cache(d, kc, vc, ks, kz, vs, vz)
+
+
+def _dims(K: torch.Tensor, Q_win: torch.Tensor):
+    Bt, Hkv, L, D = K.shape
+    _, Hq, w, _ = Q_win.shape
+    return Bt, Hq, Hkv, D, L, w
+
+
+def _dev_bf16(t: torch.Tensor) -> None:
+    assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+
+
+def window_scores(Q_win: torch.Tensor, K: torch.Tensor, pool: int = 7, workspace: torch.Tensor | None = None,
+                  scores: torch.Tensor | None = None) -> torch.Tensor:
+    _dev_bf16(Q_win); _dev_bf16(K)
+    Bt, Hq, Hkv, D, L, w = _dims(K, Q_win)
+    if scores is None:
+        scores = torch.empty((Bt, Hkv, L - w), dtype=torch.float32, device=K.device)
+    if workspace is None:
+        workspace = torch.empty(max(16, compress_workspace_bytes(Bt, Hq, Hkv, D, L, w)), dtype=torch.uint8,
+                                device=K.device)
+    _check(lib().qp_window_scores(_ptr(Q_win), _ptr(K), Bt, Hq, Hkv, D, L, w, pool, _ptr(scores),
+                                  _ptr(workspace), workspace.numel(), _stream()), "qp_window_scores")
+    return scores
+
+
+def select_topk(scores: torch.Tensor, L: int, w: int, n_keep_: int,
+                kept_idx: torch.Tensor | None = None) -> torch.Tensor:
+    assert scores.is_cuda and scores.dtype == torch.float32 and scores.is_contiguous()
+    Bt, Hkv, P = scores.shape
+    assert P == L - w
+    if kept_idx is None:
+        kept_idx = torch.empty((Bt, Hkv, n_keep_), dtype=torch.int32, device=scores.device)
+    _check(lib().qp_select_topk(_ptr(scores), Bt, Hkv, L, w, n_keep_, _ptr(kept_idx), _stream()),
+           "qp_select_topk")
+    return kept_idx
+
+
+def gather_quantize(K: torch.Tensor, V: torch.Tensor, kept_idx: torch.Tensor, cache: Cache) -> Cache:
+    _dev_bf16(K); _dev_bf16(V)
+    assert kept_idx.is_cuda and kept_idx.dtype == torch.int32 and kept_idx.is_contiguous()
+    _check(lib().qp_gather_quantize(_ptr(K), _ptr(V), _ptr(kept_idx), K.shape[2], ctypes.byref(cache.desc),
+                                    _stream()), "qp_gather_quantize")
+    return cache
+
+
+def compress_layer(K: torch.Tensor, V: torch.Tensor, Q_win: torch.Tensor, budget_bits: int, bits: int,
+                   group: int = 32, pool: int = 7, cache: Cache | None = None,
+                   kept_idx: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    """qp_compress_layer: returns (cache, kept_idx).  Buffers are allocated with torch when not given."""
+    _dev_bf16(K); _dev_bf16(V); _dev_bf16(Q_win)
+    Bt, Hq, Hkv, D, L, w = _dims(K, Q_win)
+    n = n_keep(budget_bits, bits, group, L, w)
+    if cache is None:
+        cache = alloc_cache(Bt, Hq, Hkv, D, bits, group, n, K.device)
+    if kept_idx is None:
+        kept_idx = torch.empty((Bt, Hkv, n), dtype=torch.int32, device=K.device)
+    if workspace is None:
+        workspace = torch.empty(max(16, compress_workspace_bytes(Bt, Hq, Hkv, D, L, w)), dtype=torch.uint8,
+                                device=K.device)
+    _check(lib().qp_compress_layer(_ptr(K), _ptr(V), _ptr(Q_win), Bt, Hq, Hkv, D, L, w, budget_bits, bits,
+                                   group, pool, ctypes.byref(cache.desc), _ptr(kept_idx), _ptr(workspace),
+                                   workspace.numel(), _stream()), "qp_compress_layer")
+    return cache, kept_idx
+
+
+def decode_attn(q: torch.Tensor, cache: Cache, out: torch.Tensor | None = None,
+                workspace: torch.Tensor | None = None) -> torch.Tensor:
+    _dev_bf16(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = torch.empty(max(16, decode_workspace_bytes(cache)), dtype=torch.uint8, device=q.device)
+    _check(lib().qp_decode_attn(_ptr(q), ctypes.byref(cache.desc), _ptr(out), _ptr(workspace),
+                                workspace.numel(), _stream()), "qp_decode_attn")
+    return out
+
+
+class LayerBatch:
+    """Marshalled host arrays for ``qp_decode_attn_layers`` (built once, reused every step)."""
+
+    def __init__(self, qs: list[torch.Tensor], caches: list[Cache], outs: list[torch.Tensor],
+                 workspace: torch.Tensor | None = None):
+        n = len(caches)
+        assert 1 <= n <= QP_MAX_LAYERS and len(qs) == n and len(outs) == n
+        self.n = n
+        self.keep = (qs, caches, outs)
+        self.q_arr = (ctypes.c_void_p * n)(*[t.data_ptr() for t in qs])
+        self.out_arr = (ctypes.c_void_p * n)(*[t.data_ptr() for t in outs])
+        self.cache_arr = (qp_cache * n)(*[c.desc for c in caches])
+        if workspace is None:
+            nbytes = sum(decode_workspace_bytes(c) for c in caches)
+            workspace = torch.empty(max(16, nbytes), dtype=torch.uint8, device=qs[0].device)
+        self.workspace = workspace
+
+
+def decode_attn_layers(batch: LayerBatch) -> None:
+    _check(lib().qp_decode_attn_layers(batch.n, batch.q_arr, batch.cache_arr, batch.out_arr,
+                                       _ptr(batch.workspace), batch.workspace.numel(), _stream()),
+           "qp_decode_attn_layers")
+
+
+# the C entry points under their own names
+qp_status_string = status_string
+qp_n_keep = n_keep
+qp_cache_layout = cache_layout
+qp_compress_workspace_bytes = compress_workspace_bytes
+qp_decode_workspace_bytes = decode_workspace_bytes
+qp_window_scores = window_scores
+qp_select_topk = select_topk
+qp_gather_quantize = gather_quantize
+qp_compress_layer = compress_layer
+qp_decode_attn = decode_attn
+qp_decode_attn_layers = decode_attn_layers
