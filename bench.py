@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized-pruning hot path on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: the
+prefill-side compression (window scores -> top-k -> gather+quantize+pack) of every layer,
+followed by every decode step's attention over the packed cache of every layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is the decode-attention throughput in GB/s of
+algorithmic packed-cache bytes (codes + scale/zero) with everything resident in HBM; `e2e`
+is the same quantity with the step's inputs coming from pinned host memory and the results
+going back, through the same C-ABI calls.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2412_12706_b200 import shard, synth
+
+METRIC = "decode_attn_hbm_gbs"
+UNIT = "GB/s"
+DEFAULT_WORKLOAD = synth.LLAMA8B_8K.name
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM traffic of the dominant (decode) kernel from an ncu capture, valid only for the exact
+# kernel source it was taken on: {"sha256": <hash of csrc/qp_decode.cu>, "workload": name,
+# "bytes_per_launch": dram__bytes_read.sum + dram__bytes_write.sum}
+NCU_TRAFFIC: dict = {}
+
+KERNELS_PER_COMPRESS = 6      # sweep 1, row-stat merge, sweep 2, pool, top-k, gather+quantize
+KERNELS_PER_DECODE_CALL = 2   # split-K attention, merge
+
+
+def packed_bytes(wl: synth.Workload, layer: int) -> int:
+    """Algorithmic bytes one decode step reads for one layer: codes plus fp16 scale and zero."""
+    n, b, g = wl.n_keep(layer), wl.bits, wl.group
+    elems = wl.batch * wl.n_kv_heads * n * wl.head_dim * 2            # K and V
+    return elems * 2 if b == 16 else elems * (b + 32 // g) // 8
+
+
+def hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[5:9]):
+                if val.strip().lower() == "active":
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- reference arm
+
+def oracle_sample(wl: synth.Workload, steps: int, warmup: int):
+    """The CPU oracle, as it stands, on a bounded sample of the workload (sized for roughly
+    10-20 s of host time per step): the first few layers of one sequence, each compressed once
+    and attended for `dec` decode steps."""
+    from oracle import qp_oracle as orc
+    u16 = synth.bits_u16
+    dec = 8
+    if wl.batch > 1:                                   # large configurations: one batch entry only
+        wl = synth.dataclasses.replace(wl, batch=1)
+    macs = wl.n_kv_heads * (wl.n_q_heads // wl.n_kv_heads) * wl.w * wl.L * wl.head_dim
+    n_lay = max(1, min(wl.n_layers, 16, int(2e10 // macs)))
+    layers = []
+    for l in range(n_lay):
+        k, v = synth.make_kv(wl, l)
+        layers.append((u16(k), u16(v), u16(synth.make_q_win(wl, l)),
+                       [u16(synth.make_q_dec(wl, l, s)) for s in range(dec)]))
+    t_comp, t_dec = [], []
+    for it in range(warmup + steps):
+        tc = td = 0.0
+        for l, (kb, vb, qwb, qs) in enumerate(layers):
+            t0 = time.perf_counter()
+            pk, kept, _ = orc.compress_layer(kb, vb, qwb, wl.layer_budget_bits(l), wl.bits, wl.group, wl.pool)
+            t1 = time.perf_counter()
+            for s in range(dec):
+                kd, vd = orc.dequantize(pk, wl.head_dim)    # the paper's decode dequantizes, then attends
+                orc.decode(qs[s], kd, vd)
+            t2 = time.perf_counter()
+            tc += t1 - t0; td += t2 - t1
+        if it >= warmup:
+            t_comp.append(tc); t_dec.append(td)
+    bytes_dec = sum(packed_bytes(wl, l) for l in range(n_lay)) * dec
+    return {
+        "decode_gbs": bytes_dec / statistics.mean(t_dec) / 1e9,
+        "compress_tokens_per_s": wl.batch * wl.L / (statistics.mean(t_comp) / n_lay * wl.n_layers),
+        "ms_per_step": 1e3 * (statistics.mean(t_comp) + statistics.mean(t_dec)),
+        "cores": orc.num_threads(),
+        "sample": f"layers 0..{n_lay - 1} of one sequence (batch {wl.batch}): 1 compress_layer + {dec} decode "
+                  f"steps per layer per step (of {wl.n_layers} layers x {wl.decode_steps} decode steps); "
+                  f"compress tokens/s scaled to all {wl.n_layers} layers",
+    }
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    r = oracle_sample(wl, max(1, args.steps), max(0, min(args.warmup, 1)))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": r["decode_gbs"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "sample": r["sample"]},
+        "compress_tokens_per_s": r["compress_tokens_per_s"],
+        "cpu_baseline": {"value": r["decode_gbs"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
+                         "sample": r["sample"]},
+        "e2e": {"value": r["decode_gbs"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- GPU arm
+
+def run_gpu(args, wl):
+    from paper_2412_12706_b200 import qp
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    qp.lib()
+
+    n_seq, n_layers, n_dec = args.sequences, wl.n_layers, wl.decode_steps
+    Bt, Hq, Hkv, D, L, w = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.L, wl.w
+    stream = torch.cuda.current_stream()
+
+    # ---- inputs resident in HBM: every rank and every sequence has its own seed
+    seqs = []
+    for s in range(n_seq):
+        wls = synth.dataclasses.replace(wl, seed=shard.sequence_seed(wl.seed, rank, n_seq, s))
+        Ks, Vs, Qs = [], [], []
+        for l in range(n_layers):
+            k, v = synth.make_kv(wls, l, device=dev)
+            Ks.append(k); Vs.append(v); Qs.append(synth.make_q_win(wls, l, device=dev))
+        qdec = torch.stack([torch.stack([synth.make_q_dec(wls, l, t, device=dev) for l in range(n_layers)])
+                            for t in range(n_dec)])              # [n_dec, n_layers, Bt, Hq, D]
+        seqs.append({"K": Ks, "V": Vs, "Qw": Qs, "qdec": qdec})
+    ws_c = torch.empty(qp.compress_workspace_bytes(Bt, Hq, Hkv, D, L, w), dtype=torch.uint8, device=dev)
+    for sq in seqs:
+        sq["cache"] = [qp.alloc_cache(Bt, Hq, Hkv, D, wl.bits, wl.group, wl.n_keep(l), dev) for l in range(n_layers)]
+        sq["kept"] = [torch.empty((Bt, Hkv, wl.n_keep(l)), dtype=torch.int32, device=dev) for l in range(n_layers)]
+        sq["out"] = torch.empty((n_layers, Bt, Hq, D), dtype=torch.bfloat16, device=dev)
+        ws_d = torch.empty(sum(qp.decode_workspace_bytes(c) for c in sq["cache"]), dtype=torch.uint8, device=dev)
+        sq["ws_d"] = ws_d
+        sq["batches"] = [qp.LayerBatch([sq["qdec"][t, l] for l in range(n_layers)], sq["cache"],
+                                       [sq["out"][l] for l in range(n_layers)], ws_d) for t in range(n_dec)]
+
+    dec_bytes_step = n_seq * n_dec * sum(packed_bytes(wl, l) for l in range(n_layers))
+    dec_bytes_call = sum(packed_bytes(wl, l) for l in range(n_layers))
+    ctx_tokens_step = n_seq * Bt * L
+
+    def compress_all():
+        for sq in seqs:
+            for l in range(n_layers):
+                qp.compress_layer(sq["K"][l], sq["V"][l], sq["Qw"][l], wl.layer_budget_bits(l), wl.bits, wl.group,
+                                  wl.pool, sq["cache"][l], sq["kept"][l], ws_c)
+
+    def decode_all(call_events=None):
+        for t in range(n_dec):
+            for sq in seqs:          # consecutive launches touch different sequences' caches
+                if call_events is not None:
+                    e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+                qp.decode_attn_layers(sq["batches"][t])
+                if call_events is not None:
+                    e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
+                    call_events.append((e0, e1))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        compress_all(); decode_all()
+    barrier()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    marks, call_events = [], []
+    barrier()
+    t_begin = ev(); t_begin.record(stream)
+    for _ in range(args.steps):
+        a, b, c = ev(), ev(), ev()
+        a.record(stream); compress_all(); b.record(stream); decode_all(call_events); c.record(stream)
+        marks.append((a, b, c))
+    t_end = ev(); t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+
+    total_ms = t_begin.elapsed_time(t_end)
+    comp_ms = sum(a.elapsed_time(b) for a, b, c in marks)
+    dec_ms = sum(b.elapsed_time(c) for a, b, c in marks)
+    call_ms = statistics.mean(e0.elapsed_time(e1) for e0, e1 in call_events)
+
+    # ---- end to end: host buffers in, host buffers out, through the same calls
+    e2e = run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step) if not args.no_e2e else None
+
+    def allmax(x: float) -> float:
+        return shard.max_over_ranks(x, dist, dev)
+
+    total_ms, comp_ms, dec_ms = allmax(total_ms), allmax(comp_ms), allmax(dec_ms)
+    e2e_dec_ms = allmax(e2e["dec_ms"]) if e2e else None
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    steps = args.steps
+    value = shard.whole_job_throughput(dec_bytes_step * steps, world, dec_ms * 1e-3) / 1e9
+    peak, peak_kind = hbm_peak()
+    achieved = dec_bytes_call / (call_ms * 1e-3) / 1e9
+    sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2412_12706_b200", "csrc", "qp_decode.cu"), "rb").read()).hexdigest()
+    traffic = NCU_TRAFFIC.get("bytes_per_launch") if NCU_TRAFFIC.get("sha256") == sha and \
+        NCU_TRAFFIC.get("workload") == wl.name else None
+    cpu = oracle_sample(wl, 1, 0) if world == 1 and not args.no_cpu_baseline else None
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "layers": n_layers, "batch": Bt, "q_heads": Hq, "kv_heads": Hkv,
+                   "head_dim": D, "context": L, "window": w, "bits": wl.bits, "group": wl.group,
+                   "n_keep": [wl.n_keep(0), wl.n_keep(n_layers - 1)], "decode_steps": n_dec,
+                   "sequences_per_gpu": n_seq, "parallelism": f"replicas x{world}, no collective",
+                   "decode_api": "qp_decode_attn_layers (one launch pair per decode step over all layers)",
+                   "l2": f"decode rotates over {n_seq} independent sequences "
+                         f"({n_seq * dec_bytes_call / 1e6:.0f} MB of packed cache) so consecutive launches "
+                         f"read different data; compress inputs {2 * n_seq * n_layers * Bt * Hkv * L * D * 2 / 1e9:.2f} GB"},
+        "compress_tokens_per_s": world * ctx_tokens_step * steps / (comp_ms * 1e-3),
+        "compress_ms_per_layer": comp_ms / (steps * n_seq * n_layers),
+        "decode_us_per_call": call_ms * 1e3,
+        "decode_phase_ms_per_step": dec_ms / steps,
+        "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
+        "roofline": {"bound": "hbm", "kernel": "decode attention (split-K + merge)", "achieved": achieved,
+                     "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": traffic},
+        "e2e": None if e2e is None else {
+            "value": world * dec_bytes_step * e2e["steps"] / (e2e_dec_ms * 1e-3) / 1e9, "unit": UNIT,
+            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+            "ms_per_step": e2e["total_ms"] / e2e["steps"],
+            "compress_tokens_per_s": world * ctx_tokens_step * e2e["steps"] / (e2e["comp_ms"] * 1e-3)},
+        "gpu_launches": steps * n_seq * (n_layers * KERNELS_PER_COMPRESS + n_dec * KERNELS_PER_DECODE_CALL),
+        "clocks": clocks,
+    }
+    if cpu is not None:
+        line["cpu_baseline"] = {"value": cpu["decode_gbs"], "unit": UNIT, "cores": cpu["cores"], "kind": "oracle",
+                                "sample": cpu["sample"], "compress_tokens_per_s": cpu["compress_tokens_per_s"]}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step):
+    """Same step, but every input starts in pinned host memory and every decode output is read
+    back: K, V, Q_win are uploaded layer by layer before qp_compress_layer, each decode step
+    uploads its queries and downloads its outputs."""
+    n_layers, n_dec = wl.n_layers, wl.decode_steps
+    hK = [[k.cpu().pin_memory() for k in sq["K"]] for sq in seqs]
+    hV = [[v.cpu().pin_memory() for v in sq["V"]] for sq in seqs]
+    hQ = [[q.cpu().pin_memory() for q in sq["Qw"]] for sq in seqs]
+    hq = [sq["qdec"].cpu().pin_memory() for sq in seqs]
+    hout = [torch.empty((n_dec,) + tuple(sq["out"].shape), dtype=torch.bfloat16).pin_memory() for sq in seqs]
+    dK, dV, dQ = torch.empty_like(seqs[0]["K"][0]), torch.empty_like(seqs[0]["V"][0]), torch.empty_like(seqs[0]["Qw"][0])
+    dq = [torch.empty_like(sq["qdec"][0]) for sq in seqs]
+    batches = [qp.LayerBatch([dq[i][l] for l in range(n_layers)], sq["cache"],
+                             [sq["out"][l] for l in range(n_layers)], sq["ws_d"]) for i, sq in enumerate(seqs)]
+    h2d = sum(t.numel() * 2 for per in (hK, hV, hQ) for s in per for t in s) + sum(t.numel() * 2 for t in hq)
+    d2h = sum(t.numel() * 2 for t in hout)
+
+    def step():
+        a = torch.cuda.Event(enable_timing=True); a.record(stream)
+        for i, sq in enumerate(seqs):
+            for l in range(n_layers):
+                dK.copy_(hK[i][l], non_blocking=True); dV.copy_(hV[i][l], non_blocking=True)
+                dQ.copy_(hQ[i][l], non_blocking=True)
+                qp.compress_layer(dK, dV, dQ, wl.layer_budget_bits(l), wl.bits, wl.group, wl.pool,
+                                  sq["cache"][l], sq["kept"][l], ws_c)
+        b = torch.cuda.Event(enable_timing=True); b.record(stream)
+        for t in range(n_dec):
+            for i, sq in enumerate(seqs):
+                dq[i].copy_(hq[i][t], non_blocking=True)
+                qp.decode_attn_layers(batches[i])
+                hout[i][t].copy_(sq["out"], non_blocking=True)
+        c = torch.cuda.Event(enable_timing=True); c.record(stream)
+        return a, b, c
+
+    step(); torch.cuda.synchronize()
+    k = max(1, min(args.steps, 3))
+    marks = [step() for _ in range(k)]
+    torch.cuda.synchronize()
+    return {"steps": k, "h2d": h2d, "d2h": d2h,
+            "comp_ms": sum(a.elapsed_time(b) for a, b, c in marks),
+            "dec_ms": sum(b.elapsed_time(c) for a, b, c in marks),
+            "total_ms": sum(a.elapsed_time(c) for a, b, c in marks)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="qp", choices=["qp", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--sequences", type=int, default=4,
+                    help="independent sequences per GPU (their packed caches together exceed L2)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    args = ap.parse_args()
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback "
+                             "(use --impl reference for the CPU oracle)")
+        run_gpu(args, wl)
+
+
+if __name__ == "__main__":
+    main()
