@@ -166,6 +166,30 @@ qp_status qp_decode_attn(const void* q, const qp_cache* cache /* host */, void* 
 qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches,
                                 void* const* out, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Decode attention without any caller-supplied scratch.  (The paper has no counterpart to this
+ * call; it exists for integration reasons only.)  Some hosts of this library cannot give it
+ * scratch memory: a serving process that hands all device memory to its own arena at start-up,
+ * so that a later cudaMalloc fails or is forbidden by policy; a latency-critical decode loop that
+ * may not risk the device-wide synchronisation an allocation can cause; a plugin interface that
+ * passes tensors in and out but offers no way to request temporaries.  For them the split
+ * partials of qp_decode_attn live in an array of QP_STATIC_SCRATCH_BYTES that is part of the
+ * library image: every GPU on which the library is loaded holds these bytes until the process
+ * exits.
+ *
+ * Same computation and result as qp_decode_attn(q, cache, out, ...); q, out bf16 [Bt,Hq,D] device.
+ * Returns QP_ERR_WORKSPACE, before launching anything, when this cache needs more scratch than
+ * QP_STATIC_SCRATCH_BYTES (sum over batch x KV heads x token splits x G of (D+2) floats): use
+ * qp_decode_attn with your own workspace then.  It calls no cudaMalloc/cudaFree and no allocating
+ * library routine.  The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  All calls on a device share
+ * the one array and it keeps the previous call's contents (nothing in it needs clearing: each
+ * call writes every record it later reads), so two calls whose kernels can overlap on the GPU,
+ * e.g. on different streams, race on it; serialise them on one stream or with events.
+ */
+#define QP_STATIC_SCRATCH_BYTES (4u << 20)
+qp_status qp_decode_attn_static(const void* q, const qp_cache* cache /* host */, void* out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

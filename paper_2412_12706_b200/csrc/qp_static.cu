@@ -1,0 +1,52 @@
+// qp_decode_attn_static: decode attention for callers that cannot allocate device memory.
+//
+// The split-K decode kernels need scratch for the per-split partial results.  The other
+// entry points take that scratch from the caller; this one keeps it in a fixed array that is
+// part of the library image, so the caller passes only inputs and outputs.
+#include "qp_common.cuh"
+
+namespace {
+
+// Scratch shared by every call on a device.  It lives in each GPU's memory from the moment the
+// library is loaded on that GPU until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[QP_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+// Device address of g_static_scratch per CUDA device.  The array's name is only a host-side
+// handle in host code; the address a kernel can use must be asked for, with that device current.
+void* g_scratch_addr[kMaxDevices] = {};
+
+qp_status static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return QP_ERR_CUDA;
+  if (!g_scratch_addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return QP_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  *out = g_scratch_addr[dev];
+  return QP_OK;
+}
+
+}  // namespace
+
+extern "C" qp_status qp_decode_attn_static(const void* q, const qp_cache* cache, void* out, void* stream) {
+  if (!cache) return QP_ERR_INVALID_ARG;
+  // Scratch this cache needs: one (max, sum, acc[D]) record per (batch, KV head, split, query head
+  // of the group), with the split size the decode launch will choose for this much work.
+  const size_t coarse = qp_decode_workspace_bytes(cache);
+  if (coarse == 0) return QP_ERR_INVALID_ARG;   // invalid descriptor
+  const qp::DecDims d{cache->batch, cache->n_q_heads, cache->n_kv_heads, cache->head_dim, cache->bits, cache->group};
+  const long long tokens = (long long)cache->batch * cache->n_kv_heads * cache->n_keep;
+  const int chunk = qp::decode_chunk_tokens(d, tokens);
+  const size_t splits = (size_t)(cache->n_keep + chunk - 1) / chunk;
+  const size_t need = (size_t)cache->batch * cache->n_kv_heads * splits * (size_t)(cache->n_q_heads / cache->n_kv_heads) *
+                      (size_t)(cache->head_dim + 2) * sizeof(float);
+  if (need > (size_t)QP_STATIC_SCRATCH_BYTES) return QP_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  const qp_status s = static_scratch(&scratch);
+  if (s != QP_OK) return s;
+  // Every partial record that the merge reads is written first by the attention kernel of the same
+  // call, so nothing in the array has to start at zero.
+  return qp_decode_attn(q, cache, out, scratch, QP_STATIC_SCRATCH_BYTES, stream);
+}

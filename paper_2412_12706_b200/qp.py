@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "QP_OK", 1: "QP_ERR_INVALID_ARG", 2: "QP_ERR_UNSUPPORTED", 3:
 
 EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_workspace_bytes",
            "qp_decode_workspace_bytes", "qp_window_scores", "qp_select_topk", "qp_gather_quantize",
-           "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers"]
+           "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static"]
 
 
 class QpError(RuntimeError):
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.qp_decode_attn.argtypes = [p, cp, p, p, sz, p]
         L.qp_decode_attn_layers.restype = i
         L.qp_decode_attn_layers.argtypes = [i, ctypes.POINTER(p), cp, ctypes.POINTER(p), p, sz, p]
+        L.qp_decode_attn_static.restype = i
+        L.qp_decode_attn_static.argtypes = [p, cp, p, p]
         _lib = L
     return _lib
 
@@ -261,6 +263,26 @@ def decode_attn_layers(batch: LayerBatch) -> None:
            "qp_decode_attn_layers")
 
 
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def decode_attn_static(q: torch.Tensor, cache: Cache, out: torch.Tensor | None = None) -> torch.Tensor:
+    """qp_decode_attn_static: decode attention whose split partials live in the library's built-in
+    scratch array, for hosts that cannot hand the library any temporary device memory.  Only
+    ``out`` is allocated here (by torch) when the caller passes none; the C call allocates nothing.
+    Raises QpError(QP_ERR_WORKSPACE) when the cache needs more than STATIC_SCRATCH_BYTES of scratch.
+    Calls on one device share that array: do not let two of them overlap on the GPU."""
+    _dev_bf16(q)
+    if out is None:
+        out = torch.empty_like(q)
+    st = lib().qp_decode_attn_static(_ptr(q), ctypes.byref(cache.desc), _ptr(out), _stream())
+    if st == 4:
+        raise QpError(st, f"qp_decode_attn_static: this cache needs more than the built-in "
+                          f"{STATIC_SCRATCH_BYTES} bytes of scratch; use qp_decode_attn with a workspace")
+    _check(st, "qp_decode_attn_static")
+    return out
+
+
 # the C entry points under their own names
 qp_status_string = status_string
 qp_n_keep = n_keep
@@ -273,3 +295,4 @@ qp_gather_quantize = gather_quantize
 qp_compress_layer = compress_layer
 qp_decode_attn = decode_attn
 qp_decode_attn_layers = decode_attn_layers
+qp_decode_attn_static = decode_attn_static
