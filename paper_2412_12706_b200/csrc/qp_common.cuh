@@ -101,5 +101,9 @@ struct DecDims {
 };
 int decode_chunk_tokens(const DecDims& d, long long total_tokens_per_bh_sum);
 cudaError_t launch_decode(const DecTable& tab, const DecDims& d, int max_splits, float* partials, cudaStream_t st);
+// tensor-core split-K kernel (writes the same partial records as the generic one)
+bool decode_mma_supported(const DecDims& d);
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, int max_splits, float* partials,
+                              cudaStream_t st);
 
 }  // namespace qp

@@ -204,6 +204,12 @@ int decode_chunk_tokens(const DecDims& d, long long total_tokens) {
 
 cudaError_t launch_decode(const DecTable& tab, const DecDims& d, int max_splits, float* partials, cudaStream_t st) {
   const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
+  if (decode_mma_supported(d)) {
+    const cudaError_t e = launch_decode_mma(tab, d, max_splits, partials, st);
+    if (e != cudaSuccess) return e;
+    decode_merge_kernel<<<dim3(d.Bt * d.Hq, tab.n_layers), 128, 0, st>>>(tab, d, partials);
+    return cudaGetLastError();
+  }
   switch (d.bits) {
     case 2: decode_generic_kernel<2><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
     case 4: decode_generic_kernel<4><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;

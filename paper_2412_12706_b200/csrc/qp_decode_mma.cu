@@ -1,0 +1,389 @@
+// S4 on tensor cores: split-K decode attention that keeps the packed codes packed until they
+// sit in MMA operand registers.
+//
+// Why tensor cores on an HBM-bound kernel: per byte of 4-bit cache there are 1.6 codes and each
+// code needs one FMA per query head of the GQA group on the key side (and again on the value
+// side).  On the fp32 pipes that is more issue slots than the SM has per byte it can fetch, so a
+// scalar kernel is instruction-bound far below the memory roofline.  Here the multiply-adds go
+// through mma.sync (m16n8k16, f16 operands, f32 accumulate, operands straight from registers);
+// what is left per code on the integer pipe is about 0.6 instructions of mask/shift.
+//
+// Mapping (group g = 32, so one tile = 32 tokens = one key group):
+//   keys   logit2[tok][h] = sum_d code[tok][d] * (q'[h][d] * s[d])  +  sum_d q'[h][d] * z[d]
+//          A = codes, rows = tokens, k = channels;  B = q' * scale folded per tile (f16);
+//          the zero-point term is a second small MMA whose A rows all hold z.
+//   values out[h][d] = sum_tok code[tok][d] * (p[h][tok] * s[tok][v])  +  sum_tok p[h][tok] * z[tok][v]
+//          A = codes, rows = channels, k = tokens;  B = p * scale per channel group v (f16);
+//          zero-point term: A rows = v, one MMA per 16 tokens.
+// q' = q * log2(e)/sqrt(D), softmax in the log2 domain.
+//
+// Codes become f16 operands without any conversion: a 16-bit lane holding a small integer c is
+// the f16 number c * 2^-24 (subnormals and the first binade are equally spaced), so
+// (word & 0x000f000f) is already a pair of f16 values; (word & 0x00f000f0) is the same scaled by
+// 16.  The power-of-two factors are undone once, on the f32 accumulators.
+// The packed layout stores a group's codes along the quantisation group (tokens for keys,
+// channels for values) while an MMA register pairs two elements along the contraction; the
+// transposing ldmatrix fetches 16-bit units of two different rows into one register, which is
+// exactly that pairing.  Shared-memory rows are XOR-swizzled so these loads are conflict-free.
+#include "qp_common.cuh"
+
+namespace qp {
+
+namespace {
+
+constexpr int DM_WARPS = 4;
+constexpr int DM_THREADS = DM_WARPS * 32;
+constexpr int DM_STAGES = 3;
+constexpr int SP_STRIDE = 80;            // bytes per column of the per-warp P buffer (8 columns)
+constexpr int SP_BYTES = 8 * SP_STRIDE;
+
+// byte offsets of one 32-token tile in shared memory, 4-bit codes, g = 32
+template <int D>
+struct Tile4 {
+  static constexpr int KC = 0;                    // D rows of 16 B: one channel, 32 tokens
+  static constexpr int KS = KC + D * 16;          // D halves
+  static constexpr int KZ = KS + D * 2;
+  static constexpr int VC = KZ + D * 2;           // 32 token rows of D/2 bytes
+  static constexpr int VS = VC + 16 * D;          // 32 x (D/32) halves
+  static constexpr int VZ = VS + 2 * D;
+  static constexpr int BYTES = VZ + 2 * D;
+};
+
+__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.f16x2 %0, %1, %2;\n" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts64(uint32_t a, uint32_t x, uint32_t y) {
+  asm volatile("st.shared.v2.u32 [%0], {%1,%2};\n" ::"r"(a), "r"(x), "r"(y));
+}
+
+constexpr uint32_t M0 = 0x000f000fu;   // code in bits 0..3 of each half: value c * 2^-24
+constexpr uint32_t M1 = 0x00f000f0u;   // code in bits 4..7 of each half: value c * 2^-20
+constexpr float C24 = 16777216.0f, C20 = 1048576.0f;
+
+template <int D>
+__global__ void __launch_bounds__(DM_THREADS, 3)
+decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials) {
+  using TL = Tile4<D>;
+  constexpr int NC = D / 32;       // ldmatrix.x4 calls over the channels of a key tile = value groups per token
+  constexpr int NPAIR = D / 8;     // channel pairs owned by one lane on the key side (D/4 channels)
+  extern __shared__ __align__(128) unsigned char smem[];
+
+  const int layer = blockIdx.z, bh = blockIdx.y, split = blockIdx.x;
+  const DecLayer& ly = tab.l[layer];
+  const int n = ly.n, t_begin = split * tab.chunk;
+  if (t_begin >= n) return;
+  const int t_end = min(n, t_begin + tab.chunk);
+  const int tile_begin = t_begin >> 5, n_tiles = (t_end - t_begin) >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int G = dm.Hq / dm.Hkv, b = bh / dm.Hkv, hk = bh % dm.Hkv;
+  const int n_splits = (n + tab.chunk - 1) / tab.chunk;
+
+  unsigned char* wsm = smem + warp * (DM_STAGES * TL::BYTES + SP_BYTES);
+  const uint32_t wsm_u = smem_u32(wsm);
+  const uint32_t sP = wsm_u + DM_STAGES * TL::BYTES;
+
+  // B-side query fragments: column g of the MMAs is query head g of this KV head (columns >= G are 0);
+  // this lane holds the D/4 channels [t*D/4, (t+1)*D/4) as f16 pairs
+  uint32_t qh2[NPAIR];
+  {
+    const float scale_log2 = 1.4426950408889634f * rsqrtf((float)D);
+    const uint16_t* qp = static_cast<const uint16_t*>(ly.q) + ((size_t)(b * dm.Hq + hk * G + g)) * D + (D / 4) * t;
+#pragma unroll
+    for (int i = 0; i < NPAIR; ++i) {
+      float a = 0.f, c = 0.f;
+      if (g < G) {
+        const uint32_t w2 = *reinterpret_cast<const uint32_t*>(qp + 2 * i);
+        a = bf16lo(w2) * scale_log2;
+        c = bf16hi(w2) * scale_log2;
+      }
+      qh2[i] = pack_half2(a, c);
+    }
+  }
+
+  // global sources of this (layer, batch, KV head)
+  const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * (n >> 5) * D * 16;
+  const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * (n >> 5) * D * 2;
+  const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * (n >> 5) * D * 2;
+  const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * (D / 2);
+  const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * (D / 16);
+  const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * (D / 16);
+
+  // stage one tile: 16-byte asynchronous copies, destinations swizzled for the transposing loads
+  auto issue_tile = [&](int tile, int stage) {
+    const uint32_t sb = wsm_u + stage * TL::BYTES;
+    const unsigned char* kc = gKc + (size_t)tile * D * 16;
+    const unsigned char* vc = gVc + (size_t)tile * 32 * (D / 2);
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) {
+      const int c = lane + 32 * i;                              // channel
+      const int slot = c ^ ((c / (D / 4)) << 1);
+      cp_async16(sb + TL::KC + slot * 16, kc + c * 16);
+    }
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) {
+      const int idx = lane + 32 * i;                            // 16-byte piece: token tau, value group v
+      const int tau = idx / NC, v = idx % NC;
+      const int sw = NC == 4 ? (tau >> 1) & 3 : (tau >> 2) & 1;
+      cp_async16(sb + TL::VC + tau * (D / 2) + ((v ^ sw) << 4), vc + idx * 16);
+    }
+    constexpr int MCH = D / 8;                                  // 16-byte pieces of each scale / zero array
+    if (lane < MCH) {
+      cp_async16(sb + TL::KS + lane * 16, gKs + (size_t)tile * D * 2 + lane * 16);
+      cp_async16(sb + TL::VS + lane * 16, gVs + (size_t)tile * 2 * D + lane * 16);
+    } else if (lane < 2 * MCH) {
+      const int j = lane - MCH;
+      cp_async16(sb + TL::KZ + j * 16, gKz + (size_t)tile * D * 2 + j * 16);
+      cp_async16(sb + TL::VZ + j * 16, gVz + (size_t)tile * 2 * D + j * 16);
+    }
+  };
+
+  // per-lane shared-memory offsets of the transposing loads
+  uint32_t k_off, v_off[NC];
+  {
+    const int m = lane >> 3, r = lane & 7, tq = r >> 1, p = r & 1;
+    const int ch = (D / 4) * tq + 2 * m + p;                    // + 8 per ldmatrix call
+    k_off = TL::KC + ((ch ^ (tq << 1)) << 4);
+    const int tau = 8 * m + r;                                  // matrix m = tokens 8m .. 8m+7
+    const int sw = NC == 4 ? (tau >> 1) & 3 : (tau >> 2) & 1;
+#pragma unroll
+    for (int v = 0; v < NC; ++v) v_off[v] = TL::VC + tau * (D / 2) + ((v ^ sw) << 4);
+  }
+
+  // running softmax state of columns 2t, 2t+1 and the accumulators
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  float accO[NC][2][4], accPZ[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int v = 0; v < NC; ++v)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) accO[v][mt][e] = 0.f;
+
+  const int n_my = warp < n_tiles ? (n_tiles - warp + DM_WARPS - 1) / DM_WARPS : 0;
+#pragma unroll
+  for (int s = 0; s < DM_STAGES - 1; ++s) {
+    if (s < n_my) issue_tile(tile_begin + warp + DM_WARPS * s, s);
+    cp_async_commit();
+  }
+
+  for (int it = 0; it < n_my; ++it) {
+    __syncwarp();                                               // everyone is done with the stage refilled below
+    if (it + DM_STAGES - 1 < n_my)
+      issue_tile(tile_begin + warp + DM_WARPS * (it + DM_STAGES - 1), (it + DM_STAGES - 1) % DM_STAGES);
+    cp_async_commit();
+    cp_async_wait<DM_STAGES - 1>();
+    __syncwarp();
+    const uint32_t sb = wsm_u + (it % DM_STAGES) * TL::BYTES;
+
+    // ---------------- keys: logits of 32 tokens x 8 columns
+    float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, accZ[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      const uint4 s4 = lds128(sb + TL::KS + (D / 4) * t * 2 + c * 16);
+      const uint4 z4 = lds128(sb + TL::KZ + (D / 4) * t * 2 + c * 16);
+      const uint32_t qs0 = hmul2_u32(qh2[4 * c + 0], s4.x), qs1 = hmul2_u32(qh2[4 * c + 1], s4.y);
+      const uint32_t qs2 = hmul2_u32(qh2[4 * c + 2], s4.z), qs3 = hmul2_u32(qh2[4 * c + 3], s4.w);
+      uint32_t R0, R1, R2, R3;
+      ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_off + c * 128);
+      mma_f16_m16n8k16(accK[0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, qs0, qs1);
+      const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
+      mma_f16_m16n8k16(accK[1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, qs0, qs1);
+      mma_f16_m16n8k16(accZ, z4.x, z4.x, z4.y, z4.y, qh2[4 * c + 0], qh2[4 * c + 1]);
+      mma_f16_m16n8k16(accK[0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, qs2, qs3);
+      const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
+      mma_f16_m16n8k16(accK[1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, qs2, qs3);
+      mma_f16_m16n8k16(accZ, z4.z, z4.z, z4.w, z4.w, qh2[4 * c + 2], qh2[4 * c + 3]);
+    }
+    // this lane: tokens 4g .. 4g+3 of the tile, columns 2t and 2t+1
+    //   lg[j][e]: token 4g + j, column 2t + e
+    float lg[4][2];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      lg[2 * mt][0] = fmaf(accK[mt][0], C24, accZ[0]);
+      lg[2 * mt][1] = fmaf(accK[mt][1], C24, accZ[1]);
+      lg[2 * mt + 1][0] = fmaf(accK[mt][2], C20, accZ[0]);
+      lg[2 * mt + 1][1] = fmaf(accK[mt][3], C20, accZ[1]);
+    }
+
+    // ---------------- running softmax (log2 domain)
+    float corr[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      float mx = fmaxf(fmaxf(lg[0][e], lg[1][e]), fmaxf(lg[2][e], lg[3][e]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+      const float mnew = fmaxf(m_run[e], mx);
+      corr[e] = exp2f(m_run[e] - mnew);
+      m_run[e] = mnew;
+      float sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        lg[j][e] = exp2f(lg[j][e] - mnew);
+        sum += lg[j][e];
+      }
+      l_run[e] = fmaf(l_run[e], corr[e], sum);                  // lane-local partial over its 4 tokens
+    }
+    if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+      for (int v = 0; v < NC; ++v)
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          accO[v][mt][0] *= corr[0]; accO[v][mt][1] *= corr[1];
+          accO[v][mt][2] *= corr[0]; accO[v][mt][3] *= corr[1];
+        }
+      accPZ[0] *= corr[0]; accPZ[1] *= corr[1];
+    }
+
+    // ---------------- P through shared memory: [column][token] f16, then token pairs of column g
+    sts64(sP + (2 * t) * SP_STRIDE + g * 8, pack_half2(lg[0][0], lg[1][0]), pack_half2(lg[2][0], lg[3][0]));
+    sts64(sP + (2 * t + 1) * SP_STRIDE + g * 8, pack_half2(lg[0][1], lg[1][1]), pack_half2(lg[2][1], lg[3][1]));
+    __syncwarp();
+    uint32_t p2[4];                                             // tokens (2t,2t+1) + {0, 8, 16, 24}
+#pragma unroll
+    for (int pr = 0; pr < 4; ++pr) p2[pr] = lds32(sP + g * SP_STRIDE + 4 * t + 16 * pr);
+
+    // ---------------- values: B = p * scale of the token's channel group, zero-point rows
+    uint32_t ps[4][NC], zp[4];
+#pragma unroll
+    for (int pr = 0; pr < 4; ++pr) {
+      const int a = 8 * pr + 2 * t;                             // first token of the pair
+      if constexpr (NC == 4) {
+        const uint4 x = lds128(sb + TL::VS + a * 8);
+        ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x5410));
+        ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x7632));
+        ps[pr][2] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x5410));
+        ps[pr][3] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x7632));
+        const uint4 y = lds128(sb + TL::VZ + a * 8);
+        const uint32_t lo = (g & 2) ? y.y : y.x, hi = (g & 2) ? y.w : y.z;
+        zp[pr] = g < NC ? __byte_perm(lo, hi, (g & 1) ? 0x7632 : 0x5410) : 0u;
+      } else {
+        const uint2 x = lds64(sb + TL::VS + a * 4);
+        ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x5410));
+        ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x7632));
+        const uint2 y = lds64(sb + TL::VZ + a * 4);
+        zp[pr] = g < NC ? __byte_perm(y.x, y.y, (g & 1) ? 0x7632 : 0x5410) : 0u;
+      }
+    }
+    mma_f16_m16n8k16(accPZ, zp[0], 0u, zp[1], 0u, p2[0], p2[1]);
+    mma_f16_m16n8k16(accPZ, zp[2], 0u, zp[3], 0u, p2[2], p2[3]);
+#pragma unroll
+    for (int v = 0; v < NC; ++v) {
+      uint32_t R0, R1, R2, R3;
+      ldmatrix_x4_trans(R0, R1, R2, R3, sb + v_off[v]);
+      mma_f16_m16n8k16(accO[v][0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, ps[0][v], ps[1][v]);
+      const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
+      mma_f16_m16n8k16(accO[v][1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, ps[0][v], ps[1][v]);
+      mma_f16_m16n8k16(accO[v][0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, ps[2][v], ps[3][v]);
+      const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
+      mma_f16_m16n8k16(accO[v][1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, ps[2][v], ps[3][v]);
+    }
+  }
+
+  // ---------------- per-warp result -> shared memory -> one partial per (block, query head)
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
+  }
+  cp_async_wait<0>();
+  __syncthreads();                                               // stage buffers are free: reuse them
+  float* s_acc = reinterpret_cast<float*>(smem);                 // [warp][8 columns][D]
+  float* s_m = s_acc + DM_WARPS * 8 * D;                         // [warp][8]
+  float* s_l = s_m + DM_WARPS * 8;
+#pragma unroll
+  for (int v = 0; v < NC; ++v) {
+    // zero-point term of channel group v for columns 2t, 2t+1 sits in lane (g = v, t)
+    const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * v + t);
+    const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * v + t);
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      const int ch = 32 * v + 4 * g + 2 * mt;
+      float* o0 = s_acc + ((warp * 8 + 2 * t) * D);
+      float* o1 = o0 + D;
+      o0[ch] = fmaf(accO[v][mt][0], C24, pz0);
+      o1[ch] = fmaf(accO[v][mt][1], C24, pz1);
+      o0[ch + 1] = fmaf(accO[v][mt][2], C20, pz0);
+      o1[ch + 1] = fmaf(accO[v][mt][3], C20, pz1);
+    }
+  }
+  if (g == 0) {
+    s_m[warp * 8 + 2 * t] = m_run[0]; s_m[warp * 8 + 2 * t + 1] = m_run[1];
+    s_l[warp * 8 + 2 * t] = l_run[0]; s_l[warp * 8 + 2 * t + 1] = l_run[1];
+  }
+  __syncthreads();
+  const size_t slot = (size_t)ly.part_base + (size_t)bh * n_splits + split;
+  for (int idx = tid; idx < G * D; idx += DM_THREADS) {
+    const int h = idx / D, d = idx % D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int wp = 0; wp < DM_WARPS; ++wp) M = fmaxf(M, s_m[wp * 8 + h]);
+    float Ls = 0.f, A = 0.f;
+#pragma unroll
+    for (int wp = 0; wp < DM_WARPS; ++wp) {
+      const float mw = s_m[wp * 8 + h];
+      if (mw != -INFINITY) {
+        const float f = exp2f(mw - M);
+        Ls = fmaf(s_l[wp * 8 + h], f, Ls);
+        A = fmaf(s_acc[(wp * 8 + h) * D + d], f, A);
+      }
+    }
+    float* o = partials + (slot * G + h) * (size_t)(D + 2);
+    if (d == 0) { o[0] = M; o[1] = Ls; }
+    o[2 + d] = A;
+  }
+}
+
+template <int D>
+constexpr size_t mma4_smem_bytes() {
+  return (size_t)DM_WARPS * (DM_STAGES * Tile4<D>::BYTES + SP_BYTES);
+}
+
+}  // namespace
+
+bool decode_mma_supported(const DecDims& d) {
+  return d.bits == 4 && d.group == 32 && (d.D == 128 || d.D == 64);
+}
+
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, int max_splits, float* partials,
+                              cudaStream_t st) {
+  const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
+  if (d.D == 128) {
+    constexpr size_t smem = mma4_smem_bytes<128>();
+    static_assert(smem >= (size_t)DM_WARPS * 8 * 128 * 4 + 2 * DM_WARPS * 8 * 4, "combine buffer must fit");
+    cudaError_t e = cudaFuncSetAttribute(decode_mma4_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    decode_mma4_kernel<128><<<grid, DM_THREADS, smem, st>>>(tab, d, partials);
+  } else {
+    constexpr size_t smem = mma4_smem_bytes<64>();
+    static_assert(smem >= (size_t)DM_WARPS * 8 * 64 * 4 + 2 * DM_WARPS * 8 * 4, "combine buffer must fit");
+    cudaError_t e = cudaFuncSetAttribute(decode_mma4_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    decode_mma4_kernel<64><<<grid, DM_THREADS, smem, st>>>(tab, d, partials);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace qp
