@@ -37,12 +37,6 @@ qp_status check_cache(const qp_cache* c, bool need_ptrs) {
   return QP_OK;
 }
 
-size_t decode_ws_bytes_for(const qp_cache& c, int chunk) {
-  const size_t splits = (size_t)(c.n_keep + chunk - 1) / chunk;
-  const size_t G = (size_t)(c.n_q_heads / c.n_kv_heads);
-  return (size_t)c.batch * c.n_kv_heads * splits * G * (size_t)(c.head_dim + 2) * sizeof(float);
-}
-
 }  // namespace
 
 extern "C" {
@@ -98,7 +92,8 @@ size_t qp_compress_workspace_bytes(int batch, int n_q_heads, int n_kv_heads, int
 
 size_t qp_decode_workspace_bytes(const qp_cache* cache) {
   if (check_cache(cache, false) != QP_OK) return 0;
-  return decode_ws_bytes_for(*cache, 128);   // 128 tokens is the smallest split any launch uses
+  const DecDims d{cache->batch, cache->n_q_heads, cache->n_kv_heads, cache->head_dim, cache->bits, cache->group};
+  return decode_workspace_bound(d, cache->n_keep);
 }
 
 static qp_status check_score_args(const void* Q_win, const void* K, int batch, int Hq, int Hkv, int D, int L, int w,
@@ -178,7 +173,8 @@ qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cac
   if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !q || !caches || !out || !workspace) return QP_ERR_INVALID_ARG;
   if (!aligned16(workspace)) return QP_ERR_ALIGNMENT;
   const qp_cache& c0 = caches[0];
-  long long total_tokens = 0;
+  DecTable tab;
+  tab.n_layers = n_layers;
   for (int l = 0; l < n_layers; ++l) {
     const qp_status s = check_cache(&caches[l], true);
     if (s != QP_OK) return s;
@@ -188,28 +184,15 @@ qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cac
       return QP_ERR_INVALID_ARG;
     if (!q[l] || !out[l]) return QP_ERR_INVALID_ARG;
     if (!aligned16(q[l]) || !aligned16(out[l])) return QP_ERR_ALIGNMENT;
-    total_tokens += (long long)c.batch * c.n_kv_heads * c.n_keep;
-  }
-  const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
-  DecTable tab;
-  tab.n_layers = n_layers;
-  tab.chunk = decode_chunk_tokens(d, total_tokens);
-  size_t need = 0;
-  int max_splits = 0, slot = 0;
-  for (int l = 0; l < n_layers; ++l) {
-    const qp_cache& c = caches[l];
-    const int splits = (c.n_keep + tab.chunk - 1) / tab.chunk;
     tab.l[l] = DecLayer{c.k_codes, c.v_codes,
                         static_cast<const __half*>(c.k_scale), static_cast<const __half*>(c.k_zero),
                         static_cast<const __half*>(c.v_scale), static_cast<const __half*>(c.v_zero),
-                        q[l], out[l], c.n_keep, slot};
-    slot += c.batch * c.n_kv_heads * splits;
-    need += decode_ws_bytes_for(c, tab.chunk);
-    if (splits > max_splits) max_splits = splits;
+                        q[l], out[l], c.n_keep, 0, 0, 0};
   }
-  if (workspace_bytes < need) return QP_ERR_WORKSPACE;
-  return launch_decode(tab, d, max_splits, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream)) ==
-                 cudaSuccess ? QP_OK : QP_ERR_CUDA;
+  const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
+  if (workspace_bytes < decode_plan(tab, d)) return QP_ERR_WORKSPACE;
+  return launch_decode(tab, d, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? QP_OK : QP_ERR_CUDA;
 }
 
 qp_status qp_decode_attn(const void* q, const qp_cache* cache, void* out, void* workspace, size_t workspace_bytes,

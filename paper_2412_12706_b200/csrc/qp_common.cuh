@@ -89,21 +89,30 @@ struct DecLayer {
   const void* q;
   void* out;
   int n;          // kept tokens of this layer
-  int part_base;  // first partial slot of this layer (in units of (bh, split) slots)
+  int part_base;  // chunked kernel: first partial slot of this layer (in units of (bh, split) slots)
+  int tile_base;  // flat-range kernel: index of this layer's first 32-token tile in the flat tile sequence
+  int reserved_;
 };
 struct DecTable {
   int n_layers;
-  int chunk;      // tokens per split
+  int chunk;        // chunked kernel: tokens per split
+  int total_tiles;  // flat-range kernel: tiles of all layers and heads
+  int n_workers;    // flat-range kernel: thread blocks, each owning total_tiles / n_workers consecutive tiles
   DecLayer l[QP_MAX_LAYERS];
 };
 struct DecDims {
   int Bt, Hq, Hkv, D, bits, group;
 };
-int decode_chunk_tokens(const DecDims& d, long long total_tokens_per_bh_sum);
-cudaError_t launch_decode(const DecTable& tab, const DecDims& d, int max_splits, float* partials, cudaStream_t st);
-// tensor-core split-K kernel (writes the same partial records as the generic one)
+constexpr int kMaxDecodeWorkers = 1024;
+// Chooses the decomposition for the layers in tab (n and pointers already set), fills chunk / part_base or
+// tile_base / total_tiles / n_workers and returns the bytes of partial records the launch needs.
+size_t decode_plan(DecTable& tab, const DecDims& d);
+// Upper bound of decode_plan's result for one layer of n_keep tokens, whatever else is in the launch.
+size_t decode_workspace_bound(const DecDims& d, int n_keep);
+cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+// tensor-core split-K kernel and its merge
 bool decode_mma_supported(const DecDims& d);
-cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, int max_splits, float* partials,
-                              cudaStream_t st);
+int decode_mma_blocks_per_sm();
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
 
 }  // namespace qp

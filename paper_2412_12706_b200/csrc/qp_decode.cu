@@ -192,24 +192,77 @@ decode_merge_kernel(const __grid_constant__ DecTable tab, const DecDims dm, cons
 
 }  // namespace
 
-int decode_chunk_tokens(const DecDims& d, long long total_tokens) {
-  // aim at about eight blocks per SM, in whole 128-token units
+namespace {
+
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+size_t record_bytes(const DecDims& d) { return (size_t)(d.Hq / d.Hkv) * (size_t)(d.D + 2) * sizeof(float); }
+
+// chunked kernel: about eight blocks per SM, in whole 128-token units
+int chunk_tokens(long long total_tokens) {
   long long c = (total_tokens + 148 * 8 - 1) / (148 * 8);
   c = (c + 127) / 128 * 128;
   if (c < 128) c = 128;
   if (c > 4096) c = 4096;
-  (void)d;
   return (int)c;
 }
 
-cudaError_t launch_decode(const DecTable& tab, const DecDims& d, int max_splits, float* partials, cudaStream_t st) {
-  const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
+}  // namespace
+
+size_t decode_plan(DecTable& tab, const DecDims& d) {
+  const int BH = d.Bt * d.Hkv;
   if (decode_mma_supported(d)) {
-    const cudaError_t e = launch_decode_mma(tab, d, max_splits, partials, st);
-    if (e != cudaSuccess) return e;
-    decode_merge_kernel<<<dim3(d.Bt * d.Hq, tab.n_layers), 128, 0, st>>>(tab, d, partials);
-    return cudaGetLastError();
+    long long T = 0;
+    for (int l = 0; l < tab.n_layers; ++l) {
+      tab.l[l].tile_base = (int)T;
+      tab.l[l].part_base = 0;
+      T += (long long)BH * (tab.l[l].n / 32);
+    }
+    long long W = (long long)sm_count() * decode_mma_blocks_per_sm();
+    if (W > kMaxDecodeWorkers) W = kMaxDecodeWorkers;
+    if (W > (T + 3) / 4) W = (T + 3) / 4;                       // at least one tile per warp
+    if (W < 1) W = 1;
+    while (W > 1 && T * W >= (1ll << 31)) W /= 2;               // the merge kernel's range arithmetic is 32-bit
+    tab.total_tiles = (int)T;
+    tab.n_workers = (int)W;
+    tab.chunk = 0;
+    return ((size_t)tab.n_layers * BH + (size_t)W) * record_bytes(d);
   }
+  long long total_tokens = 0;
+  for (int l = 0; l < tab.n_layers; ++l) total_tokens += (long long)BH * tab.l[l].n;
+  tab.chunk = chunk_tokens(total_tokens);
+  tab.total_tiles = tab.n_workers = 0;
+  size_t slots = 0;
+  for (int l = 0; l < tab.n_layers; ++l) {
+    tab.l[l].part_base = (int)slots;
+    tab.l[l].tile_base = 0;
+    slots += (size_t)BH * ((tab.l[l].n + tab.chunk - 1) / tab.chunk);
+  }
+  return slots * record_bytes(d);
+}
+
+size_t decode_workspace_bound(const DecDims& d, int n_keep) {
+  const size_t BH = (size_t)d.Bt * d.Hkv;
+  const size_t chunked = BH * (size_t)((n_keep + 127) / 128) * record_bytes(d);   // 128 tokens = smallest split
+  const size_t flat = (BH + kMaxDecodeWorkers) * record_bytes(d);
+  return chunked > flat ? chunked : flat;
+}
+
+cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+  if (decode_mma_supported(d)) return launch_decode_mma(tab, d, partials, st);
+  int max_splits = 1;
+  for (int l = 0; l < tab.n_layers; ++l) max_splits = max(max_splits, (tab.l[l].n + tab.chunk - 1) / tab.chunk);
+  const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
   switch (d.bits) {
     case 2: decode_generic_kernel<2><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
     case 4: decode_generic_kernel<4><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;

@@ -33,7 +33,13 @@ namespace {
 
 constexpr int DM_WARPS = 4;
 constexpr int DM_THREADS = DM_WARPS * 32;
-constexpr int DM_STAGES = 3;
+#ifndef QP_DM_STAGES
+#define QP_DM_STAGES 3
+#endif
+#ifndef QP_DM_MINB
+#define QP_DM_MINB 3
+#endif
+constexpr int DM_STAGES = QP_DM_STAGES;
 constexpr int SP_STRIDE = 80;            // bytes per column of the per-warp P buffer (8 columns)
 constexpr int SP_BYTES = 8 * SP_STRIDE;
 
@@ -41,13 +47,16 @@ constexpr int SP_BYTES = 8 * SP_STRIDE;
 template <int D>
 struct Tile4 {
   static constexpr int KC = 0;                    // D rows of 16 B: one channel, 32 tokens
-  static constexpr int KS = KC + D * 16;          // D halves
-  static constexpr int KZ = KS + D * 2;
-  static constexpr int VC = KZ + D * 2;           // 32 token rows of D/2 bytes
+  static constexpr int KS = KC + D * 16;          // D halves; channels >= 64 shifted by 16 B (bank spread)
+  static constexpr int KZ = KS + D * 2 + 16;
+  static constexpr int VC = KZ + D * 2 + 16;      // 32 token rows of D/2 bytes
   static constexpr int VS = VC + 16 * D;          // 32 x (D/32) halves
   static constexpr int VZ = VS + 2 * D;
   static constexpr int BYTES = VZ + 2 * D;
 };
+// key scale/zero of channel ch: the four lanes t read 16 B at channel (D/4)*t + 8c; the extra 16 B
+// after channel 63 keeps lanes t and t+2 out of each other's banks
+__host__ __device__ constexpr int ksz_off(int ch) { return ch * 2 + (ch / 64) * 16; }
 
 __device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
   uint32_t d;
@@ -77,89 +86,64 @@ __device__ __forceinline__ void sts64(uint32_t a, uint32_t x, uint32_t y) {
   asm volatile("st.shared.v2.u32 [%0], {%1,%2};\n" ::"r"(a), "r"(x), "r"(y));
 }
 
+// 2^x for x <= 0 (softmax weights): the hardware approximation, about 2 ulp, flushes tiny results to 0
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+
 constexpr uint32_t M0 = 0x000f000fu;   // code in bits 0..3 of each half: value c * 2^-24
 constexpr uint32_t M1 = 0x00f000f0u;   // code in bits 4..7 of each half: value c * 2^-20
 constexpr float C24 = 16777216.0f, C20 = 1048576.0f;
 
+// Work decomposition ("stream-K" over tokens): the 32-token tiles of all (layer, batch, KV head)
+// triples form one flat sequence of T tiles; block w of W owns the contiguous range
+// [w*T/W, (w+1)*T/W), so every block streams the same number of bytes (+-1 tile), the grid is one
+// wave of resident blocks and a block pays its pipeline ramp once.  A range that crosses a head
+// boundary is processed head by head ("segments"); each (head, block) pair that meets leaves one
+// partial record at slot head + block (heads and blocks both advance monotonically along the flat
+// sequence, so head + block is unique), which the merge kernel finds again by the same arithmetic.
+struct SkOwner {
+  long long T, W;
+  __host__ __device__ long long start(long long w) const { return w * T / W; }
+  // the block whose range holds flat tile f is ((f + 1) * W - 1) / T
+};
+
 template <int D>
-__global__ void __launch_bounds__(DM_THREADS, 3)
+__global__ void __launch_bounds__(DM_THREADS, QP_DM_MINB)
 decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials) {
   using TL = Tile4<D>;
   constexpr int NC = D / 32;       // ldmatrix.x4 calls over the channels of a key tile = value groups per token
   constexpr int NPAIR = D / 8;     // channel pairs owned by one lane on the key side (D/4 channels)
   extern __shared__ __align__(128) unsigned char smem[];
 
-  const int layer = blockIdx.z, bh = blockIdx.y, split = blockIdx.x;
-  const DecLayer& ly = tab.l[layer];
-  const int n = ly.n, t_begin = split * tab.chunk;
-  if (t_begin >= n) return;
-  const int t_end = min(n, t_begin + tab.chunk);
-  const int tile_begin = t_begin >> 5, n_tiles = (t_end - t_begin) >> 5;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  const int G = dm.Hq / dm.Hkv, b = bh / dm.Hkv, hk = bh % dm.Hkv;
-  const int n_splits = (n + tab.chunk - 1) / tab.chunk;
+  const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
+  const SkOwner sk{tab.total_tiles, tab.n_workers};
+  const int cta = blockIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;\n" ::);     // the merge grid may start to become resident
+  long long cur = sk.start(cta);
+  const long long f_end = sk.start(cta + 1);
 
   unsigned char* wsm = smem + warp * (DM_STAGES * TL::BYTES + SP_BYTES);
   const uint32_t wsm_u = smem_u32(wsm);
   const uint32_t sP = wsm_u + DM_STAGES * TL::BYTES;
+  // combine buffer of a finished segment; it overlays the (then idle) stage buffers
+  float* s_acc = reinterpret_cast<float*>(smem);                // [warp][8][D]
+  float* s_m = s_acc + DM_WARPS * 8 * D;                        // [warp][8]
+  float* s_l = s_m + DM_WARPS * 8;
 
-  // B-side query fragments: column g of the MMAs is query head g of this KV head (columns >= G are 0);
-  // this lane holds the D/4 channels [t*D/4, (t+1)*D/4) as f16 pairs
-  uint32_t qh2[NPAIR];
-  {
-    const float scale_log2 = 1.4426950408889634f * rsqrtf((float)D);
-    const uint16_t* qp = static_cast<const uint16_t*>(ly.q) + ((size_t)(b * dm.Hq + hk * G + g)) * D + (D / 4) * t;
+  // per-lane shared-memory offsets: destinations of the asynchronous copies, sources of the transposing loads
+  uint32_t kdst[D / 32], vdst[D / 32], k_off, v_off[NC];
 #pragma unroll
-    for (int i = 0; i < NPAIR; ++i) {
-      float a = 0.f, c = 0.f;
-      if (g < G) {
-        const uint32_t w2 = *reinterpret_cast<const uint32_t*>(qp + 2 * i);
-        a = bf16lo(w2) * scale_log2;
-        c = bf16hi(w2) * scale_log2;
-      }
-      qh2[i] = pack_half2(a, c);
-    }
+  for (int i = 0; i < D / 32; ++i) {
+    const int c = lane + 32 * i;                                // key channel
+    kdst[i] = TL::KC + ((c ^ ((c / (D / 4)) << 1)) << 4);
+    const int tau = c / NC, v = c % NC;                         // 16-byte piece of the value codes
+    const int sw = NC == 4 ? (tau >> 1) & 3 : (tau >> 2) & 1;
+    vdst[i] = TL::VC + tau * (D / 2) + ((v ^ sw) << 4);
   }
-
-  // global sources of this (layer, batch, KV head)
-  const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * (n >> 5) * D * 16;
-  const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * (n >> 5) * D * 2;
-  const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * (n >> 5) * D * 2;
-  const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * (D / 2);
-  const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * (D / 16);
-  const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * (D / 16);
-
-  // stage one tile: 16-byte asynchronous copies, destinations swizzled for the transposing loads
-  auto issue_tile = [&](int tile, int stage) {
-    const uint32_t sb = wsm_u + stage * TL::BYTES;
-    const unsigned char* kc = gKc + (size_t)tile * D * 16;
-    const unsigned char* vc = gVc + (size_t)tile * 32 * (D / 2);
-#pragma unroll
-    for (int i = 0; i < D / 32; ++i) {
-      const int c = lane + 32 * i;                              // channel
-      const int slot = c ^ ((c / (D / 4)) << 1);
-      cp_async16(sb + TL::KC + slot * 16, kc + c * 16);
-    }
-#pragma unroll
-    for (int i = 0; i < D / 32; ++i) {
-      const int idx = lane + 32 * i;                            // 16-byte piece: token tau, value group v
-      const int tau = idx / NC, v = idx % NC;
-      const int sw = NC == 4 ? (tau >> 1) & 3 : (tau >> 2) & 1;
-      cp_async16(sb + TL::VC + tau * (D / 2) + ((v ^ sw) << 4), vc + idx * 16);
-    }
-    constexpr int MCH = D / 8;                                  // 16-byte pieces of each scale / zero array
-    if (lane < MCH) {
-      cp_async16(sb + TL::KS + lane * 16, gKs + (size_t)tile * D * 2 + lane * 16);
-      cp_async16(sb + TL::VS + lane * 16, gVs + (size_t)tile * 2 * D + lane * 16);
-    } else if (lane < 2 * MCH) {
-      const int j = lane - MCH;
-      cp_async16(sb + TL::KZ + j * 16, gKz + (size_t)tile * D * 2 + j * 16);
-      cp_async16(sb + TL::VZ + j * 16, gVz + (size_t)tile * 2 * D + j * 16);
-    }
-  };
-
-  // per-lane shared-memory offsets of the transposing loads
-  uint32_t k_off, v_off[NC];
   {
     const int m = lane >> 3, r = lane & 7, tq = r >> 1, p = r & 1;
     const int ch = (D / 4) * tq + 2 * m + p;                    // + 8 per ldmatrix call
@@ -169,196 +153,303 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 #pragma unroll
     for (int v = 0; v < NC; ++v) v_off[v] = TL::VC + tau * (D / 2) + ((v ^ sw) << 4);
   }
+  constexpr int MCH = D / 8;                                    // 16-byte pieces of each scale / zero array
+  const int mj = lane < MCH ? lane : lane - MCH;                // piece handled by this lane
+  const uint32_t ksz_dst = (lane < MCH ? TL::KS : TL::KZ) + mj * 16 + (mj / 8) * 16;
+  const uint32_t vsz_dst = (lane < MCH ? TL::VS : TL::VZ) + mj * 16;
 
-  // running softmax state of columns 2t, 2t+1 and the accumulators
-  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-  float accO[NC][2][4], accPZ[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-  for (int v = 0; v < NC; ++v)
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) accO[v][mt][e] = 0.f;
+  int li = 0;
+  while (li + 1 < tab.n_layers && tab.l[li + 1].tile_base <= cur) ++li;
 
-  const int n_my = warp < n_tiles ? (n_tiles - warp + DM_WARPS - 1) / DM_WARPS : 0;
-#pragma unroll
-  for (int s = 0; s < DM_STAGES - 1; ++s) {
-    if (s < n_my) issue_tile(tile_begin + warp + DM_WARPS * s, s);
-    cp_async_commit();
-  }
+  while (cur < f_end) {
+    const DecLayer& ly = tab.l[li];
+    const int n = ly.n, tph = n >> 5;                           // tiles per head in this layer
+    const int rel = (int)(cur - ly.tile_base), bh = rel / tph, tile_begin = rel % tph;
+    const int n_tiles = (int)min((long long)(tph - tile_begin), f_end - cur);
+    const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
 
-  for (int it = 0; it < n_my; ++it) {
-    __syncwarp();                                               // everyone is done with the stage refilled below
-    if (it + DM_STAGES - 1 < n_my)
-      issue_tile(tile_begin + warp + DM_WARPS * (it + DM_STAGES - 1), (it + DM_STAGES - 1) % DM_STAGES);
-    cp_async_commit();
-    cp_async_wait<DM_STAGES - 1>();
-    __syncwarp();
-    const uint32_t sb = wsm_u + (it % DM_STAGES) * TL::BYTES;
+    // global sources of this (layer, batch, KV head)
+    const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * tph * D * 16;
+    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * tph * D * 2;
+    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * tph * D * 2;
+    const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * (D / 2);
+    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * (D / 16);
+    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * (D / 16);
+    const unsigned char* gKm = lane < MCH ? gKs : gKz;
+    const unsigned char* gVm = lane < MCH ? gVs : gVz;
 
-    // ---------------- keys: logits of 32 tokens x 8 columns
-    float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, accZ[4] = {0.f, 0.f, 0.f, 0.f};
+    // stage one tile: 16-byte asynchronous copies, destinations swizzled for the transposing loads
+    auto issue_tile = [&](int tile, int stage) {
+      const uint32_t sb = wsm_u + stage * TL::BYTES;
+      const unsigned char* kc = gKc + (size_t)tile * D * 16 + lane * 16;
+      const unsigned char* vc = gVc + (size_t)tile * 16 * D + lane * 16;
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const uint4 s4 = lds128(sb + TL::KS + (D / 4) * t * 2 + c * 16);
-      const uint4 z4 = lds128(sb + TL::KZ + (D / 4) * t * 2 + c * 16);
-      const uint32_t qs0 = hmul2_u32(qh2[4 * c + 0], s4.x), qs1 = hmul2_u32(qh2[4 * c + 1], s4.y);
-      const uint32_t qs2 = hmul2_u32(qh2[4 * c + 2], s4.z), qs3 = hmul2_u32(qh2[4 * c + 3], s4.w);
-      uint32_t R0, R1, R2, R3;
-      ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_off + c * 128);
-      mma_f16_m16n8k16(accK[0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, qs0, qs1);
-      const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
-      mma_f16_m16n8k16(accK[1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, qs0, qs1);
-      mma_f16_m16n8k16(accZ, z4.x, z4.x, z4.y, z4.y, qh2[4 * c + 0], qh2[4 * c + 1]);
-      mma_f16_m16n8k16(accK[0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, qs2, qs3);
-      const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
-      mma_f16_m16n8k16(accK[1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, qs2, qs3);
-      mma_f16_m16n8k16(accZ, z4.z, z4.z, z4.w, z4.w, qh2[4 * c + 2], qh2[4 * c + 3]);
-    }
-    // this lane: tokens 4g .. 4g+3 of the tile, columns 2t and 2t+1
-    //   lg[j][e]: token 4g + j, column 2t + e
-    float lg[4][2];
+      for (int i = 0; i < D / 32; ++i) {
+        cp_async16(sb + kdst[i], kc + i * 512);
+        cp_async16(sb + vdst[i], vc + i * 512);
+      }
+      if (lane < 2 * MCH) {
+        cp_async16(sb + ksz_dst, gKm + (size_t)tile * D * 2 + mj * 16);
+        cp_async16(sb + vsz_dst, gVm + (size_t)tile * D * 2 + mj * 16);
+      }
+    };
+
+    // tiles of this segment go round-robin to the warps; start the copies before anything else
+    const int n_my = warp < n_tiles ? (n_tiles - warp + DM_WARPS - 1) / DM_WARPS : 0;
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
-      lg[2 * mt][0] = fmaf(accK[mt][0], C24, accZ[0]);
-      lg[2 * mt][1] = fmaf(accK[mt][1], C24, accZ[1]);
-      lg[2 * mt + 1][0] = fmaf(accK[mt][2], C20, accZ[0]);
-      lg[2 * mt + 1][1] = fmaf(accK[mt][3], C20, accZ[1]);
+    for (int s = 0; s < DM_STAGES - 1; ++s) {
+      if (s < n_my) issue_tile(tile_begin + warp + DM_WARPS * s, s);
+      cp_async_commit();
     }
 
-    // ---------------- running softmax (log2 domain)
-    float corr[2];
+    // B-side query fragments: column g of the MMAs is query head g of this KV head (columns >= G are 0);
+    // this lane holds the D/4 channels [t*D/4, (t+1)*D/4) as f16 pairs
+    uint32_t qh2[NPAIR];
+    {
+      const float scale_log2 = 1.4426950408889634f * rsqrtf((float)D);
+      const uint16_t* qp = static_cast<const uint16_t*>(ly.q) + ((size_t)(b * dm.Hq + hk * G + g)) * D + (D / 4) * t;
+#pragma unroll
+      for (int i = 0; i < NPAIR; i += 4) {
+        uint4 w4 = make_uint4(0u, 0u, 0u, 0u);
+        if (g < G) w4 = *reinterpret_cast<const uint4*>(qp + 2 * i);
+        qh2[i + 0] = pack_half2(bf16lo(w4.x) * scale_log2, bf16hi(w4.x) * scale_log2);
+        qh2[i + 1] = pack_half2(bf16lo(w4.y) * scale_log2, bf16hi(w4.y) * scale_log2);
+        qh2[i + 2] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);
+        qh2[i + 3] = pack_half2(bf16lo(w4.w) * scale_log2, bf16hi(w4.w) * scale_log2);
+      }
+    }
+
+    // running softmax state of columns 2t, 2t+1 and the accumulators
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float accO[NC][2][4], accPZ[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int v = 0; v < NC; ++v)
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) accO[v][mt][e] = 0.f;
+
+    for (int it = 0; it < n_my; ++it) {
+      __syncwarp();                                             // everyone is done with the stage refilled below
+      if (it + DM_STAGES - 1 < n_my)
+        issue_tile(tile_begin + warp + DM_WARPS * (it + DM_STAGES - 1), (it + DM_STAGES - 1) % DM_STAGES);
+      cp_async_commit();
+      cp_async_wait<DM_STAGES - 1>();
+      __syncwarp();
+      const uint32_t sb = wsm_u + (it % DM_STAGES) * TL::BYTES;
+
+      // ---------------- keys: logits of 32 tokens x 8 columns
+      float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, accZ[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const uint4 s4 = lds128(sb + TL::KS + ksz_off((D / 4) * t + 8 * c));
+        const uint4 z4 = lds128(sb + TL::KZ + ksz_off((D / 4) * t + 8 * c));
+        const uint32_t qs0 = hmul2_u32(qh2[4 * c + 0], s4.x), qs1 = hmul2_u32(qh2[4 * c + 1], s4.y);
+        const uint32_t qs2 = hmul2_u32(qh2[4 * c + 2], s4.z), qs3 = hmul2_u32(qh2[4 * c + 3], s4.w);
+        uint32_t R0, R1, R2, R3;
+        ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_off + c * 128);
+        mma_f16_m16n8k16(accK[0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, qs0, qs1);
+        const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
+        mma_f16_m16n8k16(accK[1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, qs0, qs1);
+        mma_f16_m16n8k16(accZ, z4.x, z4.x, z4.y, z4.y, qh2[4 * c + 0], qh2[4 * c + 1]);
+        mma_f16_m16n8k16(accK[0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, qs2, qs3);
+        const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
+        mma_f16_m16n8k16(accK[1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, qs2, qs3);
+        mma_f16_m16n8k16(accZ, z4.z, z4.z, z4.w, z4.w, qh2[4 * c + 2], qh2[4 * c + 3]);
+      }
+      // this lane: tokens 4g .. 4g+3 of the tile, columns 2t and 2t+1
+      //   lg[j][e]: token 4g + j, column 2t + e
+      float lg[4][2];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        lg[2 * mt][0] = fmaf(accK[mt][0], C24, accZ[0]);
+        lg[2 * mt][1] = fmaf(accK[mt][1], C24, accZ[1]);
+        lg[2 * mt + 1][0] = fmaf(accK[mt][2], C20, accZ[0]);
+        lg[2 * mt + 1][1] = fmaf(accK[mt][3], C20, accZ[1]);
+      }
+
+      // ---------------- running softmax (log2 domain)
+      float corr[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float mx = fmaxf(fmaxf(lg[0][e], lg[1][e]), fmaxf(lg[2][e], lg[3][e]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+        const float mnew = fmaxf(m_run[e], mx);
+        corr[e] = ex2(m_run[e] - mnew);
+        m_run[e] = mnew;
+        float sum = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          lg[j][e] = ex2(lg[j][e] - mnew);
+          sum += lg[j][e];
+        }
+        l_run[e] = fmaf(l_run[e], corr[e], sum);                // lane-local partial over its 4 tokens
+      }
+      if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+        for (int v = 0; v < NC; ++v)
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            accO[v][mt][0] *= corr[0]; accO[v][mt][1] *= corr[1];
+            accO[v][mt][2] *= corr[0]; accO[v][mt][3] *= corr[1];
+          }
+        accPZ[0] *= corr[0]; accPZ[1] *= corr[1];
+      }
+
+      // ---------------- P through shared memory: [column][token] f16, then token pairs of column g
+      sts64(sP + (2 * t) * SP_STRIDE + g * 8, pack_half2(lg[0][0], lg[1][0]), pack_half2(lg[2][0], lg[3][0]));
+      sts64(sP + (2 * t + 1) * SP_STRIDE + g * 8, pack_half2(lg[0][1], lg[1][1]), pack_half2(lg[2][1], lg[3][1]));
+      __syncwarp();
+      uint32_t p2[4];                                           // tokens (2t,2t+1) + {0, 8, 16, 24}
+#pragma unroll
+      for (int pr = 0; pr < 4; ++pr) p2[pr] = lds32(sP + g * SP_STRIDE + 4 * t + 16 * pr);
+
+      // ---------------- values: B = p * scale of the token's channel group, zero-point rows
+      uint32_t ps[4][NC], zp[4];
+#pragma unroll
+      for (int pr = 0; pr < 4; ++pr) {
+        const int a = 8 * pr + 2 * t;                           // first token of the pair
+        zp[pr] = 0u;
+        if constexpr (NC == 4) {
+          const uint4 x = lds128(sb + TL::VS + a * 8);
+          ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x5410));
+          ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x7632));
+          ps[pr][2] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x5410));
+          ps[pr][3] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x7632));
+          if (g < NC) {                                         // rows of the zero-point MMA: value group v = g
+            const uint32_t ya = lds32(sb + TL::VZ + a * 8 + (g & 2) * 2);       // z[a][v & ~1], z[a][v | 1]
+            const uint32_t yb = lds32(sb + TL::VZ + a * 8 + 8 + (g & 2) * 2);   // same of token a + 1
+            zp[pr] = __byte_perm(ya, yb, (g & 1) ? 0x7632 : 0x5410);
+          }
+        } else {
+          const uint2 x = lds64(sb + TL::VS + a * 4);
+          ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x5410));
+          ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x7632));
+          if (g < NC) {
+            const uint2 y = lds64(sb + TL::VZ + a * 4);
+            zp[pr] = __byte_perm(y.x, y.y, (g & 1) ? 0x7632 : 0x5410);
+          }
+        }
+      }
+      mma_f16_m16n8k16(accPZ, zp[0], 0u, zp[1], 0u, p2[0], p2[1]);
+      mma_f16_m16n8k16(accPZ, zp[2], 0u, zp[3], 0u, p2[2], p2[3]);
+#pragma unroll
+      for (int v = 0; v < NC; ++v) {
+        uint32_t R0, R1, R2, R3;
+        ldmatrix_x4_trans(R0, R1, R2, R3, sb + v_off[v]);
+        mma_f16_m16n8k16(accO[v][0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, ps[0][v], ps[1][v]);
+        const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
+        mma_f16_m16n8k16(accO[v][1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, ps[0][v], ps[1][v]);
+        mma_f16_m16n8k16(accO[v][0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, ps[2][v], ps[3][v]);
+        const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
+        mma_f16_m16n8k16(accO[v][1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, ps[2][v], ps[3][v]);
+      }
+    }
+
+    // ---------------- per-warp result -> shared memory -> one partial per (head, block) and query head
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      float mx = fmaxf(fmaxf(lg[0][e], lg[1][e]), fmaxf(lg[2][e], lg[3][e]));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-      const float mnew = fmaxf(m_run[e], mx);
-      corr[e] = exp2f(m_run[e] - mnew);
-      m_run[e] = mnew;
-      float sum = 0.f;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        lg[j][e] = exp2f(lg[j][e] - mnew);
-        sum += lg[j][e];
-      }
-      l_run[e] = fmaf(l_run[e], corr[e], sum);                  // lane-local partial over its 4 tokens
+      l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+      l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+      l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
     }
-    if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
-#pragma unroll
-      for (int v = 0; v < NC; ++v)
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          accO[v][mt][0] *= corr[0]; accO[v][mt][1] *= corr[1];
-          accO[v][mt][2] *= corr[0]; accO[v][mt][3] *= corr[1];
-        }
-      accPZ[0] *= corr[0]; accPZ[1] *= corr[1];
-    }
-
-    // ---------------- P through shared memory: [column][token] f16, then token pairs of column g
-    sts64(sP + (2 * t) * SP_STRIDE + g * 8, pack_half2(lg[0][0], lg[1][0]), pack_half2(lg[2][0], lg[3][0]));
-    sts64(sP + (2 * t + 1) * SP_STRIDE + g * 8, pack_half2(lg[0][1], lg[1][1]), pack_half2(lg[2][1], lg[3][1]));
-    __syncwarp();
-    uint32_t p2[4];                                             // tokens (2t,2t+1) + {0, 8, 16, 24}
-#pragma unroll
-    for (int pr = 0; pr < 4; ++pr) p2[pr] = lds32(sP + g * SP_STRIDE + 4 * t + 16 * pr);
-
-    // ---------------- values: B = p * scale of the token's channel group, zero-point rows
-    uint32_t ps[4][NC], zp[4];
-#pragma unroll
-    for (int pr = 0; pr < 4; ++pr) {
-      const int a = 8 * pr + 2 * t;                             // first token of the pair
-      if constexpr (NC == 4) {
-        const uint4 x = lds128(sb + TL::VS + a * 8);
-        ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x5410));
-        ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x7632));
-        ps[pr][2] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x5410));
-        ps[pr][3] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x7632));
-        const uint4 y = lds128(sb + TL::VZ + a * 8);
-        const uint32_t lo = (g & 2) ? y.y : y.x, hi = (g & 2) ? y.w : y.z;
-        zp[pr] = g < NC ? __byte_perm(lo, hi, (g & 1) ? 0x7632 : 0x5410) : 0u;
-      } else {
-        const uint2 x = lds64(sb + TL::VS + a * 4);
-        ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x5410));
-        ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x7632));
-        const uint2 y = lds64(sb + TL::VZ + a * 4);
-        zp[pr] = g < NC ? __byte_perm(y.x, y.y, (g & 1) ? 0x7632 : 0x5410) : 0u;
-      }
-    }
-    mma_f16_m16n8k16(accPZ, zp[0], 0u, zp[1], 0u, p2[0], p2[1]);
-    mma_f16_m16n8k16(accPZ, zp[2], 0u, zp[3], 0u, p2[2], p2[3]);
+    __syncthreads();                                            // every warp has consumed its last stage
 #pragma unroll
     for (int v = 0; v < NC; ++v) {
-      uint32_t R0, R1, R2, R3;
-      ldmatrix_x4_trans(R0, R1, R2, R3, sb + v_off[v]);
-      mma_f16_m16n8k16(accO[v][0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, ps[0][v], ps[1][v]);
-      const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
-      mma_f16_m16n8k16(accO[v][1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, ps[0][v], ps[1][v]);
-      mma_f16_m16n8k16(accO[v][0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, ps[2][v], ps[3][v]);
-      const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
-      mma_f16_m16n8k16(accO[v][1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, ps[2][v], ps[3][v]);
-    }
-  }
-
-  // ---------------- per-warp result -> shared memory -> one partial per (block, query head)
+      // zero-point term of channel group v for columns 2t, 2t+1 sits in lane (g = v, t)
+      const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * v + t);
+      const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * v + t);
 #pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
-    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
-    l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
-  }
-  cp_async_wait<0>();
-  __syncthreads();                                               // stage buffers are free: reuse them
-  float* s_acc = reinterpret_cast<float*>(smem);                 // [warp][8 columns][D]
-  float* s_m = s_acc + DM_WARPS * 8 * D;                         // [warp][8]
-  float* s_l = s_m + DM_WARPS * 8;
-#pragma unroll
-  for (int v = 0; v < NC; ++v) {
-    // zero-point term of channel group v for columns 2t, 2t+1 sits in lane (g = v, t)
-    const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * v + t);
-    const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * v + t);
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
-      const int ch = 32 * v + 4 * g + 2 * mt;
-      float* o0 = s_acc + ((warp * 8 + 2 * t) * D);
-      float* o1 = o0 + D;
-      o0[ch] = fmaf(accO[v][mt][0], C24, pz0);
-      o1[ch] = fmaf(accO[v][mt][1], C24, pz1);
-      o0[ch + 1] = fmaf(accO[v][mt][2], C20, pz0);
-      o1[ch + 1] = fmaf(accO[v][mt][3], C20, pz1);
-    }
-  }
-  if (g == 0) {
-    s_m[warp * 8 + 2 * t] = m_run[0]; s_m[warp * 8 + 2 * t + 1] = m_run[1];
-    s_l[warp * 8 + 2 * t] = l_run[0]; s_l[warp * 8 + 2 * t + 1] = l_run[1];
-  }
-  __syncthreads();
-  const size_t slot = (size_t)ly.part_base + (size_t)bh * n_splits + split;
-  for (int idx = tid; idx < G * D; idx += DM_THREADS) {
-    const int h = idx / D, d = idx % D;
-    float M = -INFINITY;
-#pragma unroll
-    for (int wp = 0; wp < DM_WARPS; ++wp) M = fmaxf(M, s_m[wp * 8 + h]);
-    float Ls = 0.f, A = 0.f;
-#pragma unroll
-    for (int wp = 0; wp < DM_WARPS; ++wp) {
-      const float mw = s_m[wp * 8 + h];
-      if (mw != -INFINITY) {
-        const float f = exp2f(mw - M);
-        Ls = fmaf(s_l[wp * 8 + h], f, Ls);
-        A = fmaf(s_acc[(wp * 8 + h) * D + d], f, A);
+      for (int mt = 0; mt < 2; ++mt) {
+        const int ch = 32 * v + 4 * g + 2 * mt;
+        float* o0 = s_acc + ((warp * 8 + 2 * t) * D);
+        float* o1 = o0 + D;
+        *reinterpret_cast<float2*>(o0 + ch) = make_float2(fmaf(accO[v][mt][0], C24, pz0), fmaf(accO[v][mt][2], C20, pz0));
+        *reinterpret_cast<float2*>(o1 + ch) = make_float2(fmaf(accO[v][mt][1], C24, pz1), fmaf(accO[v][mt][3], C20, pz1));
       }
     }
-    float* o = partials + (slot * G + h) * (size_t)(D + 2);
-    if (d == 0) { o[0] = M; o[1] = Ls; }
-    o[2 + d] = A;
+    if (g == 0) {
+      s_m[warp * 8 + 2 * t] = m_run[0]; s_m[warp * 8 + 2 * t + 1] = m_run[1];
+      s_l[warp * 8 + 2 * t] = l_run[0]; s_l[warp * 8 + 2 * t + 1] = l_run[1];
+    }
+    __syncthreads();
+    const size_t slot = (size_t)li * BH + bh + cta;
+    for (int idx = tid; idx < G * D; idx += DM_THREADS) {
+      const int h = idx / D, d = idx % D;
+      float M = -INFINITY;
+#pragma unroll
+      for (int wp = 0; wp < DM_WARPS; ++wp) M = fmaxf(M, s_m[wp * 8 + h]);
+      float Ls = 0.f, A = 0.f;
+#pragma unroll
+      for (int wp = 0; wp < DM_WARPS; ++wp) {
+        const float mw = s_m[wp * 8 + h];
+        if (mw != -INFINITY) {
+          const float f = ex2(mw - M);
+          Ls = fmaf(s_l[wp * 8 + h], f, Ls);
+          A = fmaf(s_acc[(wp * 8 + h) * D + d], f, A);
+        }
+      }
+      float* o = partials + (slot * G + h) * (size_t)(D + 2);
+      if (d == 0) { o[0] = M; o[1] = Ls; }
+      o[2 + d] = A;
+    }
+    __syncthreads();                                            // the combine buffer is reused by the next segment
+
+    cur += n_tiles;
+    if (bh == BH - 1 && tile_begin + n_tiles == tph) ++li;
   }
+}
+
+// S5 for the decomposition above: head (layer, batch, KV head) was touched by the blocks
+// owner(first tile) .. owner(last tile); their records sit at slots head + block.
+// One warp per (layer, batch, query head), a lane per four channels.  The kernel is launched as a
+// programmatic dependent of the attention kernel: its blocks may become resident while that kernel
+// drains and wait at griddepcontrol.wait until its records are complete and visible.
+constexpr int MG_WARPS = 4;
+__global__ void __launch_bounds__(MG_WARPS * 32)
+decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, const float* __restrict__ partials) {
+  const int D = dm.D, G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv, n_bq = dm.Bt * dm.Hq;
+  const int item = blockIdx.x * MG_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  const bool active = item < n_bq * tab.n_layers;
+  const int layer = active ? item / n_bq : 0, bq = active ? item % n_bq : 0;
+  const DecLayer& ly = tab.l[layer];
+  const int b = bq / dm.Hq, h = bq % dm.Hq, bh = b * dm.Hkv + h / G, hl = h % G;
+  const unsigned T = (unsigned)tab.total_tiles, W = (unsigned)tab.n_workers;   // T * W < 2^31 (host-checked)
+  const int tph = ly.n >> 5;
+  const unsigned first = (unsigned)ly.tile_base + (unsigned)bh * tph;
+  const int w_lo = (int)(((first + 1u) * W - 1u) / T), w_hi = (int)(((first + tph) * W - 1u) / T);
+  const size_t head = (size_t)layer * BH + bh;
+  const size_t stride = (size_t)G * (D + 2);
+  const float* base = partials + (head * G + hl) * (size_t)(D + 2);
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  if (!active || 4 * lane >= D) return;
+  float M = -INFINITY;
+  for (int w = w_lo; w <= w_hi; ++w) M = fmaxf(M, base[w * stride]);
+  float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
+  for (int w = w_lo; w <= w_hi; ++w) {
+    const float* r = base + w * stride;
+    const float f = ex2(r[0] - M);
+    const float2 a01 = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
+    const float2 a23 = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
+    Ls = fmaf(r[1], f, Ls);
+    A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
+    A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
+  }
+  const float inv = __fdiv_rn(1.0f, Ls);
+  __nv_bfloat162 o01 = __floats2bfloat162_rn(A0 * inv, A1 * inv), o23 = __floats2bfloat162_rn(A2 * inv, A3 * inv);
+  uint2 packed;
+  packed.x = *reinterpret_cast<uint32_t*>(&o01);
+  packed.y = *reinterpret_cast<uint32_t*>(&o23);
+  *reinterpret_cast<uint2*>(static_cast<bf16*>(ly.out) + (size_t)bq * D + 4 * lane) = packed;
 }
 
 template <int D>
 constexpr size_t mma4_smem_bytes() {
-  return (size_t)DM_WARPS * (DM_STAGES * Tile4<D>::BYTES + SP_BYTES);
+  constexpr size_t stages = (size_t)DM_WARPS * (DM_STAGES * Tile4<D>::BYTES + SP_BYTES);
+  constexpr size_t combine = (size_t)DM_WARPS * 8 * D * 4 + 2 * DM_WARPS * 8 * 4;
+  return stages > combine ? stages : combine;
 }
 
 }  // namespace
@@ -367,23 +458,49 @@ bool decode_mma_supported(const DecDims& d) {
   return d.bits == 4 && d.group == 32 && (d.D == 128 || d.D == 64);
 }
 
-cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, int max_splits, float* partials,
-                              cudaStream_t st) {
-  const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
+int decode_mma_blocks_per_sm() { return QP_DM_MINB; }
+
+// opt in to more than 48 KB of dynamic shared memory, once per device and kernel
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes, unsigned char (&done)[64]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (done[dev]) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) done[dev] = 1;
+  return e;
+}
+
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+  const dim3 grid(tab.n_workers);
+  cudaError_t e;
   if (d.D == 128) {
     constexpr size_t smem = mma4_smem_bytes<128>();
-    static_assert(smem >= (size_t)DM_WARPS * 8 * 128 * 4 + 2 * DM_WARPS * 8 * 4, "combine buffer must fit");
-    cudaError_t e = cudaFuncSetAttribute(decode_mma4_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static unsigned char done[64] = {};
+    e = allow_smem(decode_mma4_kernel<128>, smem, done);
     if (e != cudaSuccess) return e;
     decode_mma4_kernel<128><<<grid, DM_THREADS, smem, st>>>(tab, d, partials);
   } else {
     constexpr size_t smem = mma4_smem_bytes<64>();
-    static_assert(smem >= (size_t)DM_WARPS * 8 * 64 * 4 + 2 * DM_WARPS * 8 * 4, "combine buffer must fit");
-    cudaError_t e = cudaFuncSetAttribute(decode_mma4_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static unsigned char done[64] = {};
+    e = allow_smem(decode_mma4_kernel<64>, smem, done);
     if (e != cudaSuccess) return e;
     decode_mma4_kernel<64><<<grid, DM_THREADS, smem, st>>>(tab, d, partials);
   }
-  return cudaGetLastError();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int items = d.Bt * d.Hq * tab.n_layers;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((items + MG_WARPS - 1) / MG_WARPS);
+  cfg.blockDim = dim3(MG_WARPS * 32);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_merge_sk_kernel, tab, d, (const float*)partials);
 }
 
 }  // namespace qp

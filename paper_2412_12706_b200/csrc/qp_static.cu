@@ -32,16 +32,15 @@ qp_status static_scratch(void** out) {
 
 extern "C" qp_status qp_decode_attn_static(const void* q, const qp_cache* cache, void* out, void* stream) {
   if (!cache) return QP_ERR_INVALID_ARG;
-  // Scratch this cache needs: one (max, sum, acc[D]) record per (batch, KV head, split, query head
-  // of the group), with the split size the decode launch will choose for this much work.
+  // Scratch this cache needs: (max, sum, acc[D]) records, one per query head of the group for every
+  // (batch, KV head, token split) the decode launch will use for this much work.
   const size_t coarse = qp_decode_workspace_bytes(cache);
   if (coarse == 0) return QP_ERR_INVALID_ARG;   // invalid descriptor
   const qp::DecDims d{cache->batch, cache->n_q_heads, cache->n_kv_heads, cache->head_dim, cache->bits, cache->group};
-  const long long tokens = (long long)cache->batch * cache->n_kv_heads * cache->n_keep;
-  const int chunk = qp::decode_chunk_tokens(d, tokens);
-  const size_t splits = (size_t)(cache->n_keep + chunk - 1) / chunk;
-  const size_t need = (size_t)cache->batch * cache->n_kv_heads * splits * (size_t)(cache->n_q_heads / cache->n_kv_heads) *
-                      (size_t)(cache->head_dim + 2) * sizeof(float);
+  qp::DecTable plan;
+  plan.n_layers = 1;
+  plan.l[0].n = cache->n_keep;
+  const size_t need = qp::decode_plan(plan, d);   // the same plan qp_decode_attn makes for this cache
   if (need > (size_t)QP_STATIC_SCRATCH_BYTES) return QP_ERR_WORKSPACE;
   void* scratch = nullptr;
   const qp_status s = static_scratch(&scratch);
