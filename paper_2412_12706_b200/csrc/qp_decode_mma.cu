@@ -25,7 +25,7 @@
 // channels for values) while an MMA register pairs two elements along the contraction; the
 // transposing ldmatrix fetches 16-bit units of two different rows into one register, which is
 // exactly that pairing.  Shared-memory rows are XOR-swizzled so these loads are conflict-free.
-#include "qp_common.cuh"
+#include "qp_mma.cuh"
 
 namespace qp {
 
@@ -58,57 +58,9 @@ struct Tile4 {
 // after channel 63 keeps lanes t and t+2 out of each other's banks
 __host__ __device__ constexpr int ksz_off(int ch) { return ch * 2 + (ch / 64) * 16; }
 
-__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("mul.rn.f16x2 %0, %1, %2;\n" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
-  const __half2 h = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&h);
-}
-__device__ __forceinline__ uint4 lds128(uint32_t a) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-  return v;
-}
-__device__ __forceinline__ uint2 lds64(uint32_t a) {
-  uint2 v;
-  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
-  return v;
-}
-__device__ __forceinline__ uint32_t lds32(uint32_t a) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];\n" : "=r"(v) : "r"(a));
-  return v;
-}
-__device__ __forceinline__ void sts64(uint32_t a, uint32_t x, uint32_t y) {
-  asm volatile("st.shared.v2.u32 [%0], {%1,%2};\n" ::"r"(a), "r"(x), "r"(y));
-}
-
-// 2^x for x <= 0 (softmax weights): the hardware approximation, about 2 ulp, flushes tiny results to 0
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
-  return y;
-}
-
 constexpr uint32_t M0 = 0x000f000fu;   // code in bits 0..3 of each half: value c * 2^-24
 constexpr uint32_t M1 = 0x00f000f0u;   // code in bits 4..7 of each half: value c * 2^-20
 constexpr float C24 = 16777216.0f, C20 = 1048576.0f;
-
-// Work decomposition ("stream-K" over tokens): the 32-token tiles of all (layer, batch, KV head)
-// triples form one flat sequence of T tiles; block w of W owns the contiguous range
-// [w*T/W, (w+1)*T/W), so every block streams the same number of bytes (+-1 tile), the grid is one
-// wave of resident blocks and a block pays its pipeline ramp once.  A range that crosses a head
-// boundary is processed head by head ("segments"); each (head, block) pair that meets leaves one
-// partial record at slot head + block (heads and blocks both advance monotonically along the flat
-// sequence, so head + block is unique), which the merge kernel finds again by the same arithmetic.
-struct SkOwner {
-  long long T, W;
-  __host__ __device__ long long start(long long w) const { return w * T / W; }
-  // the block whose range holds flat tile f is ((f + 1) * W - 1) / T
-};
 
 template <int D>
 __global__ void __launch_bounds__(DM_THREADS, QP_DM_MINB)
@@ -455,23 +407,13 @@ constexpr size_t mma4_smem_bytes() {
 }  // namespace
 
 bool decode_mma_supported(const DecDims& d) {
-  return d.bits == 4 && d.group == 32 && (d.D == 128 || d.D == 64);
+  if (d.group != 32 || (d.D != 128 && d.D != 64)) return false;
+  return d.bits == 4 || decode_mma2_supported(d);
 }
 
 int decode_mma_blocks_per_sm() { return QP_DM_MINB; }
 
-// opt in to more than 48 KB of dynamic shared memory, once per device and kernel
-template <typename K>
-cudaError_t allow_smem(K kernel, size_t bytes, unsigned char (&done)[64]) {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (done[dev]) return cudaSuccess;
-  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) done[dev] = 1;
-  return e;
-}
-
-cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
   const dim3 grid(tab.n_workers);
   cudaError_t e;
   if (d.D == 128) {
@@ -487,7 +429,11 @@ cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* part
     if (e != cudaSuccess) return e;
     decode_mma4_kernel<64><<<grid, DM_THREADS, smem, st>>>(tab, d, partials);
   }
-  e = cudaGetLastError();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+  cudaError_t e = d.bits == 4 ? launch_decode_mma4(tab, d, partials, st) : launch_decode_mma2(tab, d, partials, st);
   if (e != cudaSuccess) return e;
   const int items = d.Bt * d.Hq * tab.n_layers;
   cudaLaunchConfig_t cfg = {};

@@ -116,8 +116,9 @@ def test_decode_matches_oracle(bits, Hq, Hkv, D, group, n):
         out = qp.decode_attn(q.to(DEV), cache).float().cpu().numpy().astype(np.float64)
         err = np.abs(out - ref).max()
         assert err <= decode_tolerance(ref), (err, decode_tolerance(ref))
-        # the kernel itself is far tighter than the stated tolerance: bf16 output rounding dominates
-        assert err <= 2e-3 + 2.0 ** -8 * np.abs(ref).max(), err
+        # the kernel's own budget is tighter than the stated tolerance: MMA operands (q * scale, p * scale)
+        # are rounded to f16 (2^-11 relative) and the output to bf16 (2^-9 relative)
+        assert err <= 3e-3 + 2.0 ** -7 * np.abs(ref).max(), err
 
 
 def test_decode_16bit_ragged_length_and_zero_query_mean():
