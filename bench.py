@@ -40,12 +40,13 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of the dominant (decode) kernel from an ncu capture, valid only for the exact
-# kernel source it was taken on: {"sha256": <hash of csrc/qp_decode.cu>, "workload": name,
+# kernel sources it was taken on: {"sha256": <hash of DECODE_KERNEL_SOURCES>, "workload": name,
 # "bytes_per_launch": dram__bytes_read.sum + dram__bytes_write.sum}
 NCU_TRAFFIC: dict = {}
 
 KERNELS_PER_COMPRESS = 6      # sweep 1, row-stat merge, sweep 2, pool, top-k, gather+quantize
 KERNELS_PER_DECODE_CALL = 2   # split-K attention, merge
+DECODE_KERNEL_SOURCES = ("qp_decode.cu", "qp_decode_mma.cu", "qp_decode_mma2.cu", "qp_mma.cuh")
 
 
 def packed_bytes(wl: synth.Workload, layer: int) -> int:
@@ -261,7 +262,10 @@ def run_gpu(args, wl):
     call_ms = statistics.mean(e0.elapsed_time(e1) for e0, e1 in call_events)
 
     # ---- end to end: host buffers in, host buffers out, through the same calls
-    e2e = run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step) if not args.no_e2e else None
+    input_bytes = 2 * n_seq * n_layers * Bt * Hkv * L * D * 2
+    # the host-buffer leg pins a copy of every input; keep it to workloads whose inputs are a few GB
+    e2e = run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step) \
+        if not args.no_e2e and input_bytes <= 8e9 else None
 
     def allmax(x: float) -> float:
         return shard.max_over_ranks(x, dist, dev)
@@ -277,7 +281,8 @@ def run_gpu(args, wl):
     value = shard.whole_job_throughput(dec_bytes_step * steps, world, dec_ms * 1e-3) / 1e9
     peak, peak_kind = hbm_peak()
     achieved = dec_bytes_call / (call_ms * 1e-3) / 1e9
-    sha = hashlib.sha256(open(os.path.join(ROOT, "paper_2412_12706_b200", "csrc", "qp_decode.cu"), "rb").read()).hexdigest()
+    sha = hashlib.sha256(b"".join(open(os.path.join(ROOT, "paper_2412_12706_b200", "csrc", f), "rb").read()
+                                  for f in DECODE_KERNEL_SOURCES)).hexdigest()
     traffic = NCU_TRAFFIC.get("bytes_per_launch") if NCU_TRAFFIC.get("sha256") == sha and \
         NCU_TRAFFIC.get("workload") == wl.name else None
     cpu = oracle_sample(wl, 1, 0) if world == 1 and not args.no_cpu_baseline else None
@@ -298,7 +303,8 @@ def run_gpu(args, wl):
         "decode_us_per_call": call_ms * 1e3,
         "decode_phase_ms_per_step": dec_ms / steps,
         "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
-        "roofline": {"bound": "hbm", "kernel": "decode attention (split-K + merge)", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": "decode attention (split-K attention kernel + merge kernel, per call)",
+                     "achieved": achieved,
                      "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic},
         "e2e": None if e2e is None else {

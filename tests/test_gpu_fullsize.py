@@ -1,0 +1,118 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration the
+benchmark times (qp_compress_layer per layer, qp_decode_attn_layers over the layers).
+
+The oracle cannot redo a whole 32k x 8-batch layer in seconds, so the GPU runs the full problem
+and the oracle recomputes SAMPLED (batch, KV head) pairs from the same inputs: indices with the
+near-tie rule, packed bytes bit for bit on the GPU's indices, decode outputs within tolerance.
+Everything not sampled is covered by structural properties that hold at any size."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import qp_oracle as orc
+from paper_2412_12706_b200 import qp, synth
+from tests.util import assert_packed_equal, bits_u16, check_kept_against_oracle, decode_tolerance
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _slice_packed(cache, b, hk):
+    """Packed arrays of one (batch, KV head) pair as an oracle Packed with Bt = Hkv = 1."""
+    d = cache.desc
+    sl = lambda t: t[b:b + 1, hk:hk + 1].contiguous()
+    if d.bits == 16:
+        return orc.Packed(16, d.group, d.n_keep, bits_u16(sl(cache.k_codes)), bits_u16(sl(cache.v_codes)),
+                          None, None, None, None)
+    u32 = lambda t: sl(t).cpu().numpy().view(np.uint32)
+    return orc.Packed(d.bits, d.group, d.n_keep, u32(cache.k_codes), u32(cache.v_codes),
+                      bits_u16(sl(cache.k_scale)), bits_u16(sl(cache.k_zero)),
+                      bits_u16(sl(cache.v_scale)), bits_u16(sl(cache.v_zero)))
+
+
+def _check_structure(kept: torch.Tensor, L: int, w: int):
+    """Holds for every head at any size: ascending, unique, in range, window last."""
+    k = kept.long()
+    assert bool((k[..., 1:] > k[..., :-1]).all())
+    assert int(k.min()) >= 0 and int(k.max()) == L - 1
+    assert bool((k[..., -w:] == torch.arange(L - w, L, device=k.device)).all())
+
+
+def run_fullsize(wl: synth.Workload, layers, samples, variants=None, decode_steps=2):
+    """variants: list of (bits, tokens16) sharing the same K, V, Q_win (the constant-memory sweep)."""
+    variants = variants or [(wl.bits, wl.tokens16)]
+    G = wl.n_q_heads // wl.n_kv_heads
+    per_variant = {v: {"caches": [], "kept": []} for v in variants}
+    host = {}                                                   # sampled inputs per layer
+    pooled_ref = {}
+    for layer in layers:
+        k, v = synth.make_kv(wl, layer, device=DEV)
+        qw = synth.make_q_win(wl, layer, device=DEV)
+        ws = torch.empty(qp.compress_workspace_bytes(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.L, wl.w),
+                         dtype=torch.uint8, device=DEV)
+        for bits, tokens16 in variants:
+            wv = dataclasses.replace(wl, bits=bits, tokens16=tokens16)
+            cache, kept = qp.compress_layer(k, v, qw, wv.layer_budget_bits(layer), bits, wl.group, wl.pool, workspace=ws)
+            _check_structure(kept, wl.L, wl.w)
+            assert kept.shape[-1] * bits <= wv.layer_budget_bits(layer)
+            per_variant[(bits, tokens16)]["caches"].append(cache)
+            per_variant[(bits, tokens16)]["kept"].append(kept)
+        # pull the sampled pairs to the host as a pseudo batch [S,1,L,D] (the oracle threads over it)
+        ks = torch.stack([k[b, hk] for b, hk in samples])[:, None].contiguous()
+        vs = torch.stack([v[b, hk] for b, hk in samples])[:, None].contiguous()
+        qs = torch.stack([qw[b, hk * G:(hk + 1) * G] for b, hk in samples]).contiguous()
+        host[layer] = (bits_u16(ks), bits_u16(vs), bits_u16(qs))
+        pooled_ref[layer] = orc.scores(host[layer][2], host[layer][0], wl.pool)
+        del k, v, qw, ks, vs, qs
+    torch.cuda.synchronize()
+
+    swaps = 0
+    for (bits, tokens16), pv in per_variant.items():
+        # decode all layers in one launch pair, as the benchmark does
+        qd = [[synth.make_q_dec(wl, layer, s, device=DEV) for layer in layers] for s in range(decode_steps)]
+        outs = [[torch.empty_like(q) for q in row] for row in qd]
+        for s in range(decode_steps):
+            qp.decode_attn_layers(qp.LayerBatch(qd[s], pv["caches"], outs[s]))
+        torch.cuda.synchronize()
+        for li, layer in enumerate(layers):
+            cache, kept = pv["caches"][li], pv["kept"][li]
+            n = kept.shape[-1]
+            kb, vb, qb = host[layer]
+            kept_s = np.stack([kept[b, hk].cpu().numpy() for b, hk in samples])[:, None]
+            swaps += check_kept_against_oracle(kept_s, pooled_ref[layer], wl.L, wl.w, n)
+            ref = orc.quantize(kb, vb, kept_s, bits, wl.group)
+            for si, (b, hk) in enumerate(samples):
+                got = _slice_packed(cache, b, hk)
+                one = orc.Packed(ref.bits, ref.group, ref.n, ref.k_codes[si:si + 1], ref.v_codes[si:si + 1],
+                                 *(None if a is None else a[si:si + 1] for a in (ref.k_scale, ref.k_zero,
+                                                                                 ref.v_scale, ref.v_zero)))
+                assert_packed_equal(got, one)
+            kd, vd = orc.dequantize(ref, wl.head_dim)
+            for s in range(decode_steps):
+                qh = torch.stack([qd[s][li][b, hk * G:(hk + 1) * G] for b, hk in samples])    # [S,G,D]
+                ref_out = orc.decode(bits_u16(qh), kd, vd)
+                got_out = torch.stack([outs[s][li][b, hk * G:(hk + 1) * G] for b, hk in samples]).float().cpu().numpy()
+                assert np.abs(got_out - ref_out).max() <= decode_tolerance(ref_out)
+                assert bool(torch.isfinite(outs[s][li].float()).all())
+    return swaps
+
+
+def test_llama8b_32k_batch8_2bit_rotary_full_layer():
+    swaps = run_fullsize(synth.LLAMA8B_32K_B8, layers=[0, 31], samples=[(0, 0), (3, 5), (7, 7)])
+    assert swaps <= 6
+
+
+def test_llama8b_128k_constant_memory_sweep_full_layer():
+    wl = synth.sweep_128k(4)
+    variants = [(16, 1024), (8, 1024), (4, 1024), (2, 1024)]      # (B,16) (2B,8) (4B,4) (8B,2) with B = 1024
+    swaps = run_fullsize(wl, layers=[5], samples=[(0, 2)], variants=variants)
+    assert swaps <= 8
+
+
+def test_llama70b_pyramid_first_and_last_layer():
+    wl = synth.LLAMA70B_32K_B4
+    assert wl.n_keep(0) == 8192 and wl.n_keep(79) == 2048          # 2x .. 0.5x of the 4096-token mean
+    swaps = run_fullsize(wl, layers=[0, 79], samples=[(0, 0), (3, 6)])
+    assert swaps <= 4
