@@ -112,7 +112,7 @@ size_t decode_workspace_bound(const DecDims& d, int n_keep);
 cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
 // tensor-core split-K kernel and its merge
 bool decode_mma_supported(const DecDims& d);
-int decode_mma_blocks_per_sm();
+int decode_mma_blocks_per_sm(const DecDims& d);
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
 
 }  // namespace qp

@@ -228,7 +228,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
       tab.l[l].part_base = 0;
       T += (long long)BH * (tab.l[l].n / 32);
     }
-    long long W = (long long)sm_count() * decode_mma_blocks_per_sm();
+    long long W = (long long)sm_count() * decode_mma_blocks_per_sm(d);
     if (W > kMaxDecodeWorkers) W = kMaxDecodeWorkers;
     if (W > (T + 3) / 4) W = (T + 3) / 4;                       // at least one tile per warp
     if (W < 1) W = 1;

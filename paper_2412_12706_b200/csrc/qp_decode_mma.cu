@@ -408,10 +408,10 @@ constexpr size_t mma4_smem_bytes() {
 
 bool decode_mma_supported(const DecDims& d) {
   if (d.group != 32 || (d.D != 128 && d.D != 64)) return false;
-  return d.bits == 4 || decode_mma2_supported(d);
+  return d.bits == 4 || d.bits == 8 || decode_mma2_supported(d);
 }
 
-int decode_mma_blocks_per_sm() { return QP_DM_MINB; }
+int decode_mma_blocks_per_sm(const DecDims& d) { return d.bits == 8 ? decode_mma8_blocks_per_sm() : QP_DM_MINB; }
 
 cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
   const dim3 grid(tab.n_workers);
@@ -433,7 +433,9 @@ cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* par
 }
 
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
-  cudaError_t e = d.bits == 4 ? launch_decode_mma4(tab, d, partials, st) : launch_decode_mma2(tab, d, partials, st);
+  cudaError_t e = d.bits == 4   ? launch_decode_mma4(tab, d, partials, st)
+                  : d.bits == 8 ? launch_decode_mma8(tab, d, partials, st)
+                                : launch_decode_mma2(tab, d, partials, st);
   if (e != cudaSuccess) return e;
   const int items = d.Bt * d.Hq * tab.n_layers;
   cudaLaunchConfig_t cfg = {};
