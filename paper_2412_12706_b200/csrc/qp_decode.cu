@@ -226,7 +226,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
     for (int l = 0; l < tab.n_layers; ++l) {
       tab.l[l].tile_base = (int)T;
       tab.l[l].part_base = 0;
-      T += (long long)BH * (tab.l[l].n / 32);
+      T += (long long)BH * ((tab.l[l].n + 31) / 32);
     }
     long long W = (long long)sm_count() * decode_mma_blocks_per_sm(d);
     if (W > kMaxDecodeWorkers) W = kMaxDecodeWorkers;

@@ -369,7 +369,7 @@ decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, c
   const DecLayer& ly = tab.l[layer];
   const int b = bq / dm.Hq, h = bq % dm.Hq, bh = b * dm.Hkv + h / G, hl = h % G;
   const unsigned T = (unsigned)tab.total_tiles, W = (unsigned)tab.n_workers;   // T * W < 2^31 (host-checked)
-  const int tph = ly.n >> 5;
+  const int tph = (ly.n + 31) >> 5;
   const unsigned first = (unsigned)ly.tile_base + (unsigned)bh * tph;
   const int w_lo = (int)(((first + 1u) * W - 1u) / T), w_hi = (int)(((first + tph) * W - 1u) / T);
   const size_t head = (size_t)layer * BH + bh;
@@ -407,11 +407,15 @@ constexpr size_t mma4_smem_bytes() {
 }  // namespace
 
 bool decode_mma_supported(const DecDims& d) {
-  if (d.group != 32 || (d.D != 128 && d.D != 64)) return false;
+  if (d.D != 128 && d.D != 64) return false;
+  if (d.bits == 16) return true;
+  if (d.group != 32) return false;
   return d.bits == 4 || d.bits == 8 || decode_mma2_supported(d);
 }
 
-int decode_mma_blocks_per_sm(const DecDims& d) { return d.bits == 8 ? decode_mma8_blocks_per_sm() : QP_DM_MINB; }
+int decode_mma_blocks_per_sm(const DecDims& d) {
+  return d.bits == 8 ? decode_mma8_blocks_per_sm() : d.bits == 16 ? decode_mma16_blocks_per_sm() : QP_DM_MINB;
+}
 
 cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
   const dim3 grid(tab.n_workers);
@@ -435,6 +439,7 @@ cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* par
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
   cudaError_t e = d.bits == 4   ? launch_decode_mma4(tab, d, partials, st)
                   : d.bits == 8 ? launch_decode_mma8(tab, d, partials, st)
+                  : d.bits == 16 ? launch_decode_mma16(tab, d, partials, st)
                                 : launch_decode_mma2(tab, d, partials, st);
   if (e != cudaSuccess) return e;
   const int items = d.Bt * d.Hq * tab.n_layers;

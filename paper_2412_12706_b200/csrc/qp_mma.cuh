@@ -60,6 +60,8 @@ cudaError_t launch_decode_mma2(const DecTable& tab, const DecDims& d, float* par
 bool decode_mma2_supported(const DecDims& d);
 cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
 int decode_mma8_blocks_per_sm();
+cudaError_t launch_decode_mma16(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+int decode_mma16_blocks_per_sm();
 
 // opt in to more than 48 KB of dynamic shared memory, once per device and kernel
 template <typename K>
