@@ -189,6 +189,10 @@ def run_gpu(args, wl):
     qp.lib()
 
     n_seq, n_layers, n_dec = args.sequences, wl.n_layers, wl.decode_steps
+    # sequences whose layers share one qp_decode_attn_layers call (independent problems, as in continuous batching)
+    per_call = max(1, min(args.seqs_per_call, n_seq, qp.QP_MAX_LAYERS // n_layers))
+    while n_seq % per_call:
+        per_call -= 1
     Bt, Hq, Hkv, D, L, w = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.L, wl.w
     stream = torch.cuda.current_stream()
 
@@ -211,10 +215,18 @@ def run_gpu(args, wl):
         ws_d = torch.empty(sum(qp.decode_workspace_bytes(c) for c in sq["cache"]), dtype=torch.uint8, device=dev)
         sq["ws_d"] = ws_d
         sq["batches"] = [qp.LayerBatch([sq["qdec"][t, l] for l in range(n_layers)], sq["cache"],
-                                       [sq["out"][l] for l in range(n_layers)], ws_d) for t in range(n_dec)]
+                                       [sq["out"][l] for l in range(n_layers)], ws_d) for t in range(min(n_dec, 8))]
+    groups = []
+    for g0 in range(0, n_seq, per_call):
+        members = seqs[g0:g0 + per_call]
+        ws_g = torch.empty(sum(m["ws_d"].numel() for m in members), dtype=torch.uint8, device=dev)
+        groups.append([qp.LayerBatch([m["qdec"][t, l] for m in members for l in range(n_layers)],
+                                     [c for m in members for c in m["cache"]],
+                                     [m["out"][l] for m in members for l in range(n_layers)], ws_g)
+                       for t in range(n_dec)])
 
     dec_bytes_step = n_seq * n_dec * sum(packed_bytes(wl, l) for l in range(n_layers))
-    dec_bytes_call = sum(packed_bytes(wl, l) for l in range(n_layers))
+    dec_bytes_call = per_call * sum(packed_bytes(wl, l) for l in range(n_layers))
     ctx_tokens_step = n_seq * Bt * L
 
     def compress_all():
@@ -225,10 +237,10 @@ def run_gpu(args, wl):
 
     def decode_all(call_events=None):
         for t in range(n_dec):
-            for sq in seqs:          # consecutive launches touch different sequences' caches
+            for grp in groups:       # consecutive launches touch different sequences' caches
                 if call_events is not None:
                     e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
-                qp.decode_attn_layers(sq["batches"][t])
+                qp.decode_attn_layers(grp[t])
                 if call_events is not None:
                     e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
                     call_events.append((e0, e1))
@@ -261,11 +273,25 @@ def run_gpu(args, wl):
     dec_ms = sum(b.elapsed_time(c) for a, b, c in marks)
     call_ms = statistics.mean(e0.elapsed_time(e1) for e0, e1 in call_events)
 
+    # ---- the same decode attention with one sequence per call (context for the batched figure)
+    single_ms = None
+    if per_call > 1:
+        reps = 64
+        for r in range(8):
+            qp.decode_attn_layers(seqs[r % n_seq]["batches"][r % 8])
+        s0, s1 = ev(), ev()
+        s0.record(stream)
+        for r in range(reps):
+            qp.decode_attn_layers(seqs[r % n_seq]["batches"][r % 8])
+        s1.record(stream)
+        torch.cuda.synchronize()
+        single_ms = s0.elapsed_time(s1) / reps
+
     # ---- end to end: host buffers in, host buffers out, through the same calls
     input_bytes = 2 * n_seq * n_layers * Bt * Hkv * L * D * 2
     # the host-buffer leg pins a copy of every input; keep it to workloads whose inputs are a few GB
-    e2e = run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step) \
-        if not args.no_e2e and input_bytes <= 8e9 else None
+    e2e = run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step, per_call) \
+        if not args.no_e2e and input_bytes <= 10e9 else None
 
     def allmax(x: float) -> float:
         return shard.max_over_ranks(x, dist, dev)
@@ -294,13 +320,17 @@ def run_gpu(args, wl):
                    "head_dim": D, "context": L, "window": w, "bits": wl.bits, "group": wl.group,
                    "n_keep": [wl.n_keep(0), wl.n_keep(n_layers - 1)], "decode_steps": n_dec,
                    "sequences_per_gpu": n_seq, "parallelism": f"replicas x{world}, no collective",
-                   "decode_api": "qp_decode_attn_layers (one launch pair per decode step over all layers)",
-                   "l2": f"decode rotates over {n_seq} independent sequences "
-                         f"({n_seq * dec_bytes_call / 1e6:.0f} MB of packed cache) so consecutive launches "
-                         f"read different data; compress inputs {2 * n_seq * n_layers * Bt * Hkv * L * D * 2 / 1e9:.2f} GB"},
+                   "decode_api": f"qp_decode_attn_layers: one launch pair per decode step over all layers of "
+                                 f"{per_call} independent sequence(s) ({dec_bytes_call / 1e6:.0f} MB per call)",
+                   "sequences_per_call": per_call,
+                   "l2": f"decode rotates over {n_seq // per_call} group(s) of sequences "
+                         f"({n_seq * dec_bytes_call / per_call / 1e6:.0f} MB of packed cache in all) so consecutive "
+                         f"launches read different data; compress inputs {input_bytes / 1e9:.2f} GB"},
         "compress_tokens_per_s": world * ctx_tokens_step * steps / (comp_ms * 1e-3),
         "compress_ms_per_layer": comp_ms / (steps * n_seq * n_layers),
         "decode_us_per_call": call_ms * 1e3,
+        "decode_single_sequence_call": None if single_ms is None else {
+            "us_per_call": single_ms * 1e3, "GB/s": dec_bytes_call / per_call / (single_ms * 1e-3) / 1e9},
         "decode_phase_ms_per_step": dec_ms / steps,
         "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "decode attention (split-K attention kernel + merge kernel, per call)",
@@ -312,7 +342,8 @@ def run_gpu(args, wl):
             "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
             "ms_per_step": e2e["total_ms"] / e2e["steps"],
             "compress_tokens_per_s": world * ctx_tokens_step * e2e["steps"] / (e2e["comp_ms"] * 1e-3)},
-        "gpu_launches": steps * n_seq * (n_layers * KERNELS_PER_COMPRESS + n_dec * KERNELS_PER_DECODE_CALL),
+        "gpu_launches": steps * (n_seq * n_layers * KERNELS_PER_COMPRESS
+                                 + (n_seq // per_call) * n_dec * KERNELS_PER_DECODE_CALL),
         "clocks": clocks,
     }
     if cpu is not None:
@@ -323,7 +354,7 @@ def run_gpu(args, wl):
         dist.destroy_process_group()
 
 
-def run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step):
+def run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step, per_call=1):
     """Same step, but every input starts in pinned host memory and every decode output is read
     back: K, V, Q_win are uploaded layer by layer before qp_compress_layer, each decode step
     uploads its queries and downloads its outputs."""
@@ -335,8 +366,13 @@ def run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step):
     hout = [torch.empty((n_dec,) + tuple(sq["out"].shape), dtype=torch.bfloat16).pin_memory() for sq in seqs]
     dK, dV, dQ = torch.empty_like(seqs[0]["K"][0]), torch.empty_like(seqs[0]["V"][0]), torch.empty_like(seqs[0]["Qw"][0])
     dq = [torch.empty_like(sq["qdec"][0]) for sq in seqs]
-    batches = [qp.LayerBatch([dq[i][l] for l in range(n_layers)], sq["cache"],
-                             [sq["out"][l] for l in range(n_layers)], sq["ws_d"]) for i, sq in enumerate(seqs)]
+    groups = []
+    for g0 in range(0, len(seqs), per_call):
+        ids = list(range(g0, g0 + per_call))
+        ws_g = torch.empty(sum(seqs[i]["ws_d"].numel() for i in ids), dtype=torch.uint8, device=dev)
+        groups.append((ids, qp.LayerBatch([dq[i][l] for i in ids for l in range(n_layers)],
+                                          [c for i in ids for c in seqs[i]["cache"]],
+                                          [seqs[i]["out"][l] for i in ids for l in range(n_layers)], ws_g)))
     h2d = sum(t.numel() * 2 for per in (hK, hV, hQ) for s in per for t in s) + sum(t.numel() * 2 for t in hq)
     d2h = sum(t.numel() * 2 for t in hout)
 
@@ -350,10 +386,12 @@ def run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step):
                                   sq["cache"][l], sq["kept"][l], ws_c)
         b = torch.cuda.Event(enable_timing=True); b.record(stream)
         for t in range(n_dec):
-            for i, sq in enumerate(seqs):
-                dq[i].copy_(hq[i][t], non_blocking=True)
-                qp.decode_attn_layers(batches[i])
-                hout[i][t].copy_(sq["out"], non_blocking=True)
+            for ids, batch in groups:
+                for i in ids:
+                    dq[i].copy_(hq[i][t], non_blocking=True)
+                qp.decode_attn_layers(batch)
+                for i in ids:
+                    hout[i][t].copy_(seqs[i]["out"], non_blocking=True)
         c = torch.cuda.Event(enable_timing=True); c.record(stream)
         return a, b, c
 
@@ -374,12 +412,19 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="qp", choices=["qp", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--sequences", type=int, default=4,
+    ap.add_argument("--sequences", type=int, default=8,
                     help="independent sequences per GPU (their packed caches together exceed L2)")
+    ap.add_argument("--seqs-per-call", type=int, default=4,
+                    help="sequences whose layers go into one qp_decode_attn_layers call")
+    ap.add_argument("--layers", type=int, default=0, help="profiling: keep only the first N layers of the workload")
+    ap.add_argument("--batch", type=int, default=0, help="profiling: override the workload's batch size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
+    if args.layers or args.batch:      # a cut-down case of the same kernels, for ncu captures; never the bench line
+        wl = synth.dataclasses.replace(wl, n_layers=args.layers or wl.n_layers, batch=args.batch or wl.batch,
+                                       name=f"{wl.name}[layers={args.layers or wl.n_layers},batch={args.batch or wl.batch}]")
     if args.impl == "reference":
         run_reference(args, wl)
     else:
