@@ -315,7 +315,7 @@ def run_gpu(args, wl):
     achieved = dec_bytes_call / (call_ms * 1e-3) / 1e9
     sha = hashlib.sha256(b"".join(open(os.path.join(ROOT, "paper_2412_12706_b200", "csrc", f), "rb").read()
                                   for f in DECODE_KERNEL_SOURCES)).hexdigest()
-    traffic = NCU_TRAFFIC.get("bytes_per_launch") if NCU_TRAFFIC.get("sha256") == sha and \
+    traffic = NCU_TRAFFIC["bytes_per_launch_per_sequence"] * per_call if NCU_TRAFFIC.get("sha256") == sha and \
         NCU_TRAFFIC.get("workload") == wl.name else None
     cpu = oracle_sample(wl, 1, 0) if world == 1 and not args.no_cpu_baseline else None
     line = {
