@@ -66,12 +66,18 @@ struct ScoreDims {
 };
 // workspace carving for S1 (all offsets 256-byte aligned)
 struct ScoreWorkspace {
-  size_t stat_partial, rowstat, votes_partial, pooled, total;
+  size_t stat_partial, rowstat, votes_partial, pooled, error, total;   // error: one int, the last 256 bytes
   int n_rb, n_tiles, n_vote_tiles;
 };
 ScoreWorkspace score_workspace(int Bt, int Hq, int Hkv, int L, int w);
 cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDims& d, float* scores, void* ws,
                                  cudaStream_t st);
+
+// tcgen05 / TMEM form of the two score sweeps (same outputs as score_sweep_kernel)
+bool score_tc_supported(int D);
+cudaError_t launch_score_sweep_tc(int pass, const bf16* q, const bf16* k, const ScoreDims& d, const ScoreWorkspace& s,
+                                  float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
+                                  int* error_word, cudaStream_t st);
 
 cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_keep, int32_t* kept, cudaStream_t st);
 

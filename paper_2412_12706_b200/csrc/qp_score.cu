@@ -192,6 +192,7 @@ ScoreWorkspace score_workspace(int Bt, int Hq, int Hkv, int L, int w) {
   s.rowstat = off;       off += align256((size_t)BH * s.n_rb * SC_RB * sizeof(float2));
   s.votes_partial = off; off += align256((size_t)BH * s.n_rb * P * sizeof(float));
   s.pooled = off;        off += align256((size_t)BH * P * sizeof(float));
+  s.error = off;         off += 256;
   s.total = off;
   return s;
 }
@@ -208,6 +209,19 @@ cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDim
   const bf16* q = static_cast<const bf16*>(Qwin);
   const bf16* k = static_cast<const bf16*>(K);
   dim3 g1(s.n_tiles, s.n_rb, BH), g2(s.n_vote_tiles, s.n_rb, BH);
+  if (score_tc_supported(d.D)) {
+    // 5th-generation tensor-core path; the word at s.error becomes 1 if a block ever gave up on a wait
+    int* err = reinterpret_cast<int*>(base + s.error);
+    cudaError_t e = cudaMemsetAsync(err, 0, sizeof(int), st);
+    if (e != cudaSuccess) return e;
+    e = launch_score_sweep_tc(1, q, k, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st);
+    if (e != cudaSuccess) return e;
+    rowstat_merge_kernel<<<BH * s.n_rb, SC_RB, 0, st>>>(stat_partial, s.n_rb, s.n_tiles, R, rowstat);
+    e = launch_score_sweep_tc(2, q, k, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st);
+    if (e != cudaSuccess) return e;
+    pool_kernel<<<dim3((P + 255) / 256, BH), 256, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);
+    return cudaGetLastError();
+  }
   if (d.D == 128) {
     score_sweep_kernel<128, 1><<<g1, SC_THREADS, 0, st>>>(q, k, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles,
                                                          scale_log2, stat_partial, nullptr, nullptr);

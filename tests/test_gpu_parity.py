@@ -85,6 +85,19 @@ def test_window_scores_close_to_oracle(Hq, Hkv, D, L, w, pool):
     assert np.array_equal(again.astype(np.float64), got)
 
 
+def test_window_scores_tensor_memory_path_reports_no_abandoned_wait():
+    # D = 128 runs on tcgen05/TMEM; every mbarrier wait there is bounded and a block that gives up sets the
+    # error word kept in the last 256 bytes of the workspace
+    wl = small(synth.LLAMA8B_8K, L=4096 + 77, batch=2)
+    k, v, qw = make_inputs(wl)
+    nbytes = qp.compress_workspace_bytes(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.L, wl.w)
+    ws = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device=DEV)
+    got = qp.window_scores(qw.to(DEV), k.to(DEV), wl.pool, workspace=ws).cpu().numpy().astype(np.float64)
+    assert int(ws[nbytes - 256:nbytes - 252].view(torch.int32).item()) == 0
+    ref = orc.scores(bits_u16(qw), bits_u16(k), wl.pool)
+    assert (np.abs(got - ref) / ref).max() < 5e-6
+
+
 def test_window_scores_zero_queries_closed_form():
     wl = small(synth.TINY, L=600, w=16)
     k, v, qw = make_inputs(wl)
