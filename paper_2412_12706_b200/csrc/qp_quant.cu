@@ -14,7 +14,7 @@ namespace qp {
 namespace {
 
 struct QParams {
-  float zf, sf;
+  float zf, sf, inv;     // inv = 1/sf, correctly rounded (0 when sf is 0 or infinite)
   __half z16, s16;
 };
 
@@ -25,14 +25,22 @@ __device__ __forceinline__ QParams group_params(float mn, float mx, int qmax) {
   const float range = __fsub_rn(mx, p.zf);
   p.s16 = __float2half_ru(__fdiv_rn(range, (float)qmax));   // scale: rounded up, so max never clips
   p.sf = __half2float(p.s16);
+  p.inv = p.sf != 0.f ? __frcp_rn(p.sf) : 0.f;
   return p;
 }
 
+// code = clamp(rint((x - z) / s)) with the true quotient.  The quotient is first estimated as
+// (x - z) * (1/s), which is within 2^-22 relative (< 1e-4 absolute for codes up to 255) of it, so the
+// rounded integer can only differ when the estimate lies that close to a half-integer; only then is
+// the IEEE division done.  The result is the same integer in every case.
 __device__ __forceinline__ uint32_t quant_code(float x, const QParams& p, int qmax) {
   if (p.sf == 0.f) return 0u;
-  float r = rintf(__fdiv_rn(__fsub_rn(x, p.zf), p.sf));
-  r = fminf(fmaxf(r, 0.f), (float)qmax);
-  return (uint32_t)r;
+  const float d = __fsub_rn(x, p.zf);
+  float q = __fmul_rn(d, p.inv);
+  float r = rintf(q);
+  if (fabsf(q - r) > 0.4995f) r = rintf(__fdiv_rn(d, p.sf));
+  // 0 <= r <= qmax already: x >= min >= z, and the scale was rounded up so (max - z)/s <= qmax (1 + 2^-23)
+  return min((uint32_t)r, (uint32_t)qmax);
 }
 
 template <int BITS>
@@ -102,13 +110,32 @@ gather_quant_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__
     const QParams p = group_params(mn, mx, QMAX);
     const size_t gi = ((size_t)bh * n + (size_t)u * g + e) * ngv + v;
     uint32_t* dst = Vc + gi * wpg;
-    for (int wd = 0; wd < wpg; ++wd) {
-      uint32_t word = 0;
-      // PER consecutive channels per word; PER is 16, 8 or 4 -> whole 16-byte loads for PER >= 8
+    // second sweep over the group in 16-byte pieces (8 channels); a piece fills 8/PER words
+    constexpr int WPP = PER >= 8 ? 1 : 8 / PER;                 // words completed per piece (PER 16: half a word)
+    uint32_t word = 0;
+    for (int c8 = 0; c8 < g; c8 += 8) {
+      const uint4 q = *reinterpret_cast<const uint4*>(src + c8);
+      const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+      uint32_t codes[8];
 #pragma unroll
-      for (int c = 0; c < PER; ++c)
-        word |= quant_code(bf16_bits_to_f32(src[wd * PER + c]), p, QMAX) << (c * BITS);
-      dst[wd] = word;
+      for (int i = 0; i < 4; ++i) {
+        codes[2 * i] = quant_code(bf16lo(ww[i]), p, QMAX);
+        codes[2 * i + 1] = quant_code(bf16hi(ww[i]), p, QMAX);
+      }
+      if constexpr (PER == 16) {                                // 2-bit: two pieces per word
+        const int sh = (c8 & 8) ? 16 : 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) word |= codes[i] << (sh + i * BITS);
+        if (c8 & 8) { dst[c8 / 16] = word; word = 0; }
+      } else {
+#pragma unroll
+        for (int wq = 0; wq < WPP; ++wq) {
+          uint32_t wv = 0;
+#pragma unroll
+          for (int i = 0; i < PER; ++i) wv |= codes[wq * PER + i] << (i * BITS);
+          dst[(c8 / 8) * WPP + wq] = wv;
+        }
+      }
     }
     Vs[gi] = p.s16;
     Vz[gi] = p.z16;

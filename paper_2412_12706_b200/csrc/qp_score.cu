@@ -145,22 +145,38 @@ score_sweep_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K, in
   }
 }
 
-// per row: M = max over tiles, Z = sum_i s_i * 2^(m_i - M); stores (M, 1/Z); rows beyond R get 1/Z = 0
-__global__ void __launch_bounds__(SC_RB)
+// per row: M = max over tiles, Z = sum_i s_i * 2^(m_i - M); stores (M, 1/Z); rows beyond R get 1/Z = 0.
+// One block per (batch, KV head, row block): thread (row, slice) folds tiles slice, slice+8, ... into a running
+// (max, sum) pair with coalesced reads across rows; the eight slices are then combined in a fixed order.
+constexpr int RM_SLICES = 8;
+__global__ void __launch_bounds__(SC_RB * RM_SLICES)
 rowstat_merge_kernel(const float2* __restrict__ stat_partial, int n_rb, int n_tiles, int R,
                      float2* __restrict__ rowstat) {
-  const int blk = blockIdx.x;  // bh * n_rb + rb
-  const int rb = blk % n_rb, row = threadIdx.x;
+  __shared__ float2 part[RM_SLICES][SC_RB];
+  const int blk = blockIdx.x, rb = blk % n_rb, row = threadIdx.x % SC_RB, sl = threadIdx.x / SC_RB;
   const float2* p = stat_partial + (size_t)blk * n_tiles * SC_RB + row;
-  float M = -INFINITY;
-  for (int i = 0; i < n_tiles; ++i) M = fmaxf(M, p[(size_t)i * SC_RB].x);
-  float Z = 0.f;
-  for (int i = 0; i < n_tiles; ++i) {
+  float m = -INFINITY, z = 0.f;
+  for (int i = sl; i < n_tiles; i += RM_SLICES) {
     const float2 s = p[(size_t)i * SC_RB];
-    if (s.x != -INFINITY) Z += s.y * exp2f(s.x - M);
+    if (s.x != -INFINITY) {
+      const float mn = fmaxf(m, s.x);
+      z = z * exp2f(m - mn) + s.y * exp2f(s.x - mn);
+      m = mn;
+    }
   }
-  const bool valid = rb * SC_RB + row < R;
-  rowstat[(size_t)blk * SC_RB + row] = make_float2(valid ? M : 0.f, valid ? __fdiv_rn(1.0f, Z) : 0.f);
+  part[sl][row] = make_float2(m, z);
+  __syncthreads();
+  if (sl == 0) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < RM_SLICES; ++k) M = fmaxf(M, part[k][row].x);
+    float Z = 0.f;
+#pragma unroll
+    for (int k = 0; k < RM_SLICES; ++k)
+      if (part[k][row].x != -INFINITY) Z += part[k][row].y * exp2f(part[k][row].x - M);
+    const bool valid = rb * SC_RB + row < R;
+    rowstat[(size_t)blk * SC_RB + row] = make_float2(valid ? M : 0.f, valid ? __fdiv_rn(1.0f, Z) : 0.f);
+  }
 }
 
 __global__ void __launch_bounds__(256)
@@ -188,7 +204,8 @@ ScoreWorkspace score_workspace(int Bt, int Hq, int Hkv, int L, int w) {
   s.n_tiles = (L + SC_TILE - 1) / SC_TILE;
   s.n_vote_tiles = (P + SC_TILE - 1) / SC_TILE;
   size_t off = 0;
-  s.stat_partial = off;  off += align256((size_t)BH * s.n_rb * s.n_tiles * SC_RB * sizeof(float2));
+  // (max, sum) per row and key tile; the tensor-memory sweep keeps one per 64-column half tile
+  s.stat_partial = off;  off += align256((size_t)BH * s.n_rb * s.n_tiles * 2 * SC_RB * sizeof(float2));
   s.rowstat = off;       off += align256((size_t)BH * s.n_rb * SC_RB * sizeof(float2));
   s.votes_partial = off; off += align256((size_t)BH * s.n_rb * P * sizeof(float));
   s.pooled = off;        off += align256((size_t)BH * P * sizeof(float));
@@ -216,7 +233,7 @@ cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDim
     if (e != cudaSuccess) return e;
     e = launch_score_sweep_tc(1, q, k, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st);
     if (e != cudaSuccess) return e;
-    rowstat_merge_kernel<<<BH * s.n_rb, SC_RB, 0, st>>>(stat_partial, s.n_rb, s.n_tiles, R, rowstat);
+    rowstat_merge_kernel<<<BH * s.n_rb, SC_RB * RM_SLICES, 0, st>>>(stat_partial, s.n_rb, 2 * s.n_tiles, R, rowstat);
     e = launch_score_sweep_tc(2, q, k, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st);
     if (e != cudaSuccess) return e;
     pool_kernel<<<dim3((P + 255) / 256, BH), 256, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);
@@ -229,7 +246,7 @@ cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDim
     score_sweep_kernel<64, 1><<<g1, SC_THREADS, 0, st>>>(q, k, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles,
                                                         scale_log2, stat_partial, nullptr, nullptr);
   }
-  rowstat_merge_kernel<<<BH * s.n_rb, SC_RB, 0, st>>>(stat_partial, s.n_rb, s.n_tiles, R, rowstat);
+  rowstat_merge_kernel<<<BH * s.n_rb, SC_RB * RM_SLICES, 0, st>>>(stat_partial, s.n_rb, s.n_tiles, R, rowstat);
   if (d.D == 128) {
     score_sweep_kernel<128, 2><<<g2, SC_THREADS, 0, st>>>(q, k, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles,
                                                          scale_log2, nullptr, rowstat, votes_partial);

@@ -4,7 +4,8 @@
 // 128-key tiles (N).  Per tile a single thread issues D/16 tcgen05.mma (bf16 x bf16 -> f32, both
 // operands K-major in shared memory with the 128-byte swizzle), the [128 x 128] logit tile lands in
 // tensor memory, and the four warps read it back with tcgen05.ld: TMEM lane = query row, so every
-// thread owns one row and the softmax statistics of sweep 1 need no shuffles at all.  Sweep 2 turns
+// thread owns one row (two warpgroups split the columns) and the softmax statistics of sweep 1 need
+// no shuffles at all.  Sweep 2 turns
 // the tile into probabilities and sums the columns over the rows with a shuffle transpose-reduce.
 // Two TMEM buffers and two shared-memory stages let the MMA of tile i+1 and the copy of tile i+2
 // run under the epilogue of tile i.
@@ -17,7 +18,7 @@ namespace qp {
 
 namespace {
 
-constexpr int TC_THREADS = 128;
+constexpr int TC_THREADS = 256;                     // two warpgroups: each reads half of the tile's columns
 constexpr int TC_M = 128, TC_N = 128;
 constexpr uint32_t TC_TMEM_COLS = 256;                // two accumulator buffers of 128 columns
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
@@ -83,6 +84,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 2^x by the hardware approximation (about 2 ulp; results below 2^-126 flush to 0)
+__device__ __forceinline__ float ex2a(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void cp_async16_zfill(uint32_t saddr, const void* gptr, bool valid) {
   const int n = valid ? 16 : 0;
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(saddr), "l"(gptr), "r"(n));
@@ -109,6 +116,7 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
   __shared__ float sVote[PASS == 2 ? 4 : 1][TC_N];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rloc = tid & (TC_M - 1), half = tid >> 7, wq = warp & 3;   // row in the block, column half, TMEM lane quarter
   const int split = blockIdx.x, rb = blockIdx.y, bh = blockIdx.z;
   const int b = bh / Hkv, hk = bh % Hkv, G = Hq / Hkv, P = L - w, R = G * w;
   const int tile_lo = split * tiles_per_block;
@@ -170,10 +178,10 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
   };
 
   // this thread's query row and its statistics
-  const int row = rb * TC_M + tid;
+  const int row = rb * TC_M + rloc;
   const int lim = min(P + (row % w), L - 1);            // last key this row may see
   float2 st = make_float2(0.f, 0.f);
-  if (PASS == 2) st = rowstat[(size_t)(bh * n_rb + rb) * TC_M + tid];
+  if (PASS == 2) st = rowstat[(size_t)(bh * n_rb + rb) * TC_M + rloc];
 
   cp_async_wait<1>();                                   // Q and the first K tile have landed
   asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
@@ -199,37 +207,39 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
     cp_async_commit();
 
     const int tile = tile_lo + j, key0 = tile * TC_N;
-    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (j & 1) * TC_N;
+    const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (j & 1) * TC_N + half * (TC_N / 2);
+    const int col0 = key0 + half * (TC_N / 2);
     if constexpr (PASS == 1) {
       float m = -INFINITY, s = 0.f;
 #pragma unroll 1
-      for (int c0 = 0; c0 < TC_N; c0 += 32) {
+      for (int c0 = 0; c0 < TC_N / 2; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + c0, v);
         float cm = -INFINITY;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          v[i] = key0 + c0 + i <= lim ? v[i] * scale_log2 : -INFINITY;
+          v[i] = col0 + c0 + i <= lim ? v[i] * scale_log2 : -INFINITY;
           cm = fmaxf(cm, v[i]);
         }
         if (cm != -INFINITY) {
           const float mn = fmaxf(m, cm);
           float acc = 0.f;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) acc += exp2f(v[i] - mn);
-          s = s * exp2f(m - mn) + acc;
+          for (int i = 0; i < 32; ++i) acc += ex2a(v[i] - mn);
+          s = s * ex2a(m - mn) + acc;
           m = mn;
         }
       }
-      stat_partial[((size_t)(bh * n_rb + rb) * n_tiles + tile) * TC_M + tid] = make_float2(m, s);
+      // one (max, sum) per row and 64-column half tile
+      stat_partial[(((size_t)(bh * n_rb + rb) * n_tiles + tile) * 2 + half) * TC_M + rloc] = make_float2(m, s);
     } else {
 #pragma unroll 1
-      for (int c0 = 0; c0 < TC_N; c0 += 32) {
+      for (int c0 = 0; c0 < TC_N / 2; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + c0, v);
 #pragma unroll
         for (int i = 0; i < 32; ++i)
-          v[i] = key0 + c0 + i <= lim ? exp2f(v[i] * scale_log2 - st.x) * st.y : 0.f;   // rows beyond R carry 1/Z = 0
+          v[i] = col0 + c0 + i <= lim ? ex2a(fmaf(v[i], scale_log2, -st.x)) * st.y : 0.f;   // rows beyond R carry 1/Z = 0
         // column sums over the warp's 32 rows: halve the value count, double the rows covered, five times
 #pragma unroll
         for (int hstep = 16; hstep >= 1; hstep >>= 1) {
@@ -242,10 +252,10 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
           }
         }
         // lane l now holds the sum of column c0 + l over the warp's 32 rows
-        sVote[warp][c0 + lane] = v[0];
+        sVote[wq][half * (TC_N / 2) + c0 + lane] = v[0];
       }
       __syncthreads();
-      if (key0 + tid < P)
+      if (tid < TC_N && key0 + tid < P)
         votes_partial[(size_t)(bh * n_rb + rb) * P + key0 + tid] =
             ((sVote[0][tid] + sVote[1][tid]) + sVote[2][tid]) + sVote[3][tid];
     }
