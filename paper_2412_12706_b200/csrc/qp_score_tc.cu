@@ -5,8 +5,8 @@
 // operands K-major in shared memory with the 128-byte swizzle), the [128 x 128] logit tile lands in
 // tensor memory, and the four warps read it back with tcgen05.ld: TMEM lane = query row, so every
 // thread owns one row (two warpgroups split the columns) and the softmax statistics of sweep 1 need
-// no shuffles at all.  Sweep 2 turns
-// the tile into probabilities and sums the columns over the rows with a shuffle transpose-reduce.
+// no shuffles at all.  Sweep 2 swaps the operands (TMEM lane = key, column = query row), so the vote
+// of a key is again a thread-local sum.
 // Two TMEM buffers and two shared-memory stages let the MMA of tile i+1 and the copy of tile i+2
 // run under the epilogue of tile i.
 //
@@ -113,9 +113,10 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
   __shared__ uint64_t bars[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int give_up;
-  __shared__ float sVote[PASS == 2 ? 4 : 1][TC_N];
+  __shared__ float sVote[PASS == 2 ? 2 : 1][TC_N];
+  __shared__ __align__(16) float2 sRow[PASS == 2 ? TC_M : 1];      // sweep 2: (M, 1/Z) of the block's rows
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5;
   const int rloc = tid & (TC_M - 1), half = tid >> 7, wq = warp & 3;   // row in the block, column half, TMEM lane quarter
   const int split = blockIdx.x, rb = blockIdx.y, bh = blockIdx.z;
   const int b = bh / Hkv, hk = bh % Hkv, G = Hq / Hkv, P = L - w, R = G * w;
@@ -172,16 +173,19 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
     for (int kb = 0; kb < D / 64; ++kb)
 #pragma unroll
       for (int k = 0; k < 4; ++k)
-        umma_bf16(tm, smem_desc(sQ + kb * (TC_M * 128) + k * 32), smem_desc(sK + kb * (TC_N * 128) + k * 32), IDESC,
-                  (kb | k) ? 1u : 0u);
+        if (PASS == 1)      // rows = queries, columns = keys
+          umma_bf16(tm, smem_desc(sQ + kb * (TC_M * 128) + k * 32), smem_desc(sK + kb * (TC_N * 128) + k * 32), IDESC,
+                    (kb | k) ? 1u : 0u);
+        else                // rows = keys, columns = queries
+          umma_bf16(tm, smem_desc(sK + kb * (TC_N * 128) + k * 32), smem_desc(sQ + kb * (TC_M * 128) + k * 32), IDESC,
+                    (kb | k) ? 1u : 0u);
     umma_commit(bar0 + (j & 1) * 8);
   };
 
   // this thread's query row and its statistics
   const int row = rb * TC_M + rloc;
   const int lim = min(P + (row % w), L - 1);            // last key this row may see
-  float2 st = make_float2(0.f, 0.f);
-  if (PASS == 2) st = rowstat[(size_t)(bh * n_rb + rb) * TC_M + rloc];
+  if (PASS == 2 && tid < TC_M) sRow[tid] = rowstat[(size_t)(bh * n_rb + rb) * TC_M + tid];   // visible after the next barrier
 
   cp_async_wait<1>();                                   // Q and the first K tile have landed
   asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
@@ -210,54 +214,62 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
     const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (j & 1) * TC_N + half * (TC_N / 2);
     const int col0 = key0 + half * (TC_N / 2);
     if constexpr (PASS == 1) {
+      // TMEM lane = query row: this thread folds its row's 64 columns into a running (max, sum)
       float m = -INFINITY, s = 0.f;
+      const bool all_visible = key0 + TC_N - 1 <= P;            // every row sees every key up to P
 #pragma unroll 1
       for (int c0 = 0; c0 < TC_N / 2; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + c0, v);
-        float cm = -INFINITY;
+        if (all_visible) {
+          float cm = v[0];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          v[i] = col0 + c0 + i <= lim ? v[i] * scale_log2 : -INFINITY;
-          cm = fmaxf(cm, v[i]);
-        }
-        if (cm != -INFINITY) {
-          const float mn = fmaxf(m, cm);
+          for (int i = 1; i < 32; ++i) cm = fmaxf(cm, v[i]);
+          const float mn = fmaxf(m, cm * scale_log2);           // scale > 0: max commutes with it
           float acc = 0.f;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) acc += ex2a(v[i] - mn);
-          s = s * ex2a(m - mn) + acc;
+          for (int i = 0; i < 32; ++i) acc += ex2a(fmaf(v[i], scale_log2, -mn));
+          s = fmaf(s, ex2a(m - mn), acc);
           m = mn;
+        } else {
+          float cm = -INFINITY;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            v[i] = col0 + c0 + i <= lim ? v[i] * scale_log2 : -INFINITY;
+            cm = fmaxf(cm, v[i]);
+          }
+          if (cm != -INFINITY) {
+            const float mn = fmaxf(m, cm);
+            float acc = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc += ex2a(v[i] - mn);
+            s = fmaf(s, ex2a(m - mn), acc);
+            m = mn;
+          }
         }
       }
       // one (max, sum) per row and 64-column half tile
       stat_partial[(((size_t)(bh * n_rb + rb) * n_tiles + tile) * 2 + half) * TC_M + rloc] = make_float2(m, s);
     } else {
+      // operands swapped: TMEM lane = key, column = query row, so a key's vote is a thread-local sum over
+      // the rows.  Only prefix keys (< P) are written and every row sees all of them: no mask needed;
+      // rows beyond R carry 1/Z = 0.
+      float vote = 0.f;
 #pragma unroll 1
       for (int c0 = 0; c0 < TC_N / 2; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + c0, v);
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          v[i] = col0 + c0 + i <= lim ? ex2a(fmaf(v[i], scale_log2, -st.x)) * st.y : 0.f;   // rows beyond R carry 1/Z = 0
-        // column sums over the warp's 32 rows: halve the value count, double the rows covered, five times
-#pragma unroll
-        for (int hstep = 16; hstep >= 1; hstep >>= 1) {
-          const bool upper = (lane & hstep) != 0;
-#pragma unroll
-          for (int i = 0; i < hstep; ++i) {
-            const float send = upper ? v[i] : v[i + hstep];
-            const float keep = upper ? v[i + hstep] : v[i];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, hstep);
-          }
+        for (int i = 0; i < 32; i += 2) {
+          const float4 ms = *reinterpret_cast<const float4*>(&sRow[half * (TC_N / 2) + c0 + i]);   // (M, 1/Z) x 2 rows
+          vote = fmaf(ex2a(fmaf(v[i], scale_log2, -ms.x)), ms.y, vote);
+          vote = fmaf(ex2a(fmaf(v[i + 1], scale_log2, -ms.z)), ms.w, vote);
         }
-        // lane l now holds the sum of column c0 + l over the warp's 32 rows
-        sVote[wq][half * (TC_N / 2) + c0 + lane] = v[0];
       }
+      sVote[half][rloc] = vote;
       __syncthreads();
       if (tid < TC_N && key0 + tid < P)
-        votes_partial[(size_t)(bh * n_rb + rb) * P + key0 + tid] =
-            ((sVote[0][tid] + sVote[1][tid]) + sVote[2][tid]) + sVote[3][tid];
+        votes_partial[(size_t)(bh * n_rb + rb) * P + key0 + tid] = sVote[0][tid] + sVote[1][tid];
     }
     asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
     __syncthreads();                                    // TMEM buffer j & 1 and sVote may be overwritten
