@@ -12,6 +12,7 @@ namespace qp {
 namespace {
 
 constexpr int TK_THREADS = 1024;
+constexpr int TK_UNROLL = 8;
 
 // monotone map float -> uint32 (larger float = larger integer); -0 is treated as +0
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -35,55 +36,102 @@ topk_kernel(const float* __restrict__ scores, int L, int w, int n_keep, int32_t*
   __shared__ unsigned hist[256];
   __shared__ unsigned sh_prefix, sh_need;
   __shared__ unsigned warp_gt[32], warp_eq[32];
-  __shared__ unsigned run_gt, run_eq;
 
   unsigned prefix = 0, mask = 0, need = (unsigned)k;
   for (int shift = 24; shift >= 0; shift -= 8) {
     if (tid < 256) hist[tid] = 0;
     __syncthreads();
-    for (int j = tid; j < P; j += TK_THREADS) {
-      const uint32_t u = order_key(s[j]);
-      if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1u);
+    // scores cluster in a few exponents, so most elements of a warp share a digit: lanes with equal digits
+    // elect one leader that adds their count (one shared-memory atomic per distinct digit and warp)
+    // (only worth it for the two leading digits; the trailing ones are spread out).  TK_UNROLL loads are
+    // issued before any of them is used, so a sweep costs one memory latency per TK_UNROLL * 1024 elements.
+    for (int base = 0; base < P; base += TK_UNROLL * TK_THREADS) {
+      float f[TK_UNROLL];
+#pragma unroll
+      for (int q = 0; q < TK_UNROLL; ++q) {
+        const int j = base + q * TK_THREADS + tid;
+        f[q] = j < P ? s[j] : 0.f;
+      }
+#pragma unroll
+      for (int q = 0; q < TK_UNROLL; ++q) {
+        const int j = base + q * TK_THREADS + tid;
+        if (base + q * TK_THREADS >= P) break;
+        const uint32_t u = order_key(f[q]);
+        const bool cand = j < P && (u & mask) == prefix;
+        const unsigned digit = (u >> shift) & 255u;
+        if (shift >= 16) {
+          const unsigned peers = __match_any_sync(0xffffffffu, cand ? digit : 256u + lane);
+          if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+        } else if (cand) {
+          atomicAdd(&hist[digit], 1u);
+        }
+      }
     }
     __syncthreads();
-    if (tid == 0) {
-      unsigned cum = 0;
-      int b = 255;
-      for (; b > 0; --b) {
-        if (cum + hist[b] >= need) break;
-        cum += hist[b];
+    if (warp == 0) {
+      // lane l owns bins 8l .. 8l+7; find the bin where the count from the top reaches `need`
+      unsigned c[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = hist[8 * lane + i]; tot += c[i]; }
+      unsigned suf = tot;                                   // bins of this lane and all higher lanes
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned v = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += v;
       }
-      sh_need = need - cum;                 // still to take among elements with this digit
-      sh_prefix = prefix | ((unsigned)b << shift);
+      const unsigned above = suf - tot;
+      if (above < need && suf >= need) {                    // exactly one lane
+        unsigned cum = above;
+        int bsel = 7;
+        for (; bsel > 0; --bsel) {
+          if (cum + c[bsel] >= need) break;
+          cum += c[bsel];
+        }
+        sh_need = need - cum;                               // still to take among elements with this digit
+        sh_prefix = prefix | ((unsigned)(8 * lane + bsel) << shift);
+      }
     }
     __syncthreads();
     prefix = sh_prefix;
     need = sh_need;
     mask |= 0xffu << shift;
-    __syncthreads();
   }
   const uint32_t T = prefix;   // image of the k-th largest score; `need` elements equal to it are kept
 
-  if (tid == 0) { run_gt = 0; run_eq = 0; }
-  __syncthreads();
-  for (int base = 0; base < P; base += TK_THREADS) {
-    const int j = base + tid;
-    uint32_t u = 0;
-    bool gt = false, eq = false;
-    if (j < P) { u = order_key(s[j]); gt = u > T; eq = u == T; }
-    const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-    const unsigned lt_mask = (1u << lane) - 1u;
-    if (lane == 0) { warp_gt[warp] = __popc(bg); warp_eq[warp] = __popc(be); }
-    __syncthreads();
-    unsigned pg = run_gt + __popc(bg & lt_mask), pe = run_eq + __popc(be & lt_mask);
-    for (int wp = 0; wp < warp; ++wp) { pg += warp_gt[wp]; pe += warp_eq[wp]; }
-    if (gt || (eq && pe < need)) out[pg + min(pe, need)] = j;
-    __syncthreads();
-    if (tid == TK_THREADS - 1) {
-      run_gt = pg + (gt ? 1u : 0u);
-      run_eq = pe + (eq ? 1u : 0u);
+  unsigned run_g = 0, run_e = 0;                            // kept / equal elements before this chunk (all threads agree)
+  for (int base0 = 0; base0 < P; base0 += TK_UNROLL * TK_THREADS) {
+    float f[TK_UNROLL];
+#pragma unroll
+    for (int q = 0; q < TK_UNROLL; ++q) {
+      const int j = base0 + q * TK_THREADS + tid;
+      f[q] = j < P ? s[j] : 0.f;
     }
-    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < TK_UNROLL; ++q) {
+      const int base = base0 + q * TK_THREADS;
+      if (base >= P) break;
+      const int j = base + tid;
+      const uint32_t u = order_key(f[q]);
+      const bool gt = j < P && u > T, eq = j < P && u == T;
+      const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+      const unsigned lt_mask = (1u << lane) - 1u;
+      if (lane == 0) { warp_gt[warp] = __popc(bg); warp_eq[warp] = __popc(be); }
+      __syncthreads();
+      // exclusive prefix of the 32 warp counts, computed by every warp with shuffles
+      unsigned wg = warp_gt[lane], we = warp_eq[lane], sg = wg, se = we;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned vg = __shfl_up_sync(0xffffffffu, sg, o), ve = __shfl_up_sync(0xffffffffu, se, o);
+        if (lane >= o) { sg += vg; se += ve; }
+      }
+      const unsigned tot_g = __shfl_sync(0xffffffffu, sg, 31), tot_e = __shfl_sync(0xffffffffu, se, 31);
+      const unsigned pre_g = __shfl_sync(0xffffffffu, sg - wg, warp), pre_e = __shfl_sync(0xffffffffu, se - we, warp);
+      const unsigned pg = run_g + pre_g + __popc(bg & lt_mask), pe = run_e + pre_e + __popc(be & lt_mask);
+      if (gt || (eq && pe < need)) out[pg + min(pe, need)] = j;
+      run_g += tot_g;
+      run_e += tot_e;
+      __syncthreads();                                      // warp_gt / warp_eq are rewritten by the next chunk
+    }
   }
 }
 
