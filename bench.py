@@ -293,6 +293,45 @@ def run_gpu(args, wl):
         torch.cuda.synchronize()
         single_ms = s0.elapsed_time(s1) / reps
 
+    # ---- and layer by layer: one qp_decode_attn call per layer, back to back, then the same chain replayed
+    #      from a CUDA graph (what a model's decode loop would do between its other kernels)
+    layer_ms = graph_ms = None
+    if not args.no_layer_chain:
+        sq0 = seqs[0]
+        qs0, outs0 = sq0["qdec"][0], sq0["out"]
+        ws_l = torch.empty(max(qp.decode_workspace_bytes(c) for c in sq0["cache"]), dtype=torch.uint8, device=dev)
+
+        def chain():
+            for l in range(n_layers):
+                qp.decode_attn(qs0[l], sq0["cache"][l], outs0[l], ws_l)
+        for _ in range(3):
+            chain()
+        reps = 16
+        c0, c1 = ev(), ev()
+        c0.record(stream)
+        for _ in range(reps):
+            chain()
+        c1.record(stream)
+        torch.cuda.synchronize()
+        layer_ms = c0.elapsed_time(c1) / reps
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            chain()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                chain()
+            for _ in range(3):
+                graph.replay()
+            g0, g1 = ev(), ev()
+            g0.record(side)
+            for _ in range(reps):
+                graph.replay()
+            g1.record(side)
+        torch.cuda.synchronize()
+        graph_ms = g0.elapsed_time(g1) / reps
+
     # ---- end to end: host buffers in, host buffers out, through the same calls
     input_bytes = 2 * n_seq * n_layers * Bt * Hkv * L * D * 2
     # the host-buffer leg pins a copy of every input; keep it to workloads whose inputs are a few GB
@@ -337,6 +376,12 @@ def run_gpu(args, wl):
         "decode_us_per_call": call_ms * 1e3,
         "decode_single_sequence_call": None if single_ms is None else {
             "us_per_call": single_ms * 1e3, "GB/s": dec_bytes_call / per_call / (single_ms * 1e-3) / 1e9},
+        "decode_layer_by_layer": None if layer_ms is None else {
+            "note": "one sequence, one qp_decode_attn call per layer (its packed cache fits in L2 for small workloads)",
+            "us_per_layer_call": layer_ms * 1e3 / n_layers,
+            "GB/s": dec_bytes_call / per_call / (layer_ms * 1e-3) / 1e9,
+            "cuda_graph_us_per_layer_call": graph_ms * 1e3 / n_layers,
+            "cuda_graph_GB/s": dec_bytes_call / per_call / (graph_ms * 1e-3) / 1e9},
         "decode_phase_ms_per_step": dec_ms / steps,
         "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "decode attention (split-K attention kernel + merge kernel, per call)",
@@ -425,6 +470,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling: keep only the first N layers of the workload")
     ap.add_argument("--batch", type=int, default=0, help="profiling: override the workload's batch size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-layer-chain", action="store_true", help="skip the layer-by-layer / CUDA-graph figures")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
