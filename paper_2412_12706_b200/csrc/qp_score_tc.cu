@@ -12,7 +12,7 @@
 //
 // Every wait on an mbarrier is bounded: if it runs out, the block records an error word, frees its
 // tensor memory and returns.  Outputs and their layout are the ones of score_sweep_kernel.
-#include "qp_common.cuh"
+#include "qp_mma.cuh"
 
 namespace qp {
 
@@ -101,14 +101,14 @@ __device__ __forceinline__ uint32_t sw128_off(int r, int c) {
   return (uint32_t)((c >> 3) * (TC_M * 128) + (r >> 3) * 1024 + (r & 7) * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-template <int PASS>
+template <int PASS, int D>
 __global__ void __launch_bounds__(TC_THREADS, 2)
 score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K, int Hq, int Hkv, int L, int w,
                       int n_rb, int n_tiles, int tiles_per_block, float scale_log2,
                       float2* __restrict__ stat_partial, const float2* __restrict__ rowstat,
                       float* __restrict__ votes_partial, int* __restrict__ error_word) {
-  constexpr int D = 128, CPR = D / 8;                  // 16-byte chunks per row
-  constexpr uint32_t OPER_BYTES = TC_M * D * 2;        // 32 KB per operand tile
+  constexpr int CPR = D / 8;                           // 16-byte chunks per row
+  constexpr uint32_t OPER_BYTES = TC_M * D * 2;        // one operand tile: D/64 swizzled blocks of 16 KB
   extern __shared__ unsigned char smem_raw[];
   __shared__ uint64_t bars[2];
   __shared__ uint32_t tmem_base_slot;
@@ -286,7 +286,22 @@ score_sweep_tc_kernel(const bf16* __restrict__ Qwin, const bf16* __restrict__ K,
 
 }  // namespace
 
-bool score_tc_supported(int D) { return D == 128; }
+bool score_tc_supported(int D) { return D == 128 || D == 64; }
+
+namespace {
+template <int PASS, int D>
+cudaError_t launch_tc(dim3 grid, cudaStream_t st, const bf16* q, const bf16* k, const ScoreDims& d, const ScoreWorkspace& s,
+                      int per, float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
+                      int* error_word) {
+  constexpr size_t smem = 3 * (size_t)TC_M * D * 2 + 1024;   // Q + two K stages + alignment slack
+  static unsigned char done[64] = {};
+  const cudaError_t e = allow_smem(score_sweep_tc_kernel<PASS, D>, smem, done);
+  if (e != cudaSuccess) return e;
+  score_sweep_tc_kernel<PASS, D><<<grid, TC_THREADS, smem, st>>>(q, k, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles, per, scale_log2,
+                                                                stat_partial, rowstat, votes_partial, error_word);
+  return cudaGetLastError();
+}
+}  // namespace
 
 cudaError_t launch_score_sweep_tc(int pass, const bf16* q, const bf16* k, const ScoreDims& d, const ScoreWorkspace& s,
                                   float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
@@ -298,30 +313,12 @@ cudaError_t launch_score_sweep_tc(int pass, const bf16* q, const bf16* k, const 
   if (per < 2) per = 2;
   if (per > 32) per = 32;
   const int splits = (int)((tiles + per - 1) / per);
-  constexpr size_t smem = 3 * TC_M * 128 * 2 + 1024;   // Q + two K stages + alignment slack
   const dim3 grid(splits, s.n_rb, BH);
-  static unsigned char done1[64] = {}, done2[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  cudaError_t e = cudaSuccess;
-  if (pass == 1) {
-    if (!done1[dev]) {
-      e = cudaFuncSetAttribute(score_sweep_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      done1[dev] = 1;
-    }
-    score_sweep_tc_kernel<1><<<grid, TC_THREADS, smem, st>>>(q, k, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles, (int)per,
-                                                            scale_log2, stat_partial, rowstat, votes_partial, error_word);
-  } else {
-    if (!done2[dev]) {
-      e = cudaFuncSetAttribute(score_sweep_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      done2[dev] = 1;
-    }
-    score_sweep_tc_kernel<2><<<grid, TC_THREADS, smem, st>>>(q, k, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles, (int)per,
-                                                            scale_log2, stat_partial, rowstat, votes_partial, error_word);
-  }
-  return cudaGetLastError();
+  if (d.D == 128)
+    return pass == 1 ? launch_tc<1, 128>(grid, st, q, k, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
+                     : launch_tc<2, 128>(grid, st, q, k, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
+  return pass == 1 ? launch_tc<1, 64>(grid, st, q, k, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
+                   : launch_tc<2, 64>(grid, st, q, k, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
 }
 
 }  // namespace qp
