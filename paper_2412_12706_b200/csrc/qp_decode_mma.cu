@@ -43,7 +43,7 @@ constexpr int DM_STAGES = QP_DM_STAGES;
 constexpr int SP_STRIDE = 80;            // bytes per column of the per-warp P buffer (8 columns)
 constexpr int SP_BYTES = 8 * SP_STRIDE;
 
-// byte offsets of one 32-token tile in shared memory, 4-bit codes, g = 32
+// byte offsets of one 32-token tile in shared memory, 4-bit codes (value scale/zero regions sized for g = 32)
 template <int D>
 struct Tile4 {
   static constexpr int KC = 0;                    // D rows of 16 B: one channel, 32 tokens
@@ -62,12 +62,14 @@ constexpr uint32_t M0 = 0x000f000fu;   // code in bits 0..3 of each half: value 
 constexpr uint32_t M1 = 0x00f000f0u;   // code in bits 4..7 of each half: value c * 2^-20
 constexpr float C24 = 16777216.0f, C20 = 1048576.0f;
 
-template <int D>
+template <int D, int GROUP>
 __global__ void __launch_bounds__(DM_THREADS, QP_DM_MINB)
 decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials) {
   using TL = Tile4<D>;
   constexpr int NC = D / 32;       // ldmatrix.x4 calls over the channels of a key tile = value groups per token
   constexpr int NPAIR = D / 8;     // channel pairs owned by one lane on the key side (D/4 channels)
+  constexpr int NG = D / GROUP;    // value scale groups per token
+  constexpr int GT = GROUP / 32;   // 32-token tiles per key group
   extern __shared__ __align__(128) unsigned char smem[];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
@@ -121,28 +123,30 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
     const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
 
     // global sources of this (layer, batch, KV head)
+    // (a key group of GROUP tokens is GROUP/2 bytes per channel: this tile's 32 tokens are 16 of them)
     const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * tph * D * 16;
-    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * tph * D * 2;
-    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * tph * D * 2;
+    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * (n / GROUP) * D * 2;
+    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * (n / GROUP) * D * 2;
     const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * (D / 2);
-    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * (D / 16);
-    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * (D / 16);
+    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * NG * 2;
+    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * NG * 2;
     const unsigned char* gKm = lane < MCH ? gKs : gKz;
     const unsigned char* gVm = lane < MCH ? gVs : gVz;
 
     // stage one tile: 16-byte asynchronous copies, destinations swizzled for the transposing loads
     auto issue_tile = [&](int tile, int stage) {
       const uint32_t sb = wsm_u + stage * TL::BYTES;
-      const unsigned char* kc = gKc + (size_t)tile * D * 16 + lane * 16;
+      const int u = tile / GT, sub = tile % GT;
+      const unsigned char* kc = gKc + (size_t)u * D * (GROUP / 2) + sub * 16 + lane * (GROUP / 2);
       const unsigned char* vc = gVc + (size_t)tile * 16 * D + lane * 16;
 #pragma unroll
       for (int i = 0; i < D / 32; ++i) {
-        cp_async16(sb + kdst[i], kc + i * 512);
+        cp_async16(sb + kdst[i], kc + i * 32 * (GROUP / 2));
         cp_async16(sb + vdst[i], vc + i * 512);
       }
       if (lane < 2 * MCH) {
-        cp_async16(sb + ksz_dst, gKm + (size_t)tile * D * 2 + mj * 16);
-        cp_async16(sb + vsz_dst, gVm + (size_t)tile * D * 2 + mj * 16);
+        cp_async16(sb + ksz_dst, gKm + (size_t)u * D * 2 + mj * 16);
+        if (mj < 4 * NG) cp_async16(sb + vsz_dst, gVm + (size_t)tile * 64 * NG + mj * 16);
       }
     };
 
@@ -259,30 +263,33 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       for (int pr = 0; pr < 4; ++pr) p2[pr] = lds32(sP + g * SP_STRIDE + 4 * t + 16 * pr);
 
       // ---------------- values: B = p * scale of the token's channel group, zero-point rows
-      uint32_t ps[4][NC], zp[4];
+      uint32_t ps[4][NG], zp[4];                                // ps[pair][scale group], zero-point rows: group g
 #pragma unroll
       for (int pr = 0; pr < 4; ++pr) {
         const int a = 8 * pr + 2 * t;                           // first token of the pair
         zp[pr] = 0u;
-        if constexpr (NC == 4) {
+        if constexpr (NG == 4) {
           const uint4 x = lds128(sb + TL::VS + a * 8);
           ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x5410));
           ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x7632));
           ps[pr][2] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x5410));
           ps[pr][3] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x7632));
-          if (g < NC) {                                         // rows of the zero-point MMA: value group v = g
-            const uint32_t ya = lds32(sb + TL::VZ + a * 8 + (g & 2) * 2);       // z[a][v & ~1], z[a][v | 1]
+          if (g < NG) {                                         // rows of the zero-point MMA: scale group g
+            const uint32_t ya = lds32(sb + TL::VZ + a * 8 + (g & 2) * 2);       // z[a][g & ~1], z[a][g | 1]
             const uint32_t yb = lds32(sb + TL::VZ + a * 8 + 8 + (g & 2) * 2);   // same of token a + 1
             zp[pr] = __byte_perm(ya, yb, (g & 1) ? 0x7632 : 0x5410);
           }
-        } else {
+        } else if constexpr (NG == 2) {
           const uint2 x = lds64(sb + TL::VS + a * 4);
           ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x5410));
           ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x7632));
-          if (g < NC) {
+          if (g < NG) {
             const uint2 y = lds64(sb + TL::VZ + a * 4);
             zp[pr] = __byte_perm(y.x, y.y, (g & 1) ? 0x7632 : 0x5410);
           }
+        } else {                                                // one scale per token: the pair is one word
+          ps[pr][0] = hmul2_u32(p2[pr], lds32(sb + TL::VS + a * 2));
+          if (g == 0) zp[pr] = lds32(sb + TL::VZ + a * 2);
         }
       }
       mma_f16_m16n8k16(accPZ, zp[0], 0u, zp[1], 0u, p2[0], p2[1]);
@@ -291,12 +298,12 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       for (int v = 0; v < NC; ++v) {
         uint32_t R0, R1, R2, R3;
         ldmatrix_x4_trans(R0, R1, R2, R3, sb + v_off[v]);
-        mma_f16_m16n8k16(accO[v][0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, ps[0][v], ps[1][v]);
+        mma_f16_m16n8k16(accO[v][0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, ps[0][v * NG / NC], ps[1][v * NG / NC]);
         const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
-        mma_f16_m16n8k16(accO[v][1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, ps[0][v], ps[1][v]);
-        mma_f16_m16n8k16(accO[v][0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, ps[2][v], ps[3][v]);
+        mma_f16_m16n8k16(accO[v][1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, ps[0][v * NG / NC], ps[1][v * NG / NC]);
+        mma_f16_m16n8k16(accO[v][0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, ps[2][v * NG / NC], ps[3][v * NG / NC]);
         const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
-        mma_f16_m16n8k16(accO[v][1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, ps[2][v], ps[3][v]);
+        mma_f16_m16n8k16(accO[v][1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, ps[2][v * NG / NC], ps[3][v * NG / NC]);
       }
     }
 
@@ -310,9 +317,9 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
     __syncthreads();                                            // every warp has consumed its last stage
 #pragma unroll
     for (int v = 0; v < NC; ++v) {
-      // zero-point term of channel group v for columns 2t, 2t+1 sits in lane (g = v, t)
-      const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * v + t);
-      const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * v + t);
+      // zero-point term of the scale group of channels 32v.. for columns 2t, 2t+1 sits in lane (g = group, t)
+      const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * (v * NG / NC) + t);
+      const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * (v * NG / NC) + t);
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
         const int ch = 32 * v + 4 * g + 2 * mt;
@@ -409,31 +416,34 @@ constexpr size_t mma4_smem_bytes() {
 bool decode_mma_supported(const DecDims& d) {
   if (d.D != 128 && d.D != 64) return false;
   if (d.bits == 16) return true;
-  if (d.group != 32) return false;
-  return d.bits == 4 || d.bits == 8 || decode_mma2_supported(d);
+  if (d.bits == 4 || d.bits == 8) return d.D % d.group == 0;   // groups of 32, 64, 128
+  return d.group == 32 && decode_mma2_supported(d);
 }
 
 int decode_mma_blocks_per_sm(const DecDims& d) {
   return d.bits == 8 ? decode_mma8_blocks_per_sm() : d.bits == 16 ? decode_mma16_blocks_per_sm() : QP_DM_MINB;
 }
 
-cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
-  const dim3 grid(tab.n_workers);
-  cudaError_t e;
-  if (d.D == 128) {
-    constexpr size_t smem = mma4_smem_bytes<128>();
-    static unsigned char done[64] = {};
-    e = allow_smem(decode_mma4_kernel<128>, smem, done);
-    if (e != cudaSuccess) return e;
-    decode_mma4_kernel<128><<<grid, DM_THREADS, smem, st>>>(tab, d, partials);
-  } else {
-    constexpr size_t smem = mma4_smem_bytes<64>();
-    static unsigned char done[64] = {};
-    e = allow_smem(decode_mma4_kernel<64>, smem, done);
-    if (e != cudaSuccess) return e;
-    decode_mma4_kernel<64><<<grid, DM_THREADS, smem, st>>>(tab, d, partials);
-  }
+namespace {
+template <int D, int GROUP>
+cudaError_t launch_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+  constexpr size_t smem = mma4_smem_bytes<D>();
+  static unsigned char done[64] = {};
+  const cudaError_t e = allow_smem(decode_mma4_kernel<D, GROUP>, smem, done);
+  if (e != cudaSuccess) return e;
+  decode_mma4_kernel<D, GROUP><<<dim3(tab.n_workers), DM_THREADS, smem, st>>>(tab, d, partials);
   return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+  if (d.D == 128) {
+    if (d.group == 32) return launch_mma4<128, 32>(tab, d, partials, st);
+    if (d.group == 64) return launch_mma4<128, 64>(tab, d, partials, st);
+    return launch_mma4<128, 128>(tab, d, partials, st);
+  }
+  if (d.group == 32) return launch_mma4<64, 32>(tab, d, partials, st);
+  return launch_mma4<64, 64>(tab, d, partials, st);
 }
 
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {

@@ -1,4 +1,4 @@
-// S4 on tensor cores for 8-bit caches (group 32).
+// S4 on tensor cores for 8-bit caches (groups of 32, 64 or 128).
 //
 // Same scheme as the 4-bit kernel: a byte c in the low byte of a 16-bit lane is the f16 number
 // c * 2^-24 (255 is still below the end of the first binade), so (word & 0x00ff00ff) and a byte
@@ -38,11 +38,12 @@ constexpr uint32_t M8 = 0x00ff00ffu;
 constexpr float C24 = 16777216.0f;
 __device__ __forceinline__ uint32_t odd_bytes(uint32_t r) { return __byte_perm(r, 0u, 0x4341); }
 
-template <int D>
+template <int D, int GROUP>
 __global__ void __launch_bounds__(D8_THREADS, D8_MINB)
 decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials) {
   using TL = Tile8<D>;
-  constexpr int NC = D / 32;       // value scale groups per token
+  constexpr int NG = D / GROUP;    // value scale groups per token
+  constexpr int GT = GROUP / 32;   // 32-token tiles per key group
   constexpr int NQ = D / 16;       // 16-byte pieces per value row = k-steps over the key channels
   constexpr int NPAIR = D / 8;     // channel pairs owned by one lane on the key side
   extern __shared__ __align__(128) unsigned char smem[];
@@ -89,30 +90,31 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
     const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
 
     const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * tph * D * 32;
-    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * tph * D * 2;
-    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * tph * D * 2;
+    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * (n / GROUP) * D * 2;
+    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * (n / GROUP) * D * 2;
     const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * D;
-    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * (D / 16);
-    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * (D / 16);
+    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * NG * 2;
+    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * NG * 2;
     const unsigned char* gKm = lane < MCH ? gKs : gKz;
     const unsigned char* gVm = lane < MCH ? gVs : gVz;
 
     auto issue_tile = [&](int tile, int stage) {
       const uint32_t sb = wsm_u + stage * TL::BYTES;
-      const unsigned char* kc = gKc + (size_t)tile * D * 32 + lane * 16;
+      const int u = tile / GT, sub = tile % GT;                 // a key group is GROUP bytes per channel
+      const unsigned char* kc = gKc + (size_t)u * D * GROUP + sub * 32;
       const unsigned char* vc = gVc + (size_t)tile * 32 * D + lane * 16;
 #pragma unroll
       for (int i = 0; i < D / 16; ++i) {
         const int pi = lane + 32 * i;                           // key piece: channel pi/2, token half pi&1
         const int c = pi >> 1, hf = pi & 1;
-        cp_async16(sb + TL::KC + hf * 16 * D + ((c ^ ((c / (D / 4)) << 1)) << 4), kc + i * 512);
+        cp_async16(sb + TL::KC + hf * 16 * D + ((c ^ ((c / (D / 4)) << 1)) << 4), kc + c * GROUP + hf * 16);
         const int tau = pi / NQ, q = pi % NQ;                   // value piece: token tau, channels 16q .. 16q+15
         const int sw = NQ == 8 ? (tau & 7) : ((tau >> 1) & 3);
         cp_async16(sb + TL::VC + tau * D + ((q ^ sw) << 4), vc + i * 512);
       }
       if (lane < 2 * MCH) {
-        cp_async16(sb + ksz_dst, gKm + (size_t)tile * D * 2 + mj * 16);
-        cp_async16(sb + vsz_dst, gVm + (size_t)tile * D * 2 + mj * 16);
+        cp_async16(sb + ksz_dst, gKm + (size_t)u * D * 2 + mj * 16);
+        if (mj < 4 * NG) cp_async16(sb + vsz_dst, gVm + (size_t)tile * 64 * NG + mj * 16);
       }
     };
 
@@ -222,30 +224,33 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       for (int pr = 0; pr < 4; ++pr) p2[pr] = lds32(sP + g * SP8_STRIDE + 4 * t + 16 * pr);
 
       // ---------------- values
-      uint32_t ps[4][NC], zp[4];
+      uint32_t ps[4][NG], zp[4];                                // ps[pair][scale group], zero-point rows: group g
 #pragma unroll
       for (int pr = 0; pr < 4; ++pr) {
         const int a = 8 * pr + 2 * t;
         zp[pr] = 0u;
-        if constexpr (NC == 4) {
+        if constexpr (NG == 4) {
           const uint4 x = lds128(sb + TL::VS + a * 8);
           ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x5410));
           ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x7632));
           ps[pr][2] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x5410));
           ps[pr][3] = hmul2_u32(p2[pr], __byte_perm(x.y, x.w, 0x7632));
-          if (g < NC) {
+          if (g < NG) {
             const uint32_t ya = lds32(sb + TL::VZ + a * 8 + (g & 2) * 2);
             const uint32_t yb = lds32(sb + TL::VZ + a * 8 + 8 + (g & 2) * 2);
             zp[pr] = __byte_perm(ya, yb, (g & 1) ? 0x7632 : 0x5410);
           }
-        } else {
+        } else if constexpr (NG == 2) {
           const uint2 x = lds64(sb + TL::VS + a * 4);
           ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x5410));
           ps[pr][1] = hmul2_u32(p2[pr], __byte_perm(x.x, x.y, 0x7632));
-          if (g < NC) {
+          if (g < NG) {
             const uint2 y = lds64(sb + TL::VZ + a * 4);
             zp[pr] = __byte_perm(y.x, y.y, (g & 1) ? 0x7632 : 0x5410);
           }
+        } else {                                                // one scale per token: the pair is one word
+          ps[pr][0] = hmul2_u32(p2[pr], lds32(sb + TL::VS + a * 2));
+          if (g == 0) zp[pr] = lds32(sb + TL::VZ + a * 2);
         }
       }
       mma_f16_m16n8k16(accPZ, zp[0], 0u, zp[1], 0u, p2[0], p2[1]);
@@ -254,8 +259,8 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       for (int q = 0; q < NQ; ++q) {                            // rows: channels 16q + 2g (g) and 16q + 2g + 1 (g+8)
         uint32_t R0, R1, R2, R3;
         ldmatrix_x4_trans(R0, R1, R2, R3, sb + v_row + ((q ^ v_sw) << 4));
-        mma_f16_m16n8k16(accO[q], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), ps[0][q / 2], ps[1][q / 2]);
-        mma_f16_m16n8k16(accO[q], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), ps[2][q / 2], ps[3][q / 2]);
+        mma_f16_m16n8k16(accO[q], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), ps[0][q * NG / NQ], ps[1][q * NG / NQ]);
+        mma_f16_m16n8k16(accO[q], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), ps[2][q * NG / NQ], ps[3][q * NG / NQ]);
       }
     }
 
@@ -269,7 +274,7 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
     __syncthreads();
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
-      const int v = q / 2;
+      const int v = q * NG / NQ;                                // scale group of channels 16q ..
       const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * v + t);
       const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * v + t);
       const int ch = 16 * q + 2 * g;
@@ -321,23 +326,26 @@ constexpr size_t mma8_smem_bytes() {
 
 int decode_mma8_blocks_per_sm() { return D8_MINB; }
 
-cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
-  const dim3 grid(tab.n_workers);
-  cudaError_t e;
-  if (d.D == 128) {
-    constexpr size_t smem = mma8_smem_bytes<128>();
-    static unsigned char done[64] = {};
-    e = allow_smem(decode_mma8_kernel<128>, smem, done);
-    if (e != cudaSuccess) return e;
-    decode_mma8_kernel<128><<<grid, D8_THREADS, smem, st>>>(tab, d, partials);
-  } else {
-    constexpr size_t smem = mma8_smem_bytes<64>();
-    static unsigned char done[64] = {};
-    e = allow_smem(decode_mma8_kernel<64>, smem, done);
-    if (e != cudaSuccess) return e;
-    decode_mma8_kernel<64><<<grid, D8_THREADS, smem, st>>>(tab, d, partials);
-  }
+namespace {
+template <int D, int GROUP>
+cudaError_t launch_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+  constexpr size_t smem = mma8_smem_bytes<D>();
+  static unsigned char done[64] = {};
+  const cudaError_t e = allow_smem(decode_mma8_kernel<D, GROUP>, smem, done);
+  if (e != cudaSuccess) return e;
+  decode_mma8_kernel<D, GROUP><<<dim3(tab.n_workers), D8_THREADS, smem, st>>>(tab, d, partials);
   return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+  if (d.D == 128) {
+    if (d.group == 32) return launch_mma8<128, 32>(tab, d, partials, st);
+    if (d.group == 64) return launch_mma8<128, 64>(tab, d, partials, st);
+    return launch_mma8<128, 128>(tab, d, partials, st);
+  }
+  if (d.group == 32) return launch_mma8<64, 32>(tab, d, partials, st);
+  return launch_mma8<64, 64>(tab, d, partials, st);
 }
 
 }  // namespace qp
