@@ -1,12 +1,64 @@
 // C ABI of the library: argument checks, workspace carving and launches.  No allocation,
 // no synchronisation, no host copies.
+#include <algorithm>
 #include <cstring>
+#include <map>
+#include <mutex>
+#include <utility>
+#include <vector>
 
 #include "qp_common.cuh"
 
 using namespace qp;
 
 namespace {
+
+// What the last decode call on each (device, stream) wrote through its merge kernel.  The attention kernel of
+// the next call on that stream is allowed to start while that merge kernel still runs (programmatic dependent
+// launch) only if none of its inputs overlaps those outputs; otherwise it is launched in plain stream order.
+// Host bookkeeping only: a few sorted address ranges per stream.
+class PrevOutputs {
+ public:
+  using Range = std::pair<uintptr_t, uintptr_t>;   // [begin, end)
+  // true if no range of `reads` touches what the previous call on this stream wrote; then records `writes`
+  bool check_and_record(int device, cudaStream_t st, const std::vector<Range>& reads, std::vector<Range>& writes) {
+    std::sort(writes.begin(), writes.end());
+    // after sorting by begin, writes[i].second becomes the largest end among writes[0..i]: a read [b, e) meets
+    // one of the writes that begin before e exactly when that running maximum exceeds b
+    for (size_t i = 1; i < writes.size(); ++i) writes[i].second = std::max(writes[i].second, writes[i - 1].second);
+    std::lock_guard<std::mutex> lock(mu_);
+    const auto key = std::make_pair(device, st);
+    auto it = prev_.find(key);
+    bool disjoint = !forgot_;                       // a stream seen for the first time has no earlier merge kernel
+    if (it != prev_.end()) {
+      disjoint = true;
+      const std::vector<Range>& w = it->second;
+      for (const Range& r : reads) {
+        const auto lo = std::lower_bound(w.begin(), w.end(), r.second,
+                                         [](const Range& x, uintptr_t end) { return x.first < end; });
+        if (lo != w.begin() && (lo - 1)->second > r.first) { disjoint = false; break; }
+      }
+    } else if (prev_.size() >= kMaxStreams) {       // bounded memory: forget, and stop trusting absence
+      prev_.clear();
+      forgot_ = true;
+      disjoint = false;
+    }
+    prev_[key].swap(writes);
+    return disjoint;
+  }
+
+ private:
+  static constexpr size_t kMaxStreams = 256;
+  std::mutex mu_;
+  std::map<std::pair<int, cudaStream_t>, std::vector<Range>> prev_;
+  bool forgot_ = false;
+};
+PrevOutputs g_prev_outputs;
+
+inline PrevOutputs::Range range_of(const void* p, size_t bytes) {
+  const uintptr_t b = reinterpret_cast<uintptr_t>(p);
+  return {b, b + bytes};
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool pow2_bits(int b) { return b == 2 || b == 4 || b == 8 || b == 16; }
@@ -191,7 +243,30 @@ qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cac
   }
   const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
   if (workspace_bytes < decode_plan(tab, d)) return QP_ERR_WORKSPACE;
-  return launch_decode(tab, d, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream)) == cudaSuccess
+  // everything the attention kernel reads before it waits for the stream's previous kernel, and what this
+  // call's merge kernel writes
+  std::vector<PrevOutputs::Range> reads, writes;
+  reads.reserve(7 * (size_t)n_layers);
+  writes.reserve((size_t)n_layers);
+  const size_t qo_bytes = (size_t)c0.batch * c0.n_q_heads * c0.head_dim * 2;
+  for (int l = 0; l < n_layers; ++l) {
+    const qp_cache& c = caches[l];
+    reads.push_back(range_of(q[l], qo_bytes));
+    reads.push_back(range_of(c.k_codes, c.k_codes_bytes));
+    reads.push_back(range_of(c.v_codes, c.v_codes_bytes));
+    if (c.bits < 16) {
+      reads.push_back(range_of(c.k_scale, c.k_meta_bytes));
+      reads.push_back(range_of(c.k_zero, c.k_meta_bytes));
+      reads.push_back(range_of(c.v_scale, c.v_meta_bytes));
+      reads.push_back(range_of(c.v_zero, c.v_meta_bytes));
+    }
+    writes.push_back(range_of(out[l], qo_bytes));
+  }
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) return QP_ERR_CUDA;
+  const bool overlap = g_prev_outputs.check_and_record(device, static_cast<cudaStream_t>(stream), reads, writes);
+  return launch_decode(tab, d, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream), overlap) ==
+                 cudaSuccess
              ? QP_OK : QP_ERR_CUDA;
 }
 

@@ -103,22 +103,25 @@ struct DecTable {
   int n_layers;
   int chunk;        // chunked kernel: tokens per split
   int total_tiles;  // flat-range kernel: tiles of all layers and heads
-  int n_workers;    // flat-range kernel: thread blocks, each owning total_tiles / n_workers consecutive tiles
+  int n_workers;    // flat-range kernel: workers (blocks or warps, by kernel), each owning total_tiles / n_workers consecutive tiles
   DecLayer l[QP_MAX_LAYERS];
 };
 struct DecDims {
   int Bt, Hq, Hkv, D, bits, group;
 };
-constexpr int kMaxDecodeWorkers = 1024;
+constexpr int kMaxDecodeWorkers = 2048;
 // Chooses the decomposition for the layers in tab (n and pointers already set), fills chunk / part_base or
 // tile_base / total_tiles / n_workers and returns the bytes of partial records the launch needs.
 size_t decode_plan(DecTable& tab, const DecDims& d);
 // Upper bound of decode_plan's result for one layer of n_keep tokens, whatever else is in the launch.
 size_t decode_workspace_bound(const DecDims& d, int n_keep);
-cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+// overlap_prev: the attention kernel may start while the stream's previous kernel (the merge of an earlier
+// decode call) still runs; the caller guarantees that this launch reads nothing that kernel writes.
+cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 // tensor-core split-K kernel and its merge
 bool decode_mma_supported(const DecDims& d);
-int decode_mma_blocks_per_sm(const DecDims& d);
-cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+int decode_mma_workers_per_sm(const DecDims& d);     // workers (see DecTable::n_workers) resident per SM
+int decode_mma_tiles_per_worker_min(const DecDims& d);   // small launches use fewer workers, not emptier ones
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 
 }  // namespace qp

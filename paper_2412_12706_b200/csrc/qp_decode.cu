@@ -228,9 +228,10 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
       tab.l[l].part_base = 0;
       T += (long long)BH * ((tab.l[l].n + 31) / 32);
     }
-    long long W = (long long)sm_count() * decode_mma_blocks_per_sm(d);
+    long long W = (long long)sm_count() * decode_mma_workers_per_sm(d);
     if (W > kMaxDecodeWorkers) W = kMaxDecodeWorkers;
-    if (W > (T + 3) / 4) W = (T + 3) / 4;                       // at least one tile per warp
+    const int tmin = decode_mma_tiles_per_worker_min(d);        // at least one tile per warp
+    if (W > (T + tmin - 1) / tmin) W = (T + tmin - 1) / tmin;
     if (W < 1) W = 1;
     while (W > 1 && T * W >= (1ll << 31)) W /= 2;               // the merge kernel's range arithmetic is 32-bit
     tab.total_tiles = (int)T;
@@ -258,8 +259,8 @@ size_t decode_workspace_bound(const DecDims& d, int n_keep) {
   return chunked > flat ? chunked : flat;
 }
 
-cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
-  if (decode_mma_supported(d)) return launch_decode_mma(tab, d, partials, st);
+cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev) {
+  if (decode_mma_supported(d)) return launch_decode_mma(tab, d, partials, st, overlap_prev);
   int max_splits = 1;
   for (int l = 0; l < tab.n_layers; ++l) max_splits = max(max_splits, (tab.l[l].n + tab.chunk - 1) / tab.chunk);
   const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);

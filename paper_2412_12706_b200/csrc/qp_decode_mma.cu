@@ -72,21 +72,21 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   constexpr int GT = GROUP / 32;   // 32-token tiles per key group
   extern __shared__ __align__(128) unsigned char smem[];
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);       // provably warp-uniform: cursors stay in uniform registers
   const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
-  const SkOwner sk{tab.total_tiles, tab.n_workers};
-  const int cta = blockIdx.x;
   asm volatile("griddepcontrol.launch_dependents;\n" ::);     // the merge grid may start to become resident
-  long long cur = sk.start(cta);
-  const long long f_end = sk.start(cta + 1);
+  // Every warp is a worker of its own: a contiguous range of the flat tile sequence, a private copy ring,
+  // one partial record per head it touches.  Warps of a block share nothing and never synchronise.
+  const int wk = blockIdx.x * DM_WARPS + warp;
+  if (wk >= tab.n_workers) return;
+  const SkOwner sk{tab.total_tiles, tab.n_workers};
+  const long long f0 = sk.start(wk);
+  const int total = (int)(sk.start(wk + 1) - f0);
+  if (total <= 0) return;
 
-  unsigned char* wsm = smem + warp * (DM_STAGES * TL::BYTES + SP_BYTES);
-  const uint32_t wsm_u = smem_u32(wsm);
+  const uint32_t wsm_u = smem_u32(smem + warp * (DM_STAGES * TL::BYTES + SP_BYTES));
   const uint32_t sP = wsm_u + DM_STAGES * TL::BYTES;
-  // combine buffer of a finished segment; it overlays the (then idle) stage buffers
-  float* s_acc = reinterpret_cast<float*>(smem);                // [warp][8][D]
-  float* s_m = s_acc + DM_WARPS * 8 * D;                        // [warp][8]
-  float* s_l = s_m + DM_WARPS * 8;
 
   // per-lane shared-memory offsets: destinations of the asynchronous copies, sources of the transposing loads
   uint32_t kdst[D / 32], vdst[D / 32], k_off, v_off[NC];
@@ -112,56 +112,77 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const uint32_t ksz_dst = (lane < MCH ? TL::KS : TL::KZ) + mj * 16 + (mj / 8) * 16;
   const uint32_t vsz_dst = (lane < MCH ? TL::VS : TL::VZ) + mj * 16;
 
-  int li = 0;
-  while (li + 1 < tab.n_layers && tab.l[li + 1].tile_base <= cur) ++li;
+  // Two cursors walk the range: the copy cursor (p_*) runs DM_STAGES - 1 tiles ahead of the compute cursor
+  // (c_*) and crosses head and layer boundaries without draining the ring.
+  int p_li = 0;
+  while (p_li + 1 < tab.n_layers && (long long)tab.l[p_li + 1].tile_base <= f0) ++p_li;
+  int p_tph = tab.l[p_li].n >> 5;
+  int p_bh = (int)(f0 - tab.l[p_li].tile_base) / p_tph, p_tile = (int)(f0 - tab.l[p_li].tile_base) % p_tph;
+  int c_li = p_li, c_bh = p_bh, c_tile = p_tile, c_tph = p_tph;
 
-  while (cur < f_end) {
-    const DecLayer& ly = tab.l[li];
-    const int n = ly.n, tph = n >> 5;                           // tiles per head in this layer
-    const int rel = (int)(cur - ly.tile_base), bh = rel / tph, tile_begin = rel % tph;
-    const int n_tiles = (int)min((long long)(tph - tile_begin), f_end - cur);
-    const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
-
-    // global sources of this (layer, batch, KV head)
-    // (a key group of GROUP tokens is GROUP/2 bytes per channel: this tile's 32 tokens are 16 of them)
-    const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * tph * D * 16;
-    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * (n / GROUP) * D * 2;
-    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * (n / GROUP) * D * 2;
-    const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * (D / 2);
-    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * NG * 2;
-    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * NG * 2;
-    const unsigned char* gKm = lane < MCH ? gKs : gKz;
-    const unsigned char* gVm = lane < MCH ? gVs : gVz;
-
-    // stage one tile: 16-byte asynchronous copies, destinations swizzled for the transposing loads
-    auto issue_tile = [&](int tile, int stage) {
-      const uint32_t sb = wsm_u + stage * TL::BYTES;
-      const int u = tile / GT, sub = tile % GT;
-      const unsigned char* kc = gKc + (size_t)u * D * (GROUP / 2) + sub * 16 + lane * (GROUP / 2);
-      const unsigned char* vc = gVc + (size_t)tile * 16 * D + lane * 16;
+  // per-lane sources of the tile under the copy cursor; *m: scale or zero array by lane
+  const unsigned char *gKc, *gKm, *gVc, *gVm;
+  auto set_head = [&]() {
+    const DecLayer& ly = tab.l[p_li];
+    const size_t n = (size_t)ly.n, bh = (size_t)p_bh;
+    const int u = p_tile / GT, sub = p_tile % GT;
+    // (a key group of GROUP tokens is GROUP/2 bytes per channel: a tile's 32 tokens are 16 of them)
+    gKc = static_cast<const unsigned char*>(ly.kc) + bh * n * (D / 2) + (size_t)u * D * (GROUP / 2) + sub * 16 +
+          lane * (GROUP / 2);
+    gVc = static_cast<const unsigned char*>(ly.vc) + bh * n * (D / 2) + (size_t)p_tile * 16 * D + lane * 16;
+    gKm = reinterpret_cast<const unsigned char*>(lane < MCH ? ly.ks : ly.kz) + (bh * (n / GROUP) + u) * D * 2 + mj * 16;
+    gVm = reinterpret_cast<const unsigned char*>(lane < MCH ? ly.vs : ly.vz) + (bh * n + (size_t)p_tile * 32) * NG * 2 +
+          mj * 16;
+  };
+  set_head();
+  // stage the tile under the copy cursor (16-byte asynchronous copies, destinations swizzled for the
+  // transposing loads), then advance the cursor
+  auto issue_tile = [&](uint32_t sb) {
 #pragma unroll
-      for (int i = 0; i < D / 32; ++i) {
-        cp_async16(sb + kdst[i], kc + i * 32 * (GROUP / 2));
-        cp_async16(sb + vdst[i], vc + i * 512);
-      }
-      if (lane < 2 * MCH) {
-        cp_async16(sb + ksz_dst, gKm + (size_t)u * D * 2 + mj * 16);
-        if (mj < 4 * NG) cp_async16(sb + vsz_dst, gVm + (size_t)tile * 64 * NG + mj * 16);
-      }
-    };
-
-    // tiles of this segment go round-robin to the warps; start the copies before anything else
-    const int n_my = warp < n_tiles ? (n_tiles - warp + DM_WARPS - 1) / DM_WARPS : 0;
-#pragma unroll
-    for (int s = 0; s < DM_STAGES - 1; ++s) {
-      if (s < n_my) issue_tile(tile_begin + warp + DM_WARPS * s, s);
-      cp_async_commit();
+    for (int i = 0; i < D / 32; ++i) {
+      cp_async16(sb + kdst[i], gKc + i * 32 * (GROUP / 2));
+      cp_async16(sb + vdst[i], gVc + i * 512);
     }
+    if (2 * MCH == 32 || lane < 2 * MCH) {
+      cp_async16(sb + ksz_dst, gKm);
+      if (NG == 4 || mj < 4 * NG) cp_async16(sb + vsz_dst, gVm);
+    }
+    if (++p_tile == p_tph) {
+      p_tile = 0;
+      if (++p_bh == BH) {
+        p_bh = 0;
+        if (++p_li < tab.n_layers) p_tph = tab.l[p_li].n >> 5;
+      }
+      if (p_li < tab.n_layers) set_head();
+    } else {
+      gVc += 16 * D;
+      gVm += 64 * NG;
+      if (GT == 1 || p_tile % GT == 0) {
+        gKc += D * (GROUP / 2) - (GT - 1) * 16;
+        gKm += D * 2;
+      } else {
+        gKc += 16;
+      }
+    }
+  };
+#pragma unroll
+  for (int s = 0; s < DM_STAGES - 1; ++s) {
+    if (s < total) issue_tile(wsm_u + s * TL::BYTES);
+    cp_async_commit();
+  }
+  uint32_t sb = wsm_u, sb_copy = wsm_u + (DM_STAGES - 1) * TL::BYTES;   // stage computed on / stage refilled
 
-    // B-side query fragments: column g of the MMAs is query head g of this KV head (columns >= G are 0);
-    // this lane holds the D/4 channels [t*D/4, (t+1)*D/4) as f16 pairs
-    uint32_t qh2[NPAIR];
-    {
+  uint32_t qh2[NPAIR];
+  float m_run[2], l_run[2], accO[NC][2][4], accPZ[4];
+  bool fresh = true, waited = false;
+
+  for (int it = 0; it < total; ++it) {
+    if (fresh) {
+      fresh = false;
+      const DecLayer& ly = tab.l[c_li];
+      const int b = c_bh / dm.Hkv, hk = c_bh % dm.Hkv;
+      // B-side query fragments: column g of the MMAs is query head g of this KV head (columns >= G are 0);
+      // this lane holds the D/4 channels [t*D/4, (t+1)*D/4) as f16 pairs
       const float scale_log2 = 1.4426950408889634f * rsqrtf((float)D);
       const uint16_t* qp = static_cast<const uint16_t*>(ly.q) + ((size_t)(b * dm.Hq + hk * G + g)) * D + (D / 4) * t;
 #pragma unroll
@@ -173,26 +194,25 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         qh2[i + 2] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);
         qh2[i + 3] = pack_half2(bf16lo(w4.w) * scale_log2, bf16hi(w4.w) * scale_log2);
       }
+      // running softmax state of columns 2t, 2t+1 and the accumulators
+      m_run[0] = m_run[1] = -INFINITY;
+      l_run[0] = l_run[1] = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) accPZ[e] = 0.f;
+#pragma unroll
+      for (int v = 0; v < NC; ++v)
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) accO[v][mt][e] = 0.f;
     }
 
-    // running softmax state of columns 2t, 2t+1 and the accumulators
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    float accO[NC][2][4], accPZ[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int v = 0; v < NC; ++v)
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) accO[v][mt][e] = 0.f;
-
-    for (int it = 0; it < n_my; ++it) {
+    {
       __syncwarp();                                             // everyone is done with the stage refilled below
-      if (it + DM_STAGES - 1 < n_my)
-        issue_tile(tile_begin + warp + DM_WARPS * (it + DM_STAGES - 1), (it + DM_STAGES - 1) % DM_STAGES);
+      if (it + DM_STAGES - 1 < total) issue_tile(sb_copy);
       cp_async_commit();
       cp_async_wait<DM_STAGES - 1>();
       __syncwarp();
-      const uint32_t sb = wsm_u + (it % DM_STAGES) * TL::BYTES;
 
       // ---------------- keys: logits of 32 tokens x 8 columns
       float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, accZ[4] = {0.f, 0.f, 0.f, 0.f};
@@ -225,25 +245,25 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       }
 
       // ---------------- running softmax (log2 domain)
-      float corr[2];
+      // m_run is a reference, not the exact running maximum: it is renewed only when a logit exceeds it by more
+      // than kSlack, so p = 2^(logit - m_run) stays below 2^kSlack (the f16 products p * scale keep 12 binades
+      // of headroom) and the accumulators are rescaled on a few tiles per head, found without any shuffle.
+      constexpr float kSlack = 4.f;
+      const float over = fmaxf(fmaxf(fmaxf(lg[0][0], lg[1][0]), fmaxf(lg[2][0], lg[3][0])) - m_run[0],
+                               fmaxf(fmaxf(lg[0][1], lg[1][1]), fmaxf(lg[2][1], lg[3][1])) - m_run[1]);
+      if (__any_sync(0xffffffffu, over > kSlack)) {
+        float corr[2];
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        float mx = fmaxf(fmaxf(lg[0][e], lg[1][e]), fmaxf(lg[2][e], lg[3][e]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-        const float mnew = fmaxf(m_run[e], mx);
-        corr[e] = ex2(m_run[e] - mnew);
-        m_run[e] = mnew;
-        float sum = 0.f;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          lg[j][e] = ex2(lg[j][e] - mnew);
-          sum += lg[j][e];
+        for (int e = 0; e < 2; ++e) {
+          float mx = fmaxf(fmaxf(lg[0][e], lg[1][e]), fmaxf(lg[2][e], lg[3][e]));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+          const float mnew = fmaxf(m_run[e], mx);
+          corr[e] = ex2(m_run[e] - mnew);
+          m_run[e] = mnew;
+          l_run[e] *= corr[e];
         }
-        l_run[e] = fmaf(l_run[e], corr[e], sum);                // lane-local partial over its 4 tokens
-      }
-      if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
 #pragma unroll
         for (int v = 0; v < NC; ++v)
 #pragma unroll
@@ -252,6 +272,16 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
             accO[v][mt][2] *= corr[0]; accO[v][mt][3] *= corr[1];
           }
         accPZ[0] *= corr[0]; accPZ[1] *= corr[1];
+      }
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        float sum = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          lg[j][e] = ex2(lg[j][e] - m_run[e]);
+          sum += lg[j][e];
+        }
+        l_run[e] += sum;                                        // lane-local partial over its 4 tokens
       }
 
       // ---------------- P through shared memory: [column][token] f16, then token pairs of column g
@@ -305,59 +335,51 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
         mma_f16_m16n8k16(accO[v][1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, ps[2][v * NG / NC], ps[3][v * NG / NC]);
       }
+      sb_copy = sb;
+      sb = sb + TL::BYTES == sP ? wsm_u : sb + TL::BYTES;
     }
 
-    // ---------------- per-warp result -> shared memory -> one partial per (head, block) and query head
+    // ---------------- end of this head's part of the range: one partial record per query head, from registers
+    if (++c_tile == c_tph || it == total - 1) {
 #pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
-      l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
-      l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
-    }
-    __syncthreads();                                            // every warp has consumed its last stage
-#pragma unroll
-    for (int v = 0; v < NC; ++v) {
-      // zero-point term of the scale group of channels 32v.. for columns 2t, 2t+1 sits in lane (g = group, t)
-      const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * (v * NG / NC) + t);
-      const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * (v * NG / NC) + t);
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        const int ch = 32 * v + 4 * g + 2 * mt;
-        float* o0 = s_acc + ((warp * 8 + 2 * t) * D);
-        float* o1 = o0 + D;
-        *reinterpret_cast<float2*>(o0 + ch) = make_float2(fmaf(accO[v][mt][0], C24, pz0), fmaf(accO[v][mt][2], C20, pz0));
-        *reinterpret_cast<float2*>(o1 + ch) = make_float2(fmaf(accO[v][mt][1], C24, pz1), fmaf(accO[v][mt][3], C20, pz1));
+      for (int e = 0; e < 2; ++e) {
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
       }
-    }
-    if (g == 0) {
-      s_m[warp * 8 + 2 * t] = m_run[0]; s_m[warp * 8 + 2 * t + 1] = m_run[1];
-      s_l[warp * 8 + 2 * t] = l_run[0]; s_l[warp * 8 + 2 * t + 1] = l_run[1];
-    }
-    __syncthreads();
-    const size_t slot = (size_t)li * BH + bh + cta;
-    for (int idx = tid; idx < G * D; idx += DM_THREADS) {
-      const int h = idx / D, d = idx % D;
-      float M = -INFINITY;
+      if (!waited) {                                            // the previous call's merge may still read the records
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");
+        waited = true;
+      }
+      const size_t slot = (size_t)c_li * BH + c_bh + wk;
+      float* r0 = partials + (slot * G + 2 * t) * (size_t)(D + 2);      // record of column 2t; column 2t+1 follows
+      float* r1 = r0 + (D + 2);
+      const bool h0 = 2 * t < G, h1 = 2 * t + 1 < G;
 #pragma unroll
-      for (int wp = 0; wp < DM_WARPS; ++wp) M = fmaxf(M, s_m[wp * 8 + h]);
-      float Ls = 0.f, A = 0.f;
+      for (int v = 0; v < NC; ++v) {
+        // zero-point term of the scale group of channels 32v.. for columns 2t, 2t+1 sits in lane (g = group, t)
+        const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * (v * NG / NC) + t);
+        const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * (v * NG / NC) + t);
 #pragma unroll
-      for (int wp = 0; wp < DM_WARPS; ++wp) {
-        const float mw = s_m[wp * 8 + h];
-        if (mw != -INFINITY) {
-          const float f = ex2(mw - M);
-          Ls = fmaf(s_l[wp * 8 + h], f, Ls);
-          A = fmaf(s_acc[(wp * 8 + h) * D + d], f, A);
+        for (int mt = 0; mt < 2; ++mt) {
+          const int ch = 32 * v + 4 * g + 2 * mt;
+          if (h0) *reinterpret_cast<float2*>(r0 + 2 + ch) =
+                      make_float2(fmaf(accO[v][mt][0], C24, pz0), fmaf(accO[v][mt][2], C20, pz0));
+          if (h1) *reinterpret_cast<float2*>(r1 + 2 + ch) =
+                      make_float2(fmaf(accO[v][mt][1], C24, pz1), fmaf(accO[v][mt][3], C20, pz1));
         }
       }
-      float* o = partials + (slot * G + h) * (size_t)(D + 2);
-      if (d == 0) { o[0] = M; o[1] = Ls; }
-      o[2 + d] = A;
+      if (g == 0) {
+        if (h0) *reinterpret_cast<float2*>(r0) = make_float2(m_run[0], l_run[0]);
+        if (h1) *reinterpret_cast<float2*>(r1) = make_float2(m_run[1], l_run[1]);
+      }
+      c_tile = 0;
+      fresh = true;
+      if (++c_bh == BH) {
+        c_bh = 0;
+        if (++c_li < tab.n_layers) c_tph = tab.l[c_li].n >> 5;
+      }
     }
-    __syncthreads();                                            // the combine buffer is reused by the next segment
-
-    cur += n_tiles;
-    if (bh == BH - 1 && tile_begin + n_tiles == tph) ++li;
   }
 }
 
@@ -365,7 +387,9 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 // owner(first tile) .. owner(last tile); their records sit at slots head + block.
 // One warp per (layer, batch, query head), a lane per four channels.  The kernel is launched as a
 // programmatic dependent of the attention kernel: its blocks may become resident while that kernel
-// drains and wait at griddepcontrol.wait until its records are complete and visible.
+// drains and wait at griddepcontrol.wait until its records are complete and visible.  It passes the
+// permission on at once, so that the next call's attention kernel can fill the machine while this
+// one runs; that kernel reads none of this one's outputs and waits before it overwrites the records.
 constexpr int MG_WARPS = 4;
 __global__ void __launch_bounds__(MG_WARPS * 32)
 decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, const float* __restrict__ partials) {
@@ -382,17 +406,24 @@ decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, c
   const size_t head = (size_t)layer * BH + bh;
   const size_t stride = (size_t)G * (D + 2);
   const float* base = partials + (head * G + hl) * (size_t)(D + 2);
+  asm volatile("griddepcontrol.launch_dependents;\n" ::);
   asm volatile("griddepcontrol.wait;\n" ::: "memory");
-  if (!active || 4 * lane >= D) return;
+  if (!active) return;
+  // reference maxima of the records: a lane per record, then across the warp
   float M = -INFINITY;
-  for (int w = w_lo; w <= w_hi; ++w) M = fmaxf(M, base[w * stride]);
+  for (int w = w_lo + lane; w <= w_hi; w += 32) M = fmaxf(M, base[w * stride]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  if (4 * lane >= D) return;
   float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
+#pragma unroll 4
   for (int w = w_lo; w <= w_hi; ++w) {
     const float* r = base + w * stride;
-    const float f = ex2(r[0] - M);
+    const float2 ml = *reinterpret_cast<const float2*>(r);
     const float2 a01 = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
     const float2 a23 = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
-    Ls = fmaf(r[1], f, Ls);
+    const float f = ex2(ml.x - M);
+    Ls = fmaf(ml.y, f, Ls);
     A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
     A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
   }
@@ -405,11 +436,7 @@ decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, c
 }
 
 template <int D>
-constexpr size_t mma4_smem_bytes() {
-  constexpr size_t stages = (size_t)DM_WARPS * (DM_STAGES * Tile4<D>::BYTES + SP_BYTES);
-  constexpr size_t combine = (size_t)DM_WARPS * 8 * D * 4 + 2 * DM_WARPS * 8 * 4;
-  return stages > combine ? stages : combine;
-}
+constexpr size_t mma4_smem_bytes() { return (size_t)DM_WARPS * (DM_STAGES * Tile4<D>::BYTES + SP_BYTES); }
 
 }  // namespace
 
@@ -420,34 +447,50 @@ bool decode_mma_supported(const DecDims& d) {
   return d.group == 32 && decode_mma2_supported(d);
 }
 
-int decode_mma_blocks_per_sm(const DecDims& d) {
-  return d.bits == 8 ? decode_mma8_blocks_per_sm() : d.bits == 16 ? decode_mma16_blocks_per_sm() : QP_DM_MINB;
+// The 4-bit kernel's workers are warps; the other kernels' workers are blocks of four warps.
+int decode_mma_workers_per_sm(const DecDims& d) {
+  return d.bits == 4 ? QP_DM_MINB * DM_WARPS : d.bits == 8 ? decode_mma8_blocks_per_sm()
+         : d.bits == 16 ? decode_mma16_blocks_per_sm() : QP_DM_MINB;
 }
+// Small launches: four tiles per worker at least (a 4-bit worker is one warp, the others four warps with a tile
+// each); more, smaller records per head cost the merge kernel more than the attention kernel gains.
+int decode_mma_tiles_per_worker_min(const DecDims&) { return 4; }
 
 namespace {
 template <int D, int GROUP>
-cudaError_t launch_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+cudaError_t launch_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev) {
   constexpr size_t smem = mma4_smem_bytes<D>();
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(decode_mma4_kernel<D, GROUP>, smem, done);
   if (e != cudaSuccess) return e;
-  decode_mma4_kernel<D, GROUP><<<dim3(tab.n_workers), DM_THREADS, smem, st>>>(tab, d, partials);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((tab.n_workers + DM_WARPS - 1) / DM_WARPS);
+  cfg.blockDim = dim3(DM_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap_prev ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, decode_mma4_kernel<D, GROUP>, tab, d, partials);
 }
 }  // namespace
 
-cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
+                               bool overlap_prev) {
   if (d.D == 128) {
-    if (d.group == 32) return launch_mma4<128, 32>(tab, d, partials, st);
-    if (d.group == 64) return launch_mma4<128, 64>(tab, d, partials, st);
-    return launch_mma4<128, 128>(tab, d, partials, st);
+    if (d.group == 32) return launch_mma4<128, 32>(tab, d, partials, st, overlap_prev);
+    if (d.group == 64) return launch_mma4<128, 64>(tab, d, partials, st, overlap_prev);
+    return launch_mma4<128, 128>(tab, d, partials, st, overlap_prev);
   }
-  if (d.group == 32) return launch_mma4<64, 32>(tab, d, partials, st);
-  return launch_mma4<64, 64>(tab, d, partials, st);
+  if (d.group == 32) return launch_mma4<64, 32>(tab, d, partials, st, overlap_prev);
+  return launch_mma4<64, 64>(tab, d, partials, st, overlap_prev);
 }
 
-cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
-  cudaError_t e = d.bits == 4   ? launch_decode_mma4(tab, d, partials, st)
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
+                              bool overlap_prev) {
+  cudaError_t e = d.bits == 4   ? launch_decode_mma4(tab, d, partials, st, overlap_prev)
                   : d.bits == 8 ? launch_decode_mma8(tab, d, partials, st)
                   : d.bits == 16 ? launch_decode_mma16(tab, d, partials, st)
                                 : launch_decode_mma2(tab, d, partials, st);

@@ -73,7 +73,7 @@ def test_workspace_sizes():
     c = qp.cache_layout(1, 32, 8, 128, 4, 32, 2048)
     # (max, sum, acc[D]) records of G heads: the larger of one per 128-token split and one per
     # (KV head + worker block), the two decompositions the decode launch can choose from
-    assert qp.decode_workspace_bytes(c) == max(8 * (2048 // 128), 8 + 1024) * 4 * 130 * 4
+    assert qp.decode_workspace_bytes(c) == max(8 * (2048 // 128), 8 + 2048) * 4 * 130 * 4
 
 
 def test_bad_arguments_are_rejected_before_any_launch(lib):
