@@ -151,8 +151,13 @@ qp_status qp_compress_layer(const void* K, const void* V, const void* Q_win, int
  * S4 + S5, decode-step attention over the packed cache (Eq. 3 on the dequantized
  * cache of Eq. 5): out[b,h,:] = softmax_t(q[b,h].K'[t] / sqrt(D)) V' over the n kept
  * tokens of KV head h / G, no mask.  q, out bf16 [Bt,Hq,D] (device).  The token
- * range is split across thread blocks and the partial results merged; workspace
- * holds the partials.
+ * range is split across workers and the partial results merged; workspace (device,
+ * 16-byte aligned, contents irrelevant) holds the partials.  Consecutive calls on one
+ * stream may overlap on the GPU: the library starts a call's first kernel before the
+ * previous call has finished when this call reads none of the previous call's out
+ * buffers (it checks q and the cache arrays against them), and alternates between
+ * two halves of the workspace.  Results are as if the calls ran one after the other;
+ * calls on different streams must not share a workspace.
  */
 qp_status qp_decode_attn(const void* q, const qp_cache* cache /* host */, void* out, void* workspace,
                          size_t workspace_bytes, void* stream);
@@ -184,8 +189,8 @@ qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cac
  * library routine.  The first call on each device looks up the array's device address (with that
  * device current); make that first call outside any stream capture.  All calls on a device share
  * the one array and it keeps the previous call's contents (nothing in it needs clearing: each
- * call writes every record it later reads), so two calls whose kernels can overlap on the GPU,
- * e.g. on different streams, race on it; serialise them on one stream or with events.
+ * call writes every record it later reads), so two calls on different streams race on it;
+ * serialise them on one stream or with events.
  */
 #define QP_STATIC_SCRATCH_BYTES (4u << 20)
 qp_status qp_decode_attn_static(const void* q, const qp_cache* cache /* host */, void* out, void* stream);

@@ -20,8 +20,12 @@ namespace {
 class PrevOutputs {
  public:
   using Range = std::pair<uintptr_t, uintptr_t>;   // [begin, end)
-  // true if no range of `reads` touches what the previous call on this stream wrote; then records `writes`
-  bool check_and_record(int device, cudaStream_t st, const std::vector<Range>& reads, std::vector<Range>& writes) {
+  struct Decision {
+    bool overlap;   // no range of `reads` touches what the previous call on this stream wrote
+    int parity;     // workspace half of this call: alternates per (device, stream)
+  };
+  // decides for this call, then records `writes` as the stream's latest outputs
+  Decision check_and_record(int device, cudaStream_t st, const std::vector<Range>& reads, std::vector<Range>& writes) {
     std::sort(writes.begin(), writes.end());
     // after sorting by begin, writes[i].second becomes the largest end among writes[0..i]: a read [b, e) meets
     // one of the writes that begin before e exactly when that running maximum exceeds b
@@ -29,28 +33,35 @@ class PrevOutputs {
     std::lock_guard<std::mutex> lock(mu_);
     const auto key = std::make_pair(device, st);
     auto it = prev_.find(key);
-    bool disjoint = !forgot_;                       // a stream seen for the first time has no earlier merge kernel
+    Decision dec{!forgot_, 0};                      // a stream seen for the first time has no earlier decode kernel
     if (it != prev_.end()) {
-      disjoint = true;
-      const std::vector<Range>& w = it->second;
+      dec.overlap = true;
+      dec.parity = it->second.parity ^ 1;
+      const std::vector<Range>& w = it->second.outs;
       for (const Range& r : reads) {
         const auto lo = std::lower_bound(w.begin(), w.end(), r.second,
                                          [](const Range& x, uintptr_t end) { return x.first < end; });
-        if (lo != w.begin() && (lo - 1)->second > r.first) { disjoint = false; break; }
+        if (lo != w.begin() && (lo - 1)->second > r.first) { dec.overlap = false; break; }
       }
     } else if (prev_.size() >= kMaxStreams) {       // bounded memory: forget, and stop trusting absence
       prev_.clear();
       forgot_ = true;
-      disjoint = false;
+      dec.overlap = false;
     }
-    prev_[key].swap(writes);
-    return disjoint;
+    Entry& e = prev_[key];
+    e.outs.swap(writes);
+    e.parity = dec.parity;
+    return dec;
   }
 
  private:
+  struct Entry {
+    std::vector<Range> outs;
+    int parity = 0;
+  };
   static constexpr size_t kMaxStreams = 256;
   std::mutex mu_;
-  std::map<std::pair<int, cudaStream_t>, std::vector<Range>> prev_;
+  std::map<std::pair<int, cudaStream_t>, Entry> prev_;
   bool forgot_ = false;
 };
 PrevOutputs g_prev_outputs;
@@ -264,9 +275,9 @@ qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cac
   }
   int device = 0;
   if (cudaGetDevice(&device) != cudaSuccess) return QP_ERR_CUDA;
-  const bool overlap = g_prev_outputs.check_and_record(device, static_cast<cudaStream_t>(stream), reads, writes);
-  return launch_decode(tab, d, static_cast<float*>(workspace), static_cast<cudaStream_t>(stream), overlap) ==
-                 cudaSuccess
+  const PrevOutputs::Decision dec =
+      g_prev_outputs.check_and_record(device, static_cast<cudaStream_t>(stream), reads, writes);
+  return launch_decode(tab, d, workspace, dec.parity, static_cast<cudaStream_t>(stream), dec.overlap) == cudaSuccess
              ? QP_OK : QP_ERR_CUDA;
 }
 

@@ -115,13 +115,24 @@ constexpr int kMaxDecodeWorkers = 2048;
 size_t decode_plan(DecTable& tab, const DecDims& d);
 // Upper bound of decode_plan's result for one layer of n_keep tokens, whatever else is in the launch.
 size_t decode_workspace_bound(const DecDims& d, int n_keep);
-// overlap_prev: the attention kernel may start while the stream's previous kernel (the merge of an earlier
-// decode call) still runs; the caller guarantees that this launch reads nothing that kernel writes.
-cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
+// Workspace of the tensor-core kernels: two areas of partial records, used by alternate calls (parity), so that
+// a call's attention kernel can write its records while the previous call's merge kernel still reads its own.
+struct DecWorkspace {
+  size_t record_bytes;   // of one area, a multiple of 256
+  size_t total_bytes() const { return 2 * record_bytes; }
+};
+DecWorkspace decode_workspace_layout(const DecTable& tab, const DecDims& d);
+// parity: which half this call uses.  overlap_prev: the attention kernel may start while the stream's previous
+// kernel (an earlier decode call) still runs; the caller guarantees that this launch reads nothing that kernel
+// writes and that the earlier call used the other half.
+cudaError_t launch_decode(const DecTable& tab, const DecDims& d, void* workspace, int parity, cudaStream_t st,
+                          bool overlap_prev);
+int sm_count();   // SMs of the current device (cached)
 // tensor-core split-K kernel and its merge
 bool decode_mma_supported(const DecDims& d);
 int decode_mma_workers_per_sm(const DecDims& d);     // workers (see DecTable::n_workers) resident per SM
 int decode_mma_tiles_per_worker_min(const DecDims& d);   // small launches use fewer workers, not emptier ones
-cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
+cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
+                              bool overlap_prev);
 
 }  // namespace qp

@@ -192,8 +192,6 @@ decode_merge_kernel(const __grid_constant__ DecTable tab, const DecDims dm, cons
 
 }  // namespace
 
-namespace {
-
 int sm_count() {
   static int cached[64] = {};
   int dev = 0;
@@ -206,7 +204,10 @@ int sm_count() {
   return cached[dev];
 }
 
+namespace {
+
 size_t record_bytes(const DecDims& d) { return (size_t)(d.Hq / d.Hkv) * (size_t)(d.D + 2) * sizeof(float); }
+size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // chunked kernel: about eight blocks per SM, in whole 128-token units
 int chunk_tokens(long long total_tokens) {
@@ -237,7 +238,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
     tab.total_tiles = (int)T;
     tab.n_workers = (int)W;
     tab.chunk = 0;
-    return ((size_t)tab.n_layers * BH + (size_t)W) * record_bytes(d);
+    return decode_workspace_layout(tab, d).total_bytes();
   }
   long long total_tokens = 0;
   for (int l = 0; l < tab.n_layers; ++l) total_tokens += (long long)BH * tab.l[l].n;
@@ -252,15 +253,26 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
   return slots * record_bytes(d);
 }
 
+DecWorkspace decode_workspace_layout(const DecTable& tab, const DecDims& d) {
+  const size_t heads = (size_t)tab.n_layers * d.Bt * d.Hkv;
+  return DecWorkspace{round256((heads + (size_t)tab.n_workers) * record_bytes(d))};
+}
+
 size_t decode_workspace_bound(const DecDims& d, int n_keep) {
   const size_t BH = (size_t)d.Bt * d.Hkv;
   const size_t chunked = BH * (size_t)((n_keep + 127) / 128) * record_bytes(d);   // 128 tokens = smallest split
-  const size_t flat = (BH + kMaxDecodeWorkers) * record_bytes(d);
+  const size_t flat = 2 * round256((BH + kMaxDecodeWorkers) * record_bytes(d));
   return chunked > flat ? chunked : flat;
 }
 
-cudaError_t launch_decode(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev) {
-  if (decode_mma_supported(d)) return launch_decode_mma(tab, d, partials, st, overlap_prev);
+cudaError_t launch_decode(const DecTable& tab, const DecDims& d, void* workspace, int parity, cudaStream_t st,
+                          bool overlap_prev) {
+  if (decode_mma_supported(d)) {
+    const DecWorkspace ws = decode_workspace_layout(tab, d);
+    unsigned char* base = static_cast<unsigned char*>(workspace);
+    return launch_decode_mma(tab, d, reinterpret_cast<float*>(base + (parity ? ws.record_bytes : 0)), st, overlap_prev);
+  }
+  float* partials = static_cast<float*>(workspace);
   int max_splits = 1;
   for (int l = 0; l < tab.n_layers; ++l) max_splits = max(max_splits, (tab.l[l].n + tab.chunk - 1) / tab.chunk);
   const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);

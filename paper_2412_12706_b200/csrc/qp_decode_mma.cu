@@ -25,6 +25,8 @@
 // channels for values) while an MMA register pairs two elements along the contraction; the
 // transposing ldmatrix fetches 16-bit units of two different rows into one register, which is
 // exactly that pairing.  Shared-memory rows are XOR-swizzled so these loads are conflict-free.
+#include <algorithm>
+
 #include "qp_mma.cuh"
 
 namespace qp {
@@ -173,8 +175,21 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   uint32_t sb = wsm_u, sb_copy = wsm_u + (DM_STAGES - 1) * TL::BYTES;   // stage computed on / stage refilled
 
   uint32_t qh2[NPAIR];
-  float m_run[2], l_run[2], accO[NC][2][4], accPZ[4];
-  bool fresh = true, waited = false;
+  // running softmax reference of columns 2t, 2t+1 and the accumulators (cleared again after every record)
+  float m_run[2], accO[NC][2][4], accPZ[4];
+  auto clear_state = [&]() {
+    m_run[0] = m_run[1] = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) accPZ[e] = 0.f;
+#pragma unroll
+    for (int v = 0; v < NC; ++v)
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) accO[v][mt][e] = 0.f;
+  };
+  clear_state();
+  bool fresh = true;
 
   for (int it = 0; it < total; ++it) {
     if (fresh) {
@@ -190,21 +205,10 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         uint4 w4 = make_uint4(0u, 0u, 0u, 0u);
         if (g < G) w4 = *reinterpret_cast<const uint4*>(qp + 2 * i);
         qh2[i + 0] = pack_half2(bf16lo(w4.x) * scale_log2, bf16hi(w4.x) * scale_log2);
-        qh2[i + 1] = pack_half2(bf16lo(w4.y) * scale_log2, bf16hi(w4.y) * scale_log2);
-        qh2[i + 2] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);
+        qh2[i + 2] = pack_half2(bf16lo(w4.y) * scale_log2, bf16hi(w4.y) * scale_log2);   // order (0, 2, 1, 3): see
+        qh2[i + 1] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);   // the zero-point MMAs
         qh2[i + 3] = pack_half2(bf16lo(w4.w) * scale_log2, bf16hi(w4.w) * scale_log2);
       }
-      // running softmax state of columns 2t, 2t+1 and the accumulators
-      m_run[0] = m_run[1] = -INFINITY;
-      l_run[0] = l_run[1] = 0.f;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) accPZ[e] = 0.f;
-#pragma unroll
-      for (int v = 0; v < NC; ++v)
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) accO[v][mt][e] = 0.f;
     }
 
     {
@@ -215,46 +219,63 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       __syncwarp();
 
       // ---------------- keys: logits of 32 tokens x 8 columns
-      float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, accZ[4] = {0.f, 0.f, 0.f, 0.f};
+      // Zero-point term sum_d q'[h][d] z[d]: the roles are swapped (A = this lane's query pairs as they sit in
+      // registers, B = zero-point pairs as loaded), so no operand has to be copied into place.  With
+      // A = (qa, qc, qb, qd) and B = (z_a, z_b) rows g of the result hold qa z_a + qb z_b of head g, with
+      // B = (z_c, z_d) rows g+8 hold qc z_c + qd z_d; the other rows are never read.
+      float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      float accZa[4] = {0.f, 0.f, 0.f, 0.f}, accZb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < NC; ++c) {
         const uint4 s4 = lds128(sb + TL::KS + ksz_off((D / 4) * t + 8 * c));
         const uint4 z4 = lds128(sb + TL::KZ + ksz_off((D / 4) * t + 8 * c));
-        const uint32_t qs0 = hmul2_u32(qh2[4 * c + 0], s4.x), qs1 = hmul2_u32(qh2[4 * c + 1], s4.y);
-        const uint32_t qs2 = hmul2_u32(qh2[4 * c + 2], s4.z), qs3 = hmul2_u32(qh2[4 * c + 3], s4.w);
+        // qh2[4c + (0, 1, 2, 3)] hold the channel pairs (0, 2, 1, 3) of this lane's eight channels
+        const uint32_t qs0 = hmul2_u32(qh2[4 * c + 0], s4.x), qs1 = hmul2_u32(qh2[4 * c + 2], s4.y);
+        const uint32_t qs2 = hmul2_u32(qh2[4 * c + 1], s4.z), qs3 = hmul2_u32(qh2[4 * c + 3], s4.w);
         uint32_t R0, R1, R2, R3;
         ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_off + c * 128);
         mma_f16_m16n8k16(accK[0], R0 & M0, R0 & M1, R1 & M0, R1 & M1, qs0, qs1);
         const uint32_t S0 = R0 >> 8, S1 = R1 >> 8;
         mma_f16_m16n8k16(accK[1], S0 & M0, S0 & M1, S1 & M0, S1 & M1, qs0, qs1);
-        mma_f16_m16n8k16(accZ, z4.x, z4.x, z4.y, z4.y, qh2[4 * c + 0], qh2[4 * c + 1]);
+        mma_f16_m16n8k16(accZa, qh2[4 * c + 0], qh2[4 * c + 1], qh2[4 * c + 2], qh2[4 * c + 3], z4.x, z4.y);
         mma_f16_m16n8k16(accK[0], R2 & M0, R2 & M1, R3 & M0, R3 & M1, qs2, qs3);
         const uint32_t S2 = R2 >> 8, S3 = R3 >> 8;
         mma_f16_m16n8k16(accK[1], S2 & M0, S2 & M1, S3 & M0, S3 & M1, qs2, qs3);
-        mma_f16_m16n8k16(accZ, z4.z, z4.z, z4.w, z4.w, qh2[4 * c + 2], qh2[4 * c + 3]);
+        mma_f16_m16n8k16(accZb, qh2[4 * c + 0], qh2[4 * c + 1], qh2[4 * c + 2], qh2[4 * c + 3], z4.z, z4.w);
       }
+      // the term of head g sits in lanes (g, *); this lane needs those of columns 2t and 2t+1
+      const float zq = accZa[0] + accZb[2];
+      const float zq0 = __shfl_sync(0xffffffffu, zq, 8 * t), zq1 = __shfl_sync(0xffffffffu, zq, 8 * t + 4);
       // this lane: tokens 4g .. 4g+3 of the tile, columns 2t and 2t+1
-      //   lg[j][e]: token 4g + j, column 2t + e
-      float lg[4][2];
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        lg[2 * mt][0] = fmaf(accK[mt][0], C24, accZ[0]);
-        lg[2 * mt][1] = fmaf(accK[mt][1], C24, accZ[1]);
-        lg[2 * mt + 1][0] = fmaf(accK[mt][2], C20, accZ[0]);
-        lg[2 * mt + 1][1] = fmaf(accK[mt][3], C20, accZ[1]);
-      }
-
+      //   lg[j][e]: logit of token 4g + j, column 2t + e, minus the column's reference maximum
+      //
       // ---------------- running softmax (log2 domain)
       // m_run is a reference, not the exact running maximum: it is renewed only when a logit exceeds it by more
       // than kSlack, so p = 2^(logit - m_run) stays below 2^kSlack (the f16 products p * scale keep 12 binades
       // of headroom) and the accumulators are rescaled on a few tiles per head, found without any shuffle.
       constexpr float kSlack = 4.f;
-      const float over = fmaxf(fmaxf(fmaxf(lg[0][0], lg[1][0]), fmaxf(lg[2][0], lg[3][0])) - m_run[0],
-                               fmaxf(fmaxf(lg[0][1], lg[1][1]), fmaxf(lg[2][1], lg[3][1])) - m_run[1]);
-      if (__any_sync(0xffffffffu, over > kSlack)) {
+      const float zq_e[2] = {zq0, zq1};
+      float lg[4][2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float zm = zq_e[e] - m_run[e];                    // +inf on the first tile of a head
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          lg[2 * mt][e] = fmaf(accK[mt][e], C24, zm);
+          lg[2 * mt + 1][e] = fmaf(accK[mt][2 + e], C20, zm);
+        }
+      }
+      const float over = fmaxf(fmaxf(fmaxf(lg[0][0], lg[1][0]), fmaxf(lg[2][0], lg[3][0])),
+                               fmaxf(fmaxf(lg[0][1], lg[1][1]), fmaxf(lg[2][1], lg[3][1])));
+      if (__any_sync(0xffffffffu, over > kSlack)) {             // rare: renew the references, rescale
         float corr[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            lg[2 * mt][e] = fmaf(accK[mt][e], C24, zq_e[e]);
+            lg[2 * mt + 1][e] = fmaf(accK[mt][2 + e], C20, zq_e[e]);
+          }
           float mx = fmaxf(fmaxf(lg[0][e], lg[1][e]), fmaxf(lg[2][e], lg[3][e]));
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
           mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
@@ -262,7 +283,8 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
           const float mnew = fmaxf(m_run[e], mx);
           corr[e] = ex2(m_run[e] - mnew);
           m_run[e] = mnew;
-          l_run[e] *= corr[e];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) lg[j][e] -= mnew;
         }
 #pragma unroll
         for (int v = 0; v < NC; ++v)
@@ -274,15 +296,9 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         accPZ[0] *= corr[0]; accPZ[1] *= corr[1];
       }
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        float sum = 0.f;
+      for (int e = 0; e < 2; ++e)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          lg[j][e] = ex2(lg[j][e] - m_run[e]);
-          sum += lg[j][e];
-        }
-        l_run[e] += sum;                                        // lane-local partial over its 4 tokens
-      }
+        for (int j = 0; j < 4; ++j) lg[j][e] = ex2(lg[j][e]);    // p; its sum over the tokens: row NG of accPZ
 
       // ---------------- P through shared memory: [column][token] f16, then token pairs of column g
       sts64(sP + (2 * t) * SP_STRIDE + g * 8, pack_half2(lg[0][0], lg[1][0]), pack_half2(lg[2][0], lg[3][0]));
@@ -293,11 +309,13 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       for (int pr = 0; pr < 4; ++pr) p2[pr] = lds32(sP + g * SP_STRIDE + 4 * t + 16 * pr);
 
       // ---------------- values: B = p * scale of the token's channel group, zero-point rows
-      uint32_t ps[4][NG], zp[4];                                // ps[pair][scale group], zero-point rows: group g
+      // zero-point MMA: row g < NG holds the zero points of scale group g, row NG holds ones (the softmax
+      // denominator comes out of the same MMA, summed over the tokens in f32)
+      uint32_t ps[4][NG], zp[4];                                // ps[pair][scale group]
 #pragma unroll
       for (int pr = 0; pr < 4; ++pr) {
         const int a = 8 * pr + 2 * t;                           // first token of the pair
-        zp[pr] = 0u;
+        zp[pr] = g == NG ? 0x3c003c00u : 0u;
         if constexpr (NG == 4) {
           const uint4 x = lds128(sb + TL::VS + a * 8);
           ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x5410));
@@ -341,16 +359,8 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 
     // ---------------- end of this head's part of the range: one partial record per query head, from registers
     if (++c_tile == c_tph || it == total - 1) {
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
-        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
-        l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
-      }
-      if (!waited) {                                            // the previous call's merge may still read the records
-        asm volatile("griddepcontrol.wait;\n" ::: "memory");
-        waited = true;
-      }
+      // softmax denominators of columns 2t, 2t+1: row NG of the zero-point accumulator, lane (NG, t)
+      const float l0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * NG + t), l1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * NG + t);
       const size_t slot = (size_t)c_li * BH + c_bh + wk;
       float* r0 = partials + (slot * G + 2 * t) * (size_t)(D + 2);      // record of column 2t; column 2t+1 follows
       float* r1 = r0 + (D + 2);
@@ -370,9 +380,10 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         }
       }
       if (g == 0) {
-        if (h0) *reinterpret_cast<float2*>(r0) = make_float2(m_run[0], l_run[0]);
-        if (h1) *reinterpret_cast<float2*>(r1) = make_float2(m_run[1], l_run[1]);
+        if (h0) *reinterpret_cast<float2*>(r0) = make_float2(m_run[0], l0);
+        if (h1) *reinterpret_cast<float2*>(r1) = make_float2(m_run[1], l1);
       }
+      clear_state();
       c_tile = 0;
       fresh = true;
       if (++c_bh == BH) {
@@ -381,6 +392,11 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       }
     }
   }
+  // This kernel may have started while the previous call's merge kernel was still reading its records: alternate
+  // calls use alternate halves of the workspace, so nothing here had to wait for it.  The call after this one
+  // uses the previous call's half again; it starts its writes only after this grid has ended, and waiting here
+  // makes that imply that the previous call's merge has ended as well.
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
 // S5 for the decomposition above: head (layer, batch, KV head) was touched by the blocks
@@ -391,48 +407,53 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 // permission on at once, so that the next call's attention kernel can fill the machine while this
 // one runs; that kernel reads none of this one's outputs and waits before it overwrites the records.
 constexpr int MG_WARPS = 4;
-__global__ void __launch_bounds__(MG_WARPS * 32)
+// At most 32 registers per thread, so that a block fits beside the resident blocks of the attention kernel.  A
+// small launch (up to two blocks of work per SM) uses at most one block per SM: the whole grid is then resident
+// and has passed the launch permission on long before the attention kernel ends, the next call's attention
+// kernel fills the SMs as this call's drains, and this kernel runs in that kernel's shadow.  A large launch
+// would take too long that way; it uses a warp per output row and overlaps the next call's ramp only.
+__global__ void __launch_bounds__(MG_WARPS * 32, 16)
 decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, const float* __restrict__ partials) {
   const int D = dm.D, G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv, n_bq = dm.Bt * dm.Hq;
-  const int item = blockIdx.x * MG_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  const bool active = item < n_bq * tab.n_layers;
-  const int layer = active ? item / n_bq : 0, bq = active ? item % n_bq : 0;
-  const DecLayer& ly = tab.l[layer];
-  const int b = bq / dm.Hq, h = bq % dm.Hq, bh = b * dm.Hkv + h / G, hl = h % G;
+  const int lane = threadIdx.x & 31, n_items = n_bq * tab.n_layers;
   const unsigned T = (unsigned)tab.total_tiles, W = (unsigned)tab.n_workers;   // T * W < 2^31 (host-checked)
-  const int tph = (ly.n + 31) >> 5;
-  const unsigned first = (unsigned)ly.tile_base + (unsigned)bh * tph;
-  const int w_lo = (int)(((first + 1u) * W - 1u) / T), w_hi = (int)(((first + tph) * W - 1u) / T);
-  const size_t head = (size_t)layer * BH + bh;
   const size_t stride = (size_t)G * (D + 2);
-  const float* base = partials + (head * G + hl) * (size_t)(D + 2);
   asm volatile("griddepcontrol.launch_dependents;\n" ::);
   asm volatile("griddepcontrol.wait;\n" ::: "memory");
-  if (!active) return;
-  // reference maxima of the records: a lane per record, then across the warp
-  float M = -INFINITY;
-  for (int w = w_lo + lane; w <= w_hi; w += 32) M = fmaxf(M, base[w * stride]);
+  for (int item = blockIdx.x * MG_WARPS + (threadIdx.x >> 5); item < n_items; item += gridDim.x * MG_WARPS) {
+    const int layer = item / n_bq, bq = item % n_bq;
+    const DecLayer& ly = tab.l[layer];
+    const int b = bq / dm.Hq, h = bq % dm.Hq, bh = b * dm.Hkv + h / G, hl = h % G;
+    const int tph = (ly.n + 31) >> 5;
+    const unsigned first = (unsigned)ly.tile_base + (unsigned)bh * tph;
+    const int w_lo = (int)(((first + 1u) * W - 1u) / T), w_hi = (int)(((first + tph) * W - 1u) / T);
+    const size_t head = (size_t)layer * BH + bh;
+    const float* base = partials + (head * G + hl) * (size_t)(D + 2);
+    // reference maxima of the records: a lane per record, then across the warp
+    float M = -INFINITY;
+    for (int w = w_lo + lane; w <= w_hi; w += 32) M = fmaxf(M, base[w * stride]);
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-  if (4 * lane >= D) return;
-  float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
-#pragma unroll 4
-  for (int w = w_lo; w <= w_hi; ++w) {
-    const float* r = base + w * stride;
-    const float2 ml = *reinterpret_cast<const float2*>(r);
-    const float2 a01 = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
-    const float2 a23 = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
-    const float f = ex2(ml.x - M);
-    Ls = fmaf(ml.y, f, Ls);
-    A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
-    A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if (4 * lane >= D) continue;
+    float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
+#pragma unroll 2
+    for (int w = w_lo; w <= w_hi; ++w) {
+      const float* r = base + w * stride;
+      const float2 ml = *reinterpret_cast<const float2*>(r);
+      const float2 a01 = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
+      const float2 a23 = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
+      const float f = ex2(ml.x - M);
+      Ls = fmaf(ml.y, f, Ls);
+      A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
+      A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
+    }
+    const float inv = __fdiv_rn(1.0f, Ls);
+    __nv_bfloat162 o01 = __floats2bfloat162_rn(A0 * inv, A1 * inv), o23 = __floats2bfloat162_rn(A2 * inv, A3 * inv);
+    uint2 packed;
+    packed.x = *reinterpret_cast<uint32_t*>(&o01);
+    packed.y = *reinterpret_cast<uint32_t*>(&o23);
+    *reinterpret_cast<uint2*>(static_cast<bf16*>(ly.out) + (size_t)bq * D + 4 * lane) = packed;
   }
-  const float inv = __fdiv_rn(1.0f, Ls);
-  __nv_bfloat162 o01 = __floats2bfloat162_rn(A0 * inv, A1 * inv), o23 = __floats2bfloat162_rn(A2 * inv, A3 * inv);
-  uint2 packed;
-  packed.x = *reinterpret_cast<uint32_t*>(&o01);
-  packed.y = *reinterpret_cast<uint32_t*>(&o23);
-  *reinterpret_cast<uint2*>(static_cast<bf16*>(ly.out) + (size_t)bq * D + 4 * lane) = packed;
 }
 
 template <int D>
@@ -497,7 +518,8 @@ cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* part
   if (e != cudaSuccess) return e;
   const int items = d.Bt * d.Hq * tab.n_layers;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((items + MG_WARPS - 1) / MG_WARPS);
+  const int row_blocks = (items + MG_WARPS - 1) / MG_WARPS;
+  cfg.gridDim = dim3(row_blocks <= 2 * sm_count() ? std::min(row_blocks, sm_count()) : row_blocks);
   cfg.blockDim = dim3(MG_WARPS * 32);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = st;

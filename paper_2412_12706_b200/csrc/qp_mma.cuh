@@ -54,8 +54,9 @@ struct SkOwner {
 };
 
 
-// launchers of the per-bit-width attention kernels (grid = tab.n_workers blocks)
-cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
+// launchers of the per-bit-width attention kernels
+cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
+                               bool overlap_prev);
 cudaError_t launch_decode_mma2(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
 bool decode_mma2_supported(const DecDims& d);
 cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);

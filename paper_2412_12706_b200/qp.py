@@ -227,13 +227,18 @@ def compress_layer(K: torch.Tensor, V: torch.Tensor, Q_win: torch.Tensor, budget
     return cache, kept_idx
 
 
+def new_decode_workspace(nbytes: int, device) -> torch.Tensor:
+    """Scratch for the decode calls (contents irrelevant); reuse one per stream across calls."""
+    return torch.empty(max(16, nbytes), dtype=torch.uint8, device=device)
+
+
 def decode_attn(q: torch.Tensor, cache: Cache, out: torch.Tensor | None = None,
                 workspace: torch.Tensor | None = None) -> torch.Tensor:
     _dev_bf16(q)
     if out is None:
         out = torch.empty_like(q)
     if workspace is None:
-        workspace = torch.empty(max(16, decode_workspace_bytes(cache)), dtype=torch.uint8, device=q.device)
+        workspace = new_decode_workspace(decode_workspace_bytes(cache), q.device)
     _check(lib().qp_decode_attn(_ptr(q), ctypes.byref(cache.desc), _ptr(out), _ptr(workspace),
                                 workspace.numel(), _stream()), "qp_decode_attn")
     return out
@@ -252,8 +257,7 @@ class LayerBatch:
         self.out_arr = (ctypes.c_void_p * n)(*[t.data_ptr() for t in outs])
         self.cache_arr = (qp_cache * n)(*[c.desc for c in caches])
         if workspace is None:
-            nbytes = sum(decode_workspace_bytes(c) for c in caches)
-            workspace = torch.empty(max(16, nbytes), dtype=torch.uint8, device=qs[0].device)
+            workspace = new_decode_workspace(sum(decode_workspace_bytes(c) for c in caches), qs[0].device)
         self.workspace = workspace
 
 
