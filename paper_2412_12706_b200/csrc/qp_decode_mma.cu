@@ -484,17 +484,8 @@ cudaError_t launch_mma4(const DecTable& tab, const DecDims& d, float* partials, 
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(decode_mma4_kernel<D, GROUP>, smem, done);
   if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((tab.n_workers + DM_WARPS - 1) / DM_WARPS);
-  cfg.blockDim = dim3(DM_THREADS);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = overlap_prev ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, decode_mma4_kernel<D, GROUP>, tab, d, partials);
+  return launch_attention(decode_mma4_kernel<D, GROUP>, (tab.n_workers + DM_WARPS - 1) / DM_WARPS, DM_THREADS, smem, st,
+                          overlap_prev, tab, d, partials);
 }
 }  // namespace
 
@@ -512,9 +503,9 @@ cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* par
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
                               bool overlap_prev) {
   cudaError_t e = d.bits == 4   ? launch_decode_mma4(tab, d, partials, st, overlap_prev)
-                  : d.bits == 8 ? launch_decode_mma8(tab, d, partials, st)
-                  : d.bits == 16 ? launch_decode_mma16(tab, d, partials, st)
-                                : launch_decode_mma2(tab, d, partials, st);
+                  : d.bits == 8 ? launch_decode_mma8(tab, d, partials, st, overlap_prev)
+                  : d.bits == 16 ? launch_decode_mma16(tab, d, partials, st, overlap_prev)
+                                : launch_decode_mma2(tab, d, partials, st, overlap_prev);
   if (e != cudaSuccess) return e;
   const int items = d.Bt * d.Hq * tab.n_layers;
   cudaLaunchConfig_t cfg = {};

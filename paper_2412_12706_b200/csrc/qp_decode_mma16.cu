@@ -210,6 +210,9 @@ decode_mma16_kernel(const __grid_constant__ DecTable tab, const DecDims dm, floa
     cur += n_tiles;
     if (bh == BH - 1 && tile_begin + n_tiles == tph) ++li;
   }
+  // (see the 4-bit kernel: a call may start before the previous call's merge kernel has ended; the call after it
+  // relies on this grid not ending before that kernel has)
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
 template <int D>
@@ -221,23 +224,20 @@ constexpr size_t mma16_smem_bytes() {
 
 int decode_mma16_blocks_per_sm() { return D16_MINB; }
 
-cudaError_t launch_decode_mma16(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
-  const dim3 grid(tab.n_workers);
-  cudaError_t e;
+cudaError_t launch_decode_mma16(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
+                                bool overlap_prev) {
   if (d.D == 128) {
     constexpr size_t smem = mma16_smem_bytes<128>();
     static unsigned char done[64] = {};
-    e = allow_smem(decode_mma16_kernel<128>, smem, done);
+    const cudaError_t e = allow_smem(decode_mma16_kernel<128>, smem, done);
     if (e != cudaSuccess) return e;
-    decode_mma16_kernel<128><<<grid, D16_THREADS, smem, st>>>(tab, d, partials);
-  } else {
-    constexpr size_t smem = mma16_smem_bytes<64>();
-    static unsigned char done[64] = {};
-    e = allow_smem(decode_mma16_kernel<64>, smem, done);
-    if (e != cudaSuccess) return e;
-    decode_mma16_kernel<64><<<grid, D16_THREADS, smem, st>>>(tab, d, partials);
+    return launch_attention(decode_mma16_kernel<128>, tab.n_workers, D16_THREADS, smem, st, overlap_prev, tab, d, partials);
   }
-  return cudaGetLastError();
+  constexpr size_t smem = mma16_smem_bytes<64>();
+  static unsigned char done[64] = {};
+  const cudaError_t e = allow_smem(decode_mma16_kernel<64>, smem, done);
+  if (e != cudaSuccess) return e;
+  return launch_attention(decode_mma16_kernel<64>, tab.n_workers, D16_THREADS, smem, st, overlap_prev, tab, d, partials);
 }
 
 }  // namespace qp

@@ -313,6 +313,9 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
     cur += n_tiles;
     if (bh == BH - 1 && tile_begin + n_tiles == tph) ++li;
   }
+  // (see the 4-bit kernel: a call may start before the previous call's merge kernel has ended; the call after it
+  // relies on this grid not ending before that kernel has)
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
 template <int D>
@@ -328,24 +331,25 @@ int decode_mma8_blocks_per_sm() { return D8_MINB; }
 
 namespace {
 template <int D, int GROUP>
-cudaError_t launch_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+cudaError_t launch_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev) {
   constexpr size_t smem = mma8_smem_bytes<D>();
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(decode_mma8_kernel<D, GROUP>, smem, done);
   if (e != cudaSuccess) return e;
-  decode_mma8_kernel<D, GROUP><<<dim3(tab.n_workers), D8_THREADS, smem, st>>>(tab, d, partials);
-  return cudaGetLastError();
+  return launch_attention(decode_mma8_kernel<D, GROUP>, tab.n_workers, D8_THREADS, smem, st, overlap_prev, tab, d,
+                          partials);
 }
 }  // namespace
 
-cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st) {
+cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
+                               bool overlap_prev) {
   if (d.D == 128) {
-    if (d.group == 32) return launch_mma8<128, 32>(tab, d, partials, st);
-    if (d.group == 64) return launch_mma8<128, 64>(tab, d, partials, st);
-    return launch_mma8<128, 128>(tab, d, partials, st);
+    if (d.group == 32) return launch_mma8<128, 32>(tab, d, partials, st, overlap_prev);
+    if (d.group == 64) return launch_mma8<128, 64>(tab, d, partials, st, overlap_prev);
+    return launch_mma8<128, 128>(tab, d, partials, st, overlap_prev);
   }
-  if (d.group == 32) return launch_mma8<64, 32>(tab, d, partials, st);
-  return launch_mma8<64, 64>(tab, d, partials, st);
+  if (d.group == 32) return launch_mma8<64, 32>(tab, d, partials, st, overlap_prev);
+  return launch_mma8<64, 64>(tab, d, partials, st, overlap_prev);
 }
 
 }  // namespace qp

@@ -54,14 +54,32 @@ struct SkOwner {
 };
 
 
+// Launches an attention kernel; with overlap_prev as a programmatic dependent of the stream's previous kernel
+// (it may start while that one still runs; see launch_decode).
+template <typename K>
+cudaError_t launch_attention(K kernel, int blocks, int threads, size_t smem, cudaStream_t st, bool overlap_prev,
+                             const DecTable& tab, const DecDims& d, float* partials) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap_prev ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, tab, d, partials);
+}
+
 // launchers of the per-bit-width attention kernels
 cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
                                bool overlap_prev);
-cudaError_t launch_decode_mma2(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+cudaError_t launch_decode_mma2(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 bool decode_mma2_supported(const DecDims& d);
-cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 int decode_mma8_blocks_per_sm();
-cudaError_t launch_decode_mma16(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+cudaError_t launch_decode_mma16(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 int decode_mma16_blocks_per_sm();
 
 // opt in to more than 48 KB of dynamic shared memory, once per device and kernel
