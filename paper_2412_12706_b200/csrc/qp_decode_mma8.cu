@@ -48,21 +48,32 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   constexpr int NPAIR = D / 8;     // channel pairs owned by one lane on the key side
   extern __shared__ __align__(128) unsigned char smem[];
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);       // provably warp-uniform
   const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
-  const SkOwner sk{tab.total_tiles, tab.n_workers};
-  const int cta = blockIdx.x;
   asm volatile("griddepcontrol.launch_dependents;\n" ::);
-  long long cur = sk.start(cta);
-  const long long f_end = sk.start(cta + 1);
+  // every warp is a worker of its own (see the 4-bit kernel): contiguous tile range, private copy ring
+  const int wk = blockIdx.x * D8_WARPS + warp;
+  if (wk >= tab.n_workers) return;
+  const SkOwner sk{tab.total_tiles, tab.n_workers};
+  const long long f0 = sk.start(wk);
+  const int total = (int)(sk.start(wk + 1) - f0);
+  if (total <= 0) return;
 
-  unsigned char* wsm = smem + warp * (D8_STAGES * TL::BYTES + SP8_BYTES);
-  const uint32_t wsm_u = smem_u32(wsm);
+  const uint32_t wsm_u = smem_u32(smem + warp * (D8_STAGES * TL::BYTES + SP8_BYTES));
   const uint32_t sP = wsm_u + D8_STAGES * TL::BYTES;
-  float* s_acc = reinterpret_cast<float*>(smem);                // [warp][8][D], overlays the idle stages
-  float* s_m = s_acc + D8_WARPS * 8 * D;
-  float* s_l = s_m + D8_WARPS * 8;
 
+  // destinations of the asynchronous copies: key piece pi = lane + 32i is channel pi/2, token half pi&1; value
+  // piece pi is token pi/NQ, channels 16(pi%NQ) ..
+  uint32_t kdst[D / 16], vdst[D / 16];
+#pragma unroll
+  for (int i = 0; i < D / 16; ++i) {
+    const int pi = lane + 32 * i, c = pi >> 1, hf = pi & 1;
+    kdst[i] = TL::KC + hf * 16 * D + ((c ^ ((c / (D / 4)) << 1)) << 4);
+    const int tau = pi / NQ, q = pi % NQ;
+    const int sw = NQ == 8 ? (tau & 7) : ((tau >> 1) & 3);
+    vdst[i] = TL::VC + tau * D + ((q ^ sw) << 4);
+  }
   // sources of the transposing loads
   uint32_t k_plane, k_slot0, v_row, v_sw;
   {
@@ -79,54 +90,81 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const uint32_t ksz_dst = (lane < MCH ? TL::KS : TL::KZ) + mj * 16 + (mj / 8) * 16;
   const uint32_t vsz_dst = (lane < MCH ? TL::VS : TL::VZ) + mj * 16;
 
-  int li = 0;
-  while (li + 1 < tab.n_layers && tab.l[li + 1].tile_base <= cur) ++li;
+  // copy cursor (p_*) and compute cursor (c_*)
+  int p_li = 0;
+  while (p_li + 1 < tab.n_layers && (long long)tab.l[p_li + 1].tile_base <= f0) ++p_li;
+  int p_tph = tab.l[p_li].n >> 5;
+  int p_bh = (int)(f0 - tab.l[p_li].tile_base) / p_tph, p_tile = (int)(f0 - tab.l[p_li].tile_base) % p_tph;
+  int c_li = p_li, c_bh = p_bh, c_tile = p_tile, c_tph = p_tph;
 
-  while (cur < f_end) {
-    const DecLayer& ly = tab.l[li];
-    const int n = ly.n, tph = n >> 5;
-    const int rel = (int)(cur - ly.tile_base), bh = rel / tph, tile_begin = rel % tph;
-    const int n_tiles = (int)min((long long)(tph - tile_begin), f_end - cur);
-    const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
-
-    const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * tph * D * 32;
-    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * (n / GROUP) * D * 2;
-    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * (n / GROUP) * D * 2;
-    const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * D;
-    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * NG * 2;
-    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * NG * 2;
-    const unsigned char* gKm = lane < MCH ? gKs : gKz;
-    const unsigned char* gVm = lane < MCH ? gVs : gVz;
-
-    auto issue_tile = [&](int tile, int stage) {
-      const uint32_t sb = wsm_u + stage * TL::BYTES;
-      const int u = tile / GT, sub = tile % GT;                 // a key group is GROUP bytes per channel
-      const unsigned char* kc = gKc + (size_t)u * D * GROUP + sub * 32;
-      const unsigned char* vc = gVc + (size_t)tile * 32 * D + lane * 16;
+  const unsigned char *gKc, *gKm, *gVc, *gVm;                   // per-lane sources of the tile under the copy cursor
+  auto set_head = [&]() {
+    const DecLayer& ly = tab.l[p_li];
+    const size_t n = (size_t)ly.n, bh = (size_t)p_bh;
+    const int u = p_tile / GT, sub = p_tile % GT;
+    // (a key group of GROUP tokens is GROUP bytes per channel: a tile's 32 tokens are 32 of them, two pieces)
+    gKc = static_cast<const unsigned char*>(ly.kc) + bh * n * D + (size_t)u * D * GROUP + sub * 32 +
+          (lane >> 1) * GROUP + (lane & 1) * 16;
+    gVc = static_cast<const unsigned char*>(ly.vc) + bh * n * D + (size_t)p_tile * 32 * D + lane * 16;
+    gKm = reinterpret_cast<const unsigned char*>(lane < MCH ? ly.ks : ly.kz) + (bh * (n / GROUP) + u) * D * 2 + mj * 16;
+    gVm = reinterpret_cast<const unsigned char*>(lane < MCH ? ly.vs : ly.vz) + (bh * n + (size_t)p_tile * 32) * NG * 2 +
+          mj * 16;
+  };
+  set_head();
+  auto issue_tile = [&](uint32_t sb) {
 #pragma unroll
-      for (int i = 0; i < D / 16; ++i) {
-        const int pi = lane + 32 * i;                           // key piece: channel pi/2, token half pi&1
-        const int c = pi >> 1, hf = pi & 1;
-        cp_async16(sb + TL::KC + hf * 16 * D + ((c ^ ((c / (D / 4)) << 1)) << 4), kc + c * GROUP + hf * 16);
-        const int tau = pi / NQ, q = pi % NQ;                   // value piece: token tau, channels 16q .. 16q+15
-        const int sw = NQ == 8 ? (tau & 7) : ((tau >> 1) & 3);
-        cp_async16(sb + TL::VC + tau * D + ((q ^ sw) << 4), vc + i * 512);
-      }
-      if (lane < 2 * MCH) {
-        cp_async16(sb + ksz_dst, gKm + (size_t)u * D * 2 + mj * 16);
-        if (mj < 4 * NG) cp_async16(sb + vsz_dst, gVm + (size_t)tile * 64 * NG + mj * 16);
-      }
-    };
-
-    const int n_my = warp < n_tiles ? (n_tiles - warp + D8_WARPS - 1) / D8_WARPS : 0;
-#pragma unroll
-    for (int s = 0; s < D8_STAGES - 1; ++s) {
-      if (s < n_my) issue_tile(tile_begin + warp + D8_WARPS * s, s);
-      cp_async_commit();
+    for (int i = 0; i < D / 16; ++i) {
+      cp_async16(sb + kdst[i], gKc + i * 16 * GROUP);
+      cp_async16(sb + vdst[i], gVc + i * 512);
     }
+    if (2 * MCH == 32 || lane < 2 * MCH) {
+      cp_async16(sb + ksz_dst, gKm);
+      if (NG == 4 || mj < 4 * NG) cp_async16(sb + vsz_dst, gVm);
+    }
+    if (++p_tile == p_tph) {
+      p_tile = 0;
+      if (++p_bh == BH) {
+        p_bh = 0;
+        if (++p_li < tab.n_layers) p_tph = tab.l[p_li].n >> 5;
+      }
+      if (p_li < tab.n_layers) set_head();
+    } else {
+      gVc += 32 * D;
+      gVm += 64 * NG;
+      if (GT == 1 || p_tile % GT == 0) {
+        gKc += D * GROUP - (GT - 1) * 32;
+        gKm += D * 2;
+      } else {
+        gKc += 32;
+      }
+    }
+  };
+#pragma unroll
+  for (int s = 0; s < D8_STAGES - 1; ++s) {
+    if (s < total) issue_tile(wsm_u + s * TL::BYTES);
+    cp_async_commit();
+  }
+  uint32_t sb = wsm_u, sb_copy = wsm_u + (D8_STAGES - 1) * TL::BYTES;
 
-    uint32_t qh2[NPAIR];
-    {
+  uint32_t qh2[NPAIR];
+  float m_run[2], accO[NQ][4], accPZ[4];
+  auto clear_state = [&]() {
+    m_run[0] = m_run[1] = -INFINITY;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) accPZ[x] = 0.f;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q)
+#pragma unroll
+      for (int x = 0; x < 4; ++x) accO[q][x] = 0.f;
+  };
+  clear_state();
+  bool fresh = true;
+
+  for (int it = 0; it < total; ++it) {
+    if (fresh) {
+      fresh = false;
+      const DecLayer& ly = tab.l[c_li];
+      const int b = c_bh / dm.Hkv, hk = c_bh % dm.Hkv;
       const float scale_log2 = 1.4426950408889634f * rsqrtf((float)D);
       const uint16_t* qp = static_cast<const uint16_t*>(ly.q) + ((size_t)(b * dm.Hq + hk * G + g)) * D + (D / 4) * t;
 #pragma unroll
@@ -134,75 +172,78 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         uint4 w4 = make_uint4(0u, 0u, 0u, 0u);
         if (g < G) w4 = *reinterpret_cast<const uint4*>(qp + 2 * i);
         qh2[i + 0] = pack_half2(bf16lo(w4.x) * scale_log2, bf16hi(w4.x) * scale_log2);
-        qh2[i + 1] = pack_half2(bf16lo(w4.y) * scale_log2, bf16hi(w4.y) * scale_log2);
-        qh2[i + 2] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);
+        qh2[i + 2] = pack_half2(bf16lo(w4.y) * scale_log2, bf16hi(w4.y) * scale_log2);   // order (0, 2, 1, 3): see
+        qh2[i + 1] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);   // the zero-point MMAs
         qh2[i + 3] = pack_half2(bf16lo(w4.w) * scale_log2, bf16hi(w4.w) * scale_log2);
       }
     }
 
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    float accO[NQ][4], accPZ[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int q = 0; q < NQ; ++q)
-#pragma unroll
-      for (int x = 0; x < 4; ++x) accO[q][x] = 0.f;
-
-    for (int it = 0; it < n_my; ++it) {
+    {
       __syncwarp();
-      if (it + D8_STAGES - 1 < n_my)
-        issue_tile(tile_begin + warp + D8_WARPS * (it + D8_STAGES - 1), (it + D8_STAGES - 1) % D8_STAGES);
+      if (it + D8_STAGES - 1 < total) issue_tile(sb_copy);
       cp_async_commit();
       cp_async_wait<D8_STAGES - 1>();
       __syncwarp();
-      const uint32_t sb = wsm_u + (it % D8_STAGES) * TL::BYTES;
 
       // ---------------- keys: m-tile hf holds tokens 16hf + 2g (rows g) and 16hf + 2g + 1 (rows g+8)
-      float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, accZ[4] = {0.f, 0.f, 0.f, 0.f};
+      // zero-point term with swapped roles (A = query pairs as they sit in registers, B = zero-point pairs as
+      // loaded; rows g of the first, rows g+8 of the second MMA are read), as in the 4-bit kernel
+      float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      float accZa[4] = {0.f, 0.f, 0.f, 0.f}, accZb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c2 = 0; c2 < NQ / 2; ++c2) {                     // two k-steps (8 channels of this lane) per round
         const uint4 s4 = lds128(sb + TL::KS + ksz_off8((D / 4) * t + 8 * c2));
         const uint4 z4 = lds128(sb + TL::KZ + ksz_off8((D / 4) * t + 8 * c2));
-        const uint32_t sv[4] = {s4.x, s4.y, s4.z, s4.w}, zv[4] = {z4.x, z4.y, z4.z, z4.w};
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int c = 2 * c2 + cc;
-          const uint32_t b0 = hmul2_u32(qh2[2 * c], sv[2 * cc]), b1 = hmul2_u32(qh2[2 * c + 1], sv[2 * cc + 1]);
-          uint32_t R0, R1, R2, R3;
-          ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_plane + ((k_slot0 ^ (4 * c)) << 4));
-          mma_f16_m16n8k16(accK[0], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), b0, b1);
-          mma_f16_m16n8k16(accK[1], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), b0, b1);
-          mma_f16_m16n8k16(accZ, zv[2 * cc], zv[2 * cc], zv[2 * cc + 1], zv[2 * cc + 1], qh2[2 * c], qh2[2 * c + 1]);
-        }
+        // qh2[4 c2 + (0, 1, 2, 3)] hold the channel pairs (0, 2, 1, 3) of these eight channels
+        const uint32_t b00 = hmul2_u32(qh2[4 * c2 + 0], s4.x), b01 = hmul2_u32(qh2[4 * c2 + 2], s4.y);
+        const uint32_t b10 = hmul2_u32(qh2[4 * c2 + 1], s4.z), b11 = hmul2_u32(qh2[4 * c2 + 3], s4.w);
+        uint32_t R0, R1, R2, R3;
+        ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_plane + ((k_slot0 ^ (8 * c2)) << 4));
+        mma_f16_m16n8k16(accK[0], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), b00, b01);
+        mma_f16_m16n8k16(accK[1], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), b00, b01);
+        mma_f16_m16n8k16(accZa, qh2[4 * c2 + 0], qh2[4 * c2 + 1], qh2[4 * c2 + 2], qh2[4 * c2 + 3], z4.x, z4.y);
+        ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_plane + ((k_slot0 ^ (8 * c2 + 4)) << 4));
+        mma_f16_m16n8k16(accK[0], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), b10, b11);
+        mma_f16_m16n8k16(accK[1], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), b10, b11);
+        mma_f16_m16n8k16(accZb, qh2[4 * c2 + 0], qh2[4 * c2 + 1], qh2[4 * c2 + 2], qh2[4 * c2 + 3], z4.z, z4.w);
       }
-      // lg[j][x]: tokens {2g, 2g+1, 16+2g, 17+2g}[j], column 2t + x
+      const float zq = accZa[0] + accZb[2];                     // of head g; this lane needs columns 2t, 2t+1
+      const float zq_e[2] = {__shfl_sync(0xffffffffu, zq, 8 * t), __shfl_sync(0xffffffffu, zq, 8 * t + 4)};
+
+      // ---------------- running softmax (log2 domain), reference renewed lazily as in the 4-bit kernel
+      //   lg[j][x]: tokens {2g, 2g+1, 16+2g, 17+2g}[j], column 2t + x, minus the column's reference
+      constexpr float kSlack = 4.f;
       float lg[4][2];
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        lg[2 * hf][0] = fmaf(accK[hf][0], C24, accZ[0]);
-        lg[2 * hf][1] = fmaf(accK[hf][1], C24, accZ[1]);
-        lg[2 * hf + 1][0] = fmaf(accK[hf][2], C24, accZ[0]);
-        lg[2 * hf + 1][1] = fmaf(accK[hf][3], C24, accZ[1]);
-      }
-
-      float corr[2];
-#pragma unroll
       for (int x = 0; x < 2; ++x) {
-        float mx = fmaxf(fmaxf(lg[0][x], lg[1][x]), fmaxf(lg[2][x], lg[3][x]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-        const float mnew = fmaxf(m_run[x], mx);
-        corr[x] = ex2(m_run[x] - mnew);
-        m_run[x] = mnew;
-        float sum = 0.f;
+        const float zm = zq_e[x] - m_run[x];                    // +inf on the first tile of a head
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          lg[j][x] = ex2(lg[j][x] - mnew);
-          sum += lg[j][x];
+        for (int hf = 0; hf < 2; ++hf) {
+          lg[2 * hf][x] = fmaf(accK[hf][x], C24, zm);
+          lg[2 * hf + 1][x] = fmaf(accK[hf][2 + x], C24, zm);
         }
-        l_run[x] = fmaf(l_run[x], corr[x], sum);
       }
-      if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+      const float over = fmaxf(fmaxf(fmaxf(lg[0][0], lg[1][0]), fmaxf(lg[2][0], lg[3][0])),
+                               fmaxf(fmaxf(lg[0][1], lg[1][1]), fmaxf(lg[2][1], lg[3][1])));
+      if (__any_sync(0xffffffffu, over > kSlack)) {             // rare: renew the references, rescale
+        float corr[2];
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            lg[2 * hf][x] = fmaf(accK[hf][x], C24, zq_e[x]);
+            lg[2 * hf + 1][x] = fmaf(accK[hf][2 + x], C24, zq_e[x]);
+          }
+          float mx = fmaxf(fmaxf(lg[0][x], lg[1][x]), fmaxf(lg[2][x], lg[3][x]));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+          const float mnew = fmaxf(m_run[x], mx);
+          corr[x] = ex2(m_run[x] - mnew);
+          m_run[x] = mnew;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) lg[j][x] -= mnew;
+        }
 #pragma unroll
         for (int q = 0; q < NQ; ++q) {
           accO[q][0] *= corr[0]; accO[q][1] *= corr[1];
@@ -210,6 +251,10 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         }
         accPZ[0] *= corr[0]; accPZ[1] *= corr[1];
       }
+#pragma unroll
+      for (int x = 0; x < 2; ++x)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) lg[j][x] = ex2(lg[j][x]);    // p; its sum over the tokens: row NG of accPZ
 
       // ---------------- P through shared memory: [column][token] f16
 #pragma unroll
@@ -223,12 +268,12 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 #pragma unroll
       for (int pr = 0; pr < 4; ++pr) p2[pr] = lds32(sP + g * SP8_STRIDE + 4 * t + 16 * pr);
 
-      // ---------------- values
-      uint32_t ps[4][NG], zp[4];                                // ps[pair][scale group], zero-point rows: group g
+      // ---------------- values; zero-point MMA: row g < NG = zero points of scale group g, row NG = ones
+      uint32_t ps[4][NG], zp[4];                                // ps[pair][scale group]
 #pragma unroll
       for (int pr = 0; pr < 4; ++pr) {
         const int a = 8 * pr + 2 * t;
-        zp[pr] = 0u;
+        zp[pr] = g == NG ? 0x3c003c00u : 0u;
         if constexpr (NG == 4) {
           const uint4 x = lds128(sb + TL::VS + a * 8);
           ps[pr][0] = hmul2_u32(p2[pr], __byte_perm(x.x, x.z, 0x5410));
@@ -262,56 +307,38 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         mma_f16_m16n8k16(accO[q], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), ps[0][q * NG / NQ], ps[1][q * NG / NQ]);
         mma_f16_m16n8k16(accO[q], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), ps[2][q * NG / NQ], ps[3][q * NG / NQ]);
       }
+      sb_copy = sb;
+      sb = sb + TL::BYTES == sP ? wsm_u : sb + TL::BYTES;
     }
 
-    // ---------------- per-warp result -> shared memory -> one partial per (head, block) and query head
+    // ---------------- end of this head's part of the range: one partial record per query head, from registers
+    if (++c_tile == c_tph || it == total - 1) {
+      const float l0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * NG + t), l1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * NG + t);
+      const size_t slot = (size_t)c_li * BH + c_bh + wk;
+      float* r0 = partials + (slot * G + 2 * t) * (size_t)(D + 2);      // record of column 2t; column 2t+1 follows
+      float* r1 = r0 + (D + 2);
+      const bool h0 = 2 * t < G, h1 = 2 * t + 1 < G;
 #pragma unroll
-    for (int x = 0; x < 2; ++x) {
-      l_run[x] += __shfl_xor_sync(0xffffffffu, l_run[x], 4);
-      l_run[x] += __shfl_xor_sync(0xffffffffu, l_run[x], 8);
-      l_run[x] += __shfl_xor_sync(0xffffffffu, l_run[x], 16);
-    }
-    __syncthreads();
-#pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-      const int v = q * NG / NQ;                                // scale group of channels 16q ..
-      const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * v + t);
-      const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * v + t);
-      const int ch = 16 * q + 2 * g;
-      float* o0 = s_acc + ((warp * 8 + 2 * t) * D);
-      float* o1 = o0 + D;
-      *reinterpret_cast<float2*>(o0 + ch) = make_float2(fmaf(accO[q][0], C24, pz0), fmaf(accO[q][2], C24, pz0));
-      *reinterpret_cast<float2*>(o1 + ch) = make_float2(fmaf(accO[q][1], C24, pz1), fmaf(accO[q][3], C24, pz1));
-    }
-    if (g == 0) {
-      s_m[warp * 8 + 2 * t] = m_run[0]; s_m[warp * 8 + 2 * t + 1] = m_run[1];
-      s_l[warp * 8 + 2 * t] = l_run[0]; s_l[warp * 8 + 2 * t + 1] = l_run[1];
-    }
-    __syncthreads();
-    const size_t slot = (size_t)li * BH + bh + cta;
-    for (int idx = tid; idx < G * D; idx += D8_THREADS) {
-      const int h = idx / D, d = idx % D;
-      float M = -INFINITY;
-#pragma unroll
-      for (int wp = 0; wp < D8_WARPS; ++wp) M = fmaxf(M, s_m[wp * 8 + h]);
-      float Ls = 0.f, A = 0.f;
-#pragma unroll
-      for (int wp = 0; wp < D8_WARPS; ++wp) {
-        const float mw = s_m[wp * 8 + h];
-        if (mw != -INFINITY) {
-          const float f = ex2(mw - M);
-          Ls = fmaf(s_l[wp * 8 + h], f, Ls);
-          A = fmaf(s_acc[(wp * 8 + h) * D + d], f, A);
-        }
+      for (int q = 0; q < NQ; ++q) {
+        const int v = q * NG / NQ;                              // scale group of channels 16q ..
+        const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * v + t);
+        const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * v + t);
+        const int ch = 16 * q + 2 * g;
+        if (h0) *reinterpret_cast<float2*>(r0 + 2 + ch) = make_float2(fmaf(accO[q][0], C24, pz0), fmaf(accO[q][2], C24, pz0));
+        if (h1) *reinterpret_cast<float2*>(r1 + 2 + ch) = make_float2(fmaf(accO[q][1], C24, pz1), fmaf(accO[q][3], C24, pz1));
       }
-      float* op = partials + (slot * G + h) * (size_t)(D + 2);
-      if (d == 0) { op[0] = M; op[1] = Ls; }
-      op[2 + d] = A;
+      if (g == 0) {
+        if (h0) *reinterpret_cast<float2*>(r0) = make_float2(m_run[0], l0);
+        if (h1) *reinterpret_cast<float2*>(r1) = make_float2(m_run[1], l1);
+      }
+      clear_state();
+      c_tile = 0;
+      fresh = true;
+      if (++c_bh == BH) {
+        c_bh = 0;
+        if (++c_li < tab.n_layers) c_tph = tab.l[c_li].n >> 5;
+      }
     }
-    __syncthreads();
-
-    cur += n_tiles;
-    if (bh == BH - 1 && tile_begin + n_tiles == tph) ++li;
   }
   // (see the 4-bit kernel: a call may start before the previous call's merge kernel has ended; the call after it
   // relies on this grid not ending before that kernel has)
@@ -319,15 +346,12 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 }
 
 template <int D>
-constexpr size_t mma8_smem_bytes() {
-  constexpr size_t stages = (size_t)D8_WARPS * (D8_STAGES * Tile8<D>::BYTES + SP8_BYTES);
-  constexpr size_t combine = (size_t)D8_WARPS * 8 * D * 4 + 2 * D8_WARPS * 8 * 4;
-  return stages > combine ? stages : combine;
-}
+constexpr size_t mma8_smem_bytes() { return (size_t)D8_WARPS * (D8_STAGES * Tile8<D>::BYTES + SP8_BYTES); }
 
 }  // namespace
 
 int decode_mma8_blocks_per_sm() { return D8_MINB; }
+int decode_mma8_warps() { return D8_WARPS; }
 
 namespace {
 template <int D, int GROUP>
@@ -336,8 +360,8 @@ cudaError_t launch_mma8(const DecTable& tab, const DecDims& d, float* partials, 
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(decode_mma8_kernel<D, GROUP>, smem, done);
   if (e != cudaSuccess) return e;
-  return launch_attention(decode_mma8_kernel<D, GROUP>, tab.n_workers, D8_THREADS, smem, st, overlap_prev, tab, d,
-                          partials);
+  return launch_attention(decode_mma8_kernel<D, GROUP>, (tab.n_workers + D8_WARPS - 1) / D8_WARPS, D8_THREADS, smem, st,
+                          overlap_prev, tab, d, partials);
 }
 }  // namespace
 

@@ -79,6 +79,7 @@ cudaError_t launch_decode_mma2(const DecTable& tab, const DecDims& d, float* par
 bool decode_mma2_supported(const DecDims& d);
 cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 int decode_mma8_blocks_per_sm();
+int decode_mma8_warps();
 cudaError_t launch_decode_mma16(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 int decode_mma16_blocks_per_sm();
 
