@@ -468,10 +468,10 @@ bool decode_mma_supported(const DecDims& d) {
   return d.group == 32 && decode_mma2_supported(d);
 }
 
-// The 4-bit and 8-bit kernels' workers are warps; the other kernels' workers are blocks of four warps.
+// The quantized kernels' workers are warps; the 16-bit kernel's workers are blocks of four warps.
 int decode_mma_workers_per_sm(const DecDims& d) {
   return d.bits == 4 ? QP_DM_MINB * DM_WARPS : d.bits == 8 ? decode_mma8_blocks_per_sm() * decode_mma8_warps()
-         : d.bits == 16 ? decode_mma16_blocks_per_sm() : QP_DM_MINB;
+         : d.bits == 16 ? decode_mma16_blocks_per_sm() : decode_mma2_workers_per_sm();
 }
 // Small launches: four tiles per worker at least (a 4-bit worker is one warp, the others four warps with a tile
 // each); more, smaller records per head cost the merge kernel more than the attention kernel gains.

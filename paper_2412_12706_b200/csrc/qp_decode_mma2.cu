@@ -14,6 +14,9 @@
 // A 16-bit unit holds 8 codes; code j sits at bits 2j, and (word & (0x00030003 << 2j)) is an f16
 // pair worth c * 4^j * 2^-24 as long as the pattern stays below 2^11 (j <= 4); j = 5..7 use the
 // word shifted right by 10.  The powers of two are undone on the f32 accumulators.
+// Decomposition, softmax bookkeeping and the zero-point MMAs follow the 4-bit kernel: every warp is a worker of
+// its own over a contiguous range of 32-token tiles, which it walks in pairs (the last tile before a head
+// boundary or the end of the range may be single).
 #include "qp_mma.cuh"
 
 namespace qp {
@@ -83,22 +86,40 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   constexpr int NPAIR = D / 8;     // channel pairs owned by one lane on the key side
   extern __shared__ __align__(128) unsigned char smem[];
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);       // provably warp-uniform
   const int e = g >> 2, o = g & 3;                              // variant bit and unit index of this lane's MMA rows
   const bool lane_valid = e == (t >> 1);                        // this lane's accumulator entries are an e = e' block
   const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
-  const SkOwner sk{tab.total_tiles, tab.n_workers};
-  const int cta = blockIdx.x;
   asm volatile("griddepcontrol.launch_dependents;\n" ::);
-  long long cur = sk.start(cta);
-  const long long f_end = sk.start(cta + 1);
+  const int wk = blockIdx.x * D2_WARPS + warp;
+  if (wk >= tab.n_workers) return;
+  const SkOwner sk{tab.total_tiles, tab.n_workers};
+  const long long f0 = sk.start(wk);
+  const int total = (int)(sk.start(wk + 1) - f0);
+  if (total <= 0) return;
 
-  unsigned char* wsm = smem + warp * (D2_STAGES * TL::BYTES + SP2_BYTES);
-  const uint32_t wsm_u = smem_u32(wsm);
+  const uint32_t wsm_u = smem_u32(smem + warp * (D2_STAGES * TL::BYTES + SP2_BYTES));
   const uint32_t sP = wsm_u + D2_STAGES * TL::BYTES;
-  float* s_acc = reinterpret_cast<float*>(smem);                // [warp][4 heads][D], overlays the idle stages
-  float* s_m = s_acc + D2_WARPS * 4 * D;                        // [warp][4]
-  float* s_l = s_m + D2_WARPS * 4;
+
+  // destinations of the asynchronous copies (8-byte pieces of the codes: tile te of the pair goes to half te of
+  // a key row; a value piece (token, group vv) goes to half vv / NCH of row (token, vv % NCH))
+  uint32_t kdst[D / 32], vdst[2][D / 32];
+#pragma unroll
+  for (int i = 0; i < D / 32; ++i) {
+    const int c = lane + 32 * i;
+    kdst[i] = TL::KC + (c ^ ((c / (D / 4)) << 1)) * 16;
+#pragma unroll
+    for (int te = 0; te < 2; ++te) {
+      const int tau = 32 * te + c / NC, vv = c % NC;
+      const int rho = tau * NCH + vv % NCH;
+      vdst[te][i] = TL::VC + (NCH == 2 ? rho ^ ((tau >> 2) & 1) : rho) * 16 + (vv / NCH) * 8;
+    }
+  }
+  constexpr int MCH = D / 8;                                    // 16-byte pieces of a key scale or zero array
+  constexpr int VCH = D / 4;                                    // 16-byte pieces of the value scales of a pair
+  const int k_arr = lane / MCH, k_j = lane % MCH;               // lanes < 2 MCH: array (0 scale, 1 zero) and piece
+  const uint32_t kmeta_dst = TL::KS0 + k_arr * TL::KMETA + k_j * 16 + (k_j / 8) * 16;   // + 2 te KMETA
 
   // sources of the transposing loads
   uint32_t k_off, v_off[NCH];
@@ -114,82 +135,95 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
     }
   }
 
-  int li = 0;
-  while (li + 1 < tab.n_layers && tab.l[li + 1].tile_base <= cur) ++li;
+  // copy cursor (p_*) and compute cursor (c_*): both walk the range in the same pairs
+  int p_li = 0;
+  while (p_li + 1 < tab.n_layers && (long long)tab.l[p_li + 1].tile_base <= f0) ++p_li;
+  int p_tph = tab.l[p_li].n >> 5;
+  int p_bh = (int)(f0 - tab.l[p_li].tile_base) / p_tph, p_tile = (int)(f0 - tab.l[p_li].tile_base) % p_tph;
+  int c_li = p_li, c_bh = p_bh, c_tile = p_tile, c_tph = p_tph;
+  int p_left = total, c_left = total;
 
-  while (cur < f_end) {
-    const DecLayer& ly = tab.l[li];
-    const int n = ly.n, tph = n >> 5;
-    const int rel = (int)(cur - ly.tile_base), bh = rel / tph, tile_begin = rel % tph;
-    const int n_tiles = (int)min((long long)(tph - tile_begin), f_end - cur);
-    const int n_dt = (n_tiles + 1) >> 1;                        // double tiles of this segment
-    const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
-
-    const unsigned char* gKc = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * tph * D * 8;
-    const unsigned char* gKs = reinterpret_cast<const unsigned char*>(ly.ks) + (size_t)bh * tph * D * 2;
-    const unsigned char* gKz = reinterpret_cast<const unsigned char*>(ly.kz) + (size_t)bh * tph * D * 2;
-    const unsigned char* gVc = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * (D / 4);
-    const unsigned char* gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (size_t)bh * n * (D / 16);
-    const unsigned char* gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (size_t)bh * n * (D / 16);
-
-    // stage double tile `dt` (tiles tile_begin + 2dt and, if inside the segment, + 1); a missing second tile is zero
-    auto issue_dt = [&](int dt, int stage) {
-      const uint32_t sb = wsm_u + stage * TL::BYTES;
-      const int tile = tile_begin + 2 * dt;
-      const bool two = 2 * dt + 1 < n_tiles;
-      // key codes: per tile D pieces of 8 B (channel c), into half `te` of row slot(c)
+  const unsigned char *gKc, *gKm, *gVc, *gVs, *gVz;             // per-lane sources of the tile under the copy cursor
+  auto set_head = [&]() {
+    const DecLayer& ly = tab.l[p_li];
+    const size_t n = (size_t)ly.n, bh = (size_t)p_bh, tile = (size_t)p_tile;
+    gKc = static_cast<const unsigned char*>(ly.kc) + bh * n * (D / 4) + tile * D * 8 + lane * 8;
+    gVc = static_cast<const unsigned char*>(ly.vc) + bh * n * (D / 4) + tile * 8 * D + lane * 8;
+    gKm = reinterpret_cast<const unsigned char*>(k_arr ? ly.kz : ly.ks) + (bh * (n >> 5) + tile) * D * 2 + k_j * 16;
+    gVs = reinterpret_cast<const unsigned char*>(ly.vs) + (bh * n + tile * 32) * (D / 16) + lane * 16;
+    gVz = reinterpret_cast<const unsigned char*>(ly.vz) + (bh * n + tile * 32) * (D / 16) + lane * 16;
+  };
+  set_head();
+  // stage the pair of tiles under the copy cursor (a missing second tile is zero-filled), advance the cursor
+  auto issue_pair = [&](uint32_t sb) {
+    const bool two = p_tile + 1 < p_tph && p_left >= 2;
 #pragma unroll
-      for (int te = 0; te < 2; ++te) {
-        const unsigned char* src = gKc + (size_t)(tile + (two ? te : 0)) * D * 8 + lane * 8;
+    for (int te = 0; te < 2; ++te) {
+      const bool ok = te == 0 || two;
+      const unsigned char* kc = gKc + (ok ? te : 0) * (D * 8);
+      const unsigned char* vc = gVc + (ok ? te : 0) * (8 * D);
 #pragma unroll
-        for (int i = 0; i < D / 32; ++i) {
-          const int c = lane + 32 * i;
-          const int slot = c ^ ((c / (D / 4)) << 1);
-          cp_async8_zfill(sb + TL::KC + slot * 16 + te * 8, src + i * 256, te == 0 || two);
-        }
+      for (int i = 0; i < D / 32; ++i) {
+        cp_async8_zfill(sb + kdst[i] + te * 8, kc + i * 256, ok);
+        cp_async8_zfill(sb + vdst[te][i], vc + i * 256, ok);
       }
-      // value codes: per tile 32 tokens x NC pieces of 8 B (token tau, group vv)
-#pragma unroll
-      for (int te = 0; te < 2; ++te) {
-        const unsigned char* src = gVc + (size_t)(tile + (two ? te : 0)) * 8 * D + lane * 8;
-#pragma unroll
-        for (int i = 0; i < D / 32; ++i) {
-          const int idx = lane + 32 * i, tau = 32 * te + idx / NC, vv = idx % NC;
-          const int rho = tau * NCH + vv % NCH;
-          const int row = NCH == 2 ? rho ^ ((tau >> 2) & 1) : rho;
-          cp_async8_zfill(sb + TL::VC + row * 16 + (vv / NCH) * 8, src + i * 256, te == 0 || two);
-        }
-      }
-      // key scale / zero: per tile and array D/8 pieces of 16 B
-      constexpr int MCH = D / 8;
-#pragma unroll
-      for (int te = 0; te < 2; ++te) {
-        if (lane < 2 * MCH) {
-          const int arr = lane / MCH, j = lane % MCH;           // 0 = scale, 1 = zero
-          const unsigned char* src = (arr ? gKz : gKs) + (size_t)(tile + (two ? te : 0)) * D * 2 + j * 16;
-          cp_async16_zfill(sb + TL::KS0 + (2 * te + arr) * TL::KMETA + j * 16 + (j / 8) * 16, src, te == 0 || two);
-        }
-      }
-      // value scale / zero: the two tiles are contiguous, D/4 pieces of 16 B per array
-      constexpr int VCH = D / 4;
-      if (lane < VCH) {
-        const bool ok = lane < VCH / 2 || two;
-        const size_t off = (size_t)tile * 2 * D + (ok ? lane * 16 : 0);
-        cp_async16_zfill(sb + TL::VS + lane * 16, gVs + off, ok);
-        cp_async16_zfill(sb + TL::VZ + lane * 16, gVz + off, ok);
-      }
-    };
-
-    const int n_my = warp < n_dt ? (n_dt - warp + D2_WARPS - 1) / D2_WARPS : 0;
-#pragma unroll
-    for (int s = 0; s < D2_STAGES - 1; ++s) {
-      if (s < n_my) issue_dt(warp + D2_WARPS * s, s);
-      cp_async_commit();
+      if (2 * MCH == 32 || lane < 2 * MCH)
+        cp_async16_zfill(sb + kmeta_dst + 2 * te * TL::KMETA, gKm + (ok ? te : 0) * (D * 2), ok);
     }
+    if (VCH == 32 || lane < VCH) {                              // the two tiles' value scales are contiguous
+      const bool ok = lane < VCH / 2 || two;
+      const int back = ok ? 0 : (VCH / 2) * 16;                 // keep the address inside the array
+      cp_async16_zfill(sb + TL::VS + lane * 16, gVs - back, ok);
+      cp_async16_zfill(sb + TL::VZ + lane * 16, gVz - back, ok);
+    }
+    const int adv = two ? 2 : 1;
+    p_left -= adv;
+    p_tile += adv;
+    if (p_tile == p_tph) {
+      p_tile = 0;
+      if (++p_bh == BH) {
+        p_bh = 0;
+        if (++p_li < tab.n_layers) p_tph = tab.l[p_li].n >> 5;
+      }
+      if (p_li < tab.n_layers) set_head();
+    } else {
+      gKc += adv * (D * 8);
+      gVc += adv * (8 * D);
+      gKm += adv * (D * 2);
+      gVs += adv * (2 * D);
+      gVz += adv * (2 * D);
+    }
+  };
+#pragma unroll
+  for (int s = 0; s < D2_STAGES - 1; ++s) {
+    if (p_left > 0) issue_pair(wsm_u + s * TL::BYTES);
+    cp_async_commit();
+  }
+  uint32_t sb = wsm_u, sb_copy = wsm_u + (D2_STAGES - 1) * TL::BYTES;
 
-    // query fragments: column g of the MMAs = (variant g>>2, head g&3); both variants carry the same q'
-    uint32_t qh2[NPAIR];
-    {
+  uint32_t qh2[NPAIR];
+  // softmax reference of heads 2(t&1), 2(t&1)+1 (identical in all lanes with the same t&1) and accumulators
+  float m_run[2], accO[NCH][4][4], accPZ[4];
+  auto clear_state = [&]() {
+    m_run[0] = m_run[1] = -INFINITY;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) accPZ[x] = 0.f;
+#pragma unroll
+    for (int v = 0; v < NCH; ++v)
+#pragma unroll
+      for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+        for (int x = 0; x < 4; ++x) accO[v][mt][x] = 0.f;
+  };
+  clear_state();
+  bool fresh = true;
+
+  while (c_left > 0) {
+    if (fresh) {
+      fresh = false;
+      const DecLayer& ly = tab.l[c_li];
+      const int b = c_bh / dm.Hkv, hk = c_bh % dm.Hkv;
+      // query fragments: column g of the MMAs = (variant g>>2, head g&3); both variants carry the same q'
       const float scale_log2 = 1.4426950408889634f * rsqrtf((float)D);
       const uint16_t* qp = static_cast<const uint16_t*>(ly.q) + ((size_t)(b * dm.Hq + hk * G + o)) * D + (D / 4) * t;
 #pragma unroll
@@ -197,33 +231,24 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         uint4 w4 = make_uint4(0u, 0u, 0u, 0u);
         if (o < G) w4 = *reinterpret_cast<const uint4*>(qp + 2 * i);
         qh2[i + 0] = pack_half2(bf16lo(w4.x) * scale_log2, bf16hi(w4.x) * scale_log2);
-        qh2[i + 1] = pack_half2(bf16lo(w4.y) * scale_log2, bf16hi(w4.y) * scale_log2);
-        qh2[i + 2] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);
+        qh2[i + 2] = pack_half2(bf16lo(w4.y) * scale_log2, bf16hi(w4.y) * scale_log2);   // order (0, 2, 1, 3): see
+        qh2[i + 1] = pack_half2(bf16lo(w4.z) * scale_log2, bf16hi(w4.z) * scale_log2);   // the zero-point MMAs
         qh2[i + 3] = pack_half2(bf16lo(w4.w) * scale_log2, bf16hi(w4.w) * scale_log2);
       }
     }
-
-    // softmax state of heads 2(t&1), 2(t&1)+1 (identical in all lanes with the same t&1) and accumulators
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    float accO[NCH][4][4], accPZ[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int v = 0; v < NCH; ++v)
-#pragma unroll
-      for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-        for (int x = 0; x < 4; ++x) accO[v][mt][x] = 0.f;
-
-    for (int it = 0; it < n_my; ++it) {
+    const bool two = c_tile + 1 < c_tph && c_left >= 2;         // the same pairing as the copy cursor's
+    {
       __syncwarp();
-      if (it + D2_STAGES - 1 < n_my) issue_dt(warp + D2_WARPS * (it + D2_STAGES - 1), (it + D2_STAGES - 1) % D2_STAGES);
+      if (p_left > 0) issue_pair(sb_copy);
       cp_async_commit();
       cp_async_wait<D2_STAGES - 1>();
       __syncwarp();
-      const uint32_t sb = wsm_u + (it % D2_STAGES) * TL::BYTES;
-      const bool tile_present = e == 0 || 2 * (warp + D2_WARPS * it) + 1 < n_tiles;   // is this lane's tile real?
+      const bool tile_present = e == 0 || two;                  // is this lane's tile real?
 
       // ---------------- keys: rows (e, o) = tokens 8o..8o+7 of tile e; columns (e', h)
-      float accK[4][4], accZ[4] = {0.f, 0.f, 0.f, 0.f};
+      // zero-point term with swapped roles (A = query pairs as they sit in registers, B = zero-point pairs of the
+      // tile of this lane's column variant; rows g of the first, rows g+8 of the second MMA are read)
+      float accK[4][4], accZa[4] = {0.f, 0.f, 0.f, 0.f}, accZb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
@@ -235,45 +260,57 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         const uint4 z4 = lds128(kz_e + ksz_off2((D / 4) * t + 8 * c));
         uint32_t R0, R1, R2, R3;
         ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_off + c * 128);
-        mma_unit8(accK, R0, R1, hmul2_u32(qh2[4 * c + 0], s4.x), hmul2_u32(qh2[4 * c + 1], s4.y));
-        mma_f16_m16n8k16(accZ, z4.x, z4.x, z4.y, z4.y, qh2[4 * c + 0], qh2[4 * c + 1]);
-        mma_unit8(accK, R2, R3, hmul2_u32(qh2[4 * c + 2], s4.z), hmul2_u32(qh2[4 * c + 3], s4.w));
-        mma_f16_m16n8k16(accZ, z4.z, z4.z, z4.w, z4.w, qh2[4 * c + 2], qh2[4 * c + 3]);
+        // qh2[4c + (0, 1, 2, 3)] hold the channel pairs (0, 2, 1, 3) of this lane's eight channels
+        mma_unit8(accK, R0, R1, hmul2_u32(qh2[4 * c + 0], s4.x), hmul2_u32(qh2[4 * c + 2], s4.y));
+        mma_f16_m16n8k16(accZa, qh2[4 * c + 0], qh2[4 * c + 1], qh2[4 * c + 2], qh2[4 * c + 3], z4.x, z4.y);
+        mma_unit8(accK, R2, R3, hmul2_u32(qh2[4 * c + 1], s4.z), hmul2_u32(qh2[4 * c + 3], s4.w));
+        mma_f16_m16n8k16(accZb, qh2[4 * c + 0], qh2[4 * c + 1], qh2[4 * c + 2], qh2[4 * c + 3], z4.z, z4.w);
       }
-      // lg[2mt + rh][c]: token 8o + 2mt + rh of tile e, head 2(t&1) + c
-      float lg[8][2];
-      const bool use = lane_valid && tile_present;
-#pragma unroll
-      for (int mt = 0; mt < 4; ++mt) {
-        lg[2 * mt][0] = use ? fmaf(accK[mt][0], cfac(2 * mt), accZ[0]) : -INFINITY;
-        lg[2 * mt][1] = use ? fmaf(accK[mt][1], cfac(2 * mt), accZ[1]) : -INFINITY;
-        lg[2 * mt + 1][0] = use ? fmaf(accK[mt][2], cfac(2 * mt + 1), accZ[0]) : -INFINITY;
-        lg[2 * mt + 1][1] = use ? fmaf(accK[mt][3], cfac(2 * mt + 1), accZ[1]) : -INFINITY;
-      }
+      // lanes (g, t) hold the term of head g&3 and the tile of column variant t>>1; this lane needs heads
+      // 2(t&1), 2(t&1)+1 of variant t>>1
+      const float zq = accZa[0] + accZb[2];
+      const float zq_c[2] = {__shfl_sync(0xffffffffu, zq, 8 * (t & 1) + t),
+                             __shfl_sync(0xffffffffu, zq, 8 * (t & 1) + 4 + t)};
 
-      // ---------------- running softmax over the 64 tokens (log2 domain)
-      float corr[2];
+      // ---------------- running softmax over the 64 tokens (log2 domain), reference renewed lazily
+      //   lg[2mt + rh][c]: token 8o + 2mt + rh of tile e, head 2(t&1) + c, minus the head's reference
+      constexpr float kSlack = 4.f;
+      const bool use = lane_valid && tile_present;
+      float lg[8][2];
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        float mx = lg[0][c];
+        const float zm = zq_c[c] - m_run[c];                    // +inf on the first pair of a head
 #pragma unroll
-        for (int j = 1; j < 8; ++j) mx = fmaxf(mx, lg[j][c]);
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));    // lanes with the same t&1 share the two heads
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-        const float mnew = fmaxf(m_run[c], mx);
-        corr[c] = ex2(m_run[c] - mnew);
-        m_run[c] = mnew;
-        float sum = 0.f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          lg[j][c] = ex2(lg[j][c] - mnew);                      // 0 for entries that are not logits
-          sum += lg[j][c];
+        for (int mt = 0; mt < 4; ++mt) {
+          lg[2 * mt][c] = use ? fmaf(accK[mt][c], cfac(2 * mt), zm) : -INFINITY;
+          lg[2 * mt + 1][c] = use ? fmaf(accK[mt][2 + c], cfac(2 * mt + 1), zm) : -INFINITY;
         }
-        l_run[c] = fmaf(l_run[c], corr[c], sum);
       }
-      if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+      float over = fmaxf(lg[0][0], lg[0][1]);
+#pragma unroll
+      for (int j = 1; j < 8; ++j) over = fmaxf(over, fmaxf(lg[j][0], lg[j][1]));
+      if (__any_sync(0xffffffffu, over > kSlack)) {             // rare: renew the references, rescale
+        float corr[2];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+#pragma unroll
+          for (int mt = 0; mt < 4; ++mt) {
+            lg[2 * mt][c] = use ? fmaf(accK[mt][c], cfac(2 * mt), zq_c[c]) : -INFINITY;
+            lg[2 * mt + 1][c] = use ? fmaf(accK[mt][2 + c], cfac(2 * mt + 1), zq_c[c]) : -INFINITY;
+          }
+          float mx = lg[0][c];
+#pragma unroll
+          for (int j = 1; j < 8; ++j) mx = fmaxf(mx, lg[j][c]);
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));    // lanes with the same t&1 share the two heads
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+          const float mnew = fmaxf(m_run[c], mx);
+          corr[c] = ex2(m_run[c] - mnew);
+          m_run[c] = mnew;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) lg[j][c] -= mnew;
+        }
 #pragma unroll
         for (int v = 0; v < NCH; ++v)
 #pragma unroll
@@ -283,6 +320,10 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
           }
         accPZ[0] *= corr[0]; accPZ[1] *= corr[1];
       }
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) lg[j][c] = ex2(lg[j][c]);    // p (0 for entries that are not logits)
 
       // ---------------- P through shared memory: [head][64 tokens] f16
       if (lane_valid) {
@@ -295,6 +336,7 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       __syncwarp();
 
       // ---------------- values: rows (e, o) = channels 8o..8o+7 of group v + e*NCH; columns (e', h)
+      // zero-point MMA: row g < NC = zero points of value group g, row NC = ones (softmax denominators)
 #pragma unroll
       for (int kp = 0; kp < 2; ++kp) {                          // 32 tokens = two k-steps per transposed load
         uint32_t p2[2][2], ps[2][2][NCH], zp[2][2];             // [k-step][token-pair half]
@@ -314,8 +356,8 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
               const uint2 x = lds64(sb + TL::VS + a * 4);
               ps[kk][hf][0] = hmul2_u32(p2[kk][hf], __byte_perm(x.x, x.y, e ? 0x7632 : 0x5410));
             }
-            zp[kk][hf] = 0u;
-            if (g < NC) {                                       // zero-point MMA: row g = value group g
+            zp[kk][hf] = g == NC ? 0x3c003c00u : 0u;
+            if (g < NC) {
               if constexpr (NC == 4) {
                 const uint32_t ya = lds32(sb + TL::VZ + a * 8 + (g & 2) * 2);
                 const uint32_t yb = lds32(sb + TL::VZ + a * 8 + 8 + (g & 2) * 2);
@@ -336,65 +378,52 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
           mma_unit8(accO[v], R2, R3, ps[1][0][v], ps[1][1][v]);
         }
       }
+      sb_copy = sb;
+      sb = sb + TL::BYTES == sP ? wsm_u : sb + TL::BYTES;
     }
 
-    // ---------------- per-warp result -> shared memory -> one partial per (head, block) and query head
+    // ---------------- end of this head's part of the range: one partial record per query head, from registers
+    const int adv = two ? 2 : 1;
+    c_left -= adv;
+    c_tile += adv;
+    if (c_tile == c_tph || c_left == 0) {
+      // softmax denominators of heads 2(t&1), +1: row NC of the zero-point accumulator, columns (0, h)
+      const float l0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * NC + (t & 1));
+      const float l1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * NC + (t & 1));
+      const size_t slot = (size_t)c_li * BH + c_bh + wk;
+      const int h0i = 2 * (t & 1);
+      float* r0 = partials + (slot * G + h0i) * (size_t)(D + 2);
+      float* r1 = r0 + (D + 2);
+      const bool h0 = lane_valid && h0i < G, h1 = lane_valid && h0i + 1 < G;
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 2);
-      l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 4);
-      l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 8);
-      l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 16);
-    }
-    __syncthreads();                                            // every warp has consumed its last stage
-#pragma unroll
-    for (int v = 0; v < NCH; ++v) {
-      // zero-point term of group vv = v + e*NCH for heads 2(t&1), +1: row vv of accPZ, columns (0, h)
-      const int vv = v + e * NCH;
-      const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * vv + (t & 1));
-      const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * vv + (t & 1));
-      if (lane_valid) {
-        float* o0 = s_acc + ((warp * 4 + 2 * (t & 1)) * D);
-        float* o1 = o0 + D;
+      for (int v = 0; v < NCH; ++v) {
+        // zero-point term of group vv = v + e*NCH for heads 2(t&1), +1: row vv of accPZ, columns (0, h)
+        const int vv = v + e * NCH;
+        const float pz0 = __shfl_sync(0xffffffffu, accPZ[0], 4 * vv + (t & 1));
+        const float pz1 = __shfl_sync(0xffffffffu, accPZ[1], 4 * vv + (t & 1));
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt) {
           const int ch = 32 * vv + 8 * o + 2 * mt;
-          *reinterpret_cast<float2*>(o0 + ch) =
-              make_float2(fmaf(accO[v][mt][0], cfac(2 * mt), pz0), fmaf(accO[v][mt][2], cfac(2 * mt + 1), pz0));
-          *reinterpret_cast<float2*>(o1 + ch) =
-              make_float2(fmaf(accO[v][mt][1], cfac(2 * mt), pz1), fmaf(accO[v][mt][3], cfac(2 * mt + 1), pz1));
+          if (h0) *reinterpret_cast<float2*>(r0 + 2 + ch) =
+                      make_float2(fmaf(accO[v][mt][0], cfac(2 * mt), pz0), fmaf(accO[v][mt][2], cfac(2 * mt + 1), pz0));
+          if (h1) *reinterpret_cast<float2*>(r1 + 2 + ch) =
+                      make_float2(fmaf(accO[v][mt][1], cfac(2 * mt), pz1), fmaf(accO[v][mt][3], cfac(2 * mt + 1), pz1));
+        }
+      }
+      if (g == 0 && t < 2) {                                    // lanes (0, 0) and (0, 1): e = 0 = t>>1
+        if (h0) *reinterpret_cast<float2*>(r0) = make_float2(m_run[0], l0);
+        if (h1) *reinterpret_cast<float2*>(r1) = make_float2(m_run[1], l1);
+      }
+      clear_state();
+      fresh = true;
+      if (c_tile == c_tph) {
+        c_tile = 0;
+        if (++c_bh == BH) {
+          c_bh = 0;
+          if (++c_li < tab.n_layers) c_tph = tab.l[c_li].n >> 5;
         }
       }
     }
-    if (g == 0 && t < 2) {
-      s_m[warp * 4 + 2 * t] = m_run[0]; s_m[warp * 4 + 2 * t + 1] = m_run[1];
-      s_l[warp * 4 + 2 * t] = l_run[0]; s_l[warp * 4 + 2 * t + 1] = l_run[1];
-    }
-    __syncthreads();
-    const size_t slot = (size_t)li * BH + bh + cta;
-    for (int idx = tid; idx < G * D; idx += D2_THREADS) {
-      const int h = idx / D, d = idx % D;
-      float M = -INFINITY;
-#pragma unroll
-      for (int wp = 0; wp < D2_WARPS; ++wp) M = fmaxf(M, s_m[wp * 4 + h]);
-      float Ls = 0.f, A = 0.f;
-#pragma unroll
-      for (int wp = 0; wp < D2_WARPS; ++wp) {
-        const float mw = s_m[wp * 4 + h];
-        if (mw != -INFINITY) {
-          const float f = ex2(mw - M);
-          Ls = fmaf(s_l[wp * 4 + h], f, Ls);
-          A = fmaf(s_acc[(wp * 4 + h) * D + d], f, A);
-        }
-      }
-      float* op = partials + (slot * G + h) * (size_t)(D + 2);
-      if (d == 0) { op[0] = M; op[1] = Ls; }
-      op[2 + d] = A;
-    }
-    __syncthreads();
-
-    cur += n_tiles;
-    if (bh == BH - 1 && tile_begin + n_tiles == tph) ++li;
   }
   // (see the 4-bit kernel: a call may start before the previous call's merge kernel has ended; the call after it
   // relies on this grid not ending before that kernel has)
@@ -402,32 +431,30 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 }
 
 template <int D>
-constexpr size_t mma2_smem_bytes() {
-  constexpr size_t stages = (size_t)D2_WARPS * (D2_STAGES * Tile2<D>::BYTES + SP2_BYTES);
-  constexpr size_t combine = (size_t)D2_WARPS * 4 * D * 4 + 2 * D2_WARPS * 4 * 4;
-  return stages > combine ? stages : combine;
-}
+constexpr size_t mma2_smem_bytes() { return (size_t)D2_WARPS * (D2_STAGES * Tile2<D>::BYTES + SP2_BYTES); }
 
 }  // namespace
 
 bool decode_mma2_supported(const DecDims& d) {
   return d.bits == 2 && d.group == 32 && (d.D == 128 || d.D == 64) && d.Hq / d.Hkv <= 4;
 }
+int decode_mma2_workers_per_sm() { return QP_D2_MINB * D2_WARPS; }
 
 cudaError_t launch_decode_mma2(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
                                bool overlap_prev) {
+  const int blocks = (tab.n_workers + D2_WARPS - 1) / D2_WARPS;
   if (d.D == 128) {
     constexpr size_t smem = mma2_smem_bytes<128>();
     static unsigned char done[64] = {};
     const cudaError_t e = allow_smem(decode_mma2_kernel<128>, smem, done);
     if (e != cudaSuccess) return e;
-    return launch_attention(decode_mma2_kernel<128>, tab.n_workers, D2_THREADS, smem, st, overlap_prev, tab, d, partials);
+    return launch_attention(decode_mma2_kernel<128>, blocks, D2_THREADS, smem, st, overlap_prev, tab, d, partials);
   }
   constexpr size_t smem = mma2_smem_bytes<64>();
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(decode_mma2_kernel<64>, smem, done);
   if (e != cudaSuccess) return e;
-  return launch_attention(decode_mma2_kernel<64>, tab.n_workers, D2_THREADS, smem, st, overlap_prev, tab, d, partials);
+  return launch_attention(decode_mma2_kernel<64>, blocks, D2_THREADS, smem, st, overlap_prev, tab, d, partials);
 }
 
 }  // namespace qp

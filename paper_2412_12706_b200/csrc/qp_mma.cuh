@@ -77,6 +77,7 @@ cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* par
                                bool overlap_prev);
 cudaError_t launch_decode_mma2(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 bool decode_mma2_supported(const DecDims& d);
+int decode_mma2_workers_per_sm();
 cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
 int decode_mma8_blocks_per_sm();
 int decode_mma8_warps();
