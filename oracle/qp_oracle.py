@@ -180,3 +180,69 @@ def compress_layer(k, v, q_win, budget_bits: int, bits: int, group: int = 32, po
     pooled = scores(q_win, k, pool)
     kept = select(pooled, L, w, n)
     return quantize(k, v, kept, bits, group), kept, pooled
+
+
+# ------------------------------------------------------------------ decode-time appends (Eq. 2)
+
+@dataclass
+class GenState:
+    """Cache of one layer during generation: the packed part plus a 16-bit tail.
+
+    Eq. 2 appends the new token's key and value to the cache.  The paper does not say how a
+    quantized cache takes in single tokens, and key groups span g tokens, so the reading here is:
+    appended tokens wait, unquantized (bf16), in a tail of fewer than g tokens per KV head;
+    attention runs over the packed tokens followed by the tail; as soon as the tail holds g tokens
+    they are quantized by Eq. 4 exactly like g kept tokens of the prompt (one key group per channel,
+    g value rows) and become the last g tokens of the packed part.  At 16 bit nothing waits: the
+    row goes straight into the cache.  Nothing is pruned after the prompt.
+    """
+    packed: Packed
+    tail_k: np.ndarray   # u16(bf16) [Bt,Hkv,n_tail,D], 0 <= n_tail < g
+    tail_v: np.ndarray
+
+    @property
+    def n_tail(self) -> int:
+        return self.tail_k.shape[2]
+
+
+def gen_state(pk: Packed, D: int) -> GenState:
+    Bt, Hkv = pk.k_codes.shape[:2]
+    e = np.empty((Bt, Hkv, 0, D), np.uint16)
+    return GenState(pk, e, e.copy())
+
+
+def _concat_packed(a: Packed, b: Packed) -> Packed:
+    """The tokens of b after the tokens of a (every array of the layout has its token or
+    token-group axis third)."""
+    cat = lambda x, y: None if x is None else np.concatenate([x, y], axis=2)
+    return Packed(a.bits, a.group, a.n + b.n, cat(a.k_codes, b.k_codes), cat(a.v_codes, b.v_codes),
+                  cat(a.k_scale, b.k_scale), cat(a.k_zero, b.k_zero),
+                  cat(a.v_scale, b.v_scale), cat(a.v_zero, b.v_zero))
+
+
+def append(st: GenState, k_new: np.ndarray, v_new: np.ndarray) -> GenState:
+    """k_new, v_new u16(bf16) [Bt,Hkv,D]: the new token's key and value rows (Eq. 2)."""
+    k_new, v_new = _c(k_new, np.uint16), _c(v_new, np.uint16)
+    tk = np.concatenate([st.tail_k, k_new[:, :, None, :]], axis=2)
+    tv = np.concatenate([st.tail_v, v_new[:, :, None, :]], axis=2)
+    pk = st.packed
+    full = 1 if pk.bits == 16 else pk.group
+    if tk.shape[2] < full:
+        return GenState(pk, tk, tv)
+    Bt, Hkv, _, D = tk.shape
+    ident = np.broadcast_to(np.arange(full, dtype=np.int32), (Bt, Hkv, full)).copy()
+    flushed = quantize(tk, tv, ident, pk.bits, pk.group)
+    return GenState(_concat_packed(pk, flushed), tk[:, :, :0].copy(), tv[:, :, :0].copy())
+
+
+def _bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def decode_state(q: np.ndarray, st: GenState, D: int) -> np.ndarray:
+    """Eq. 3 over the dequantized packed tokens (Eq. 5) followed by the tail's exact values."""
+    kd, vd = dequantize(st.packed, D)
+    if st.n_tail:
+        kd = np.concatenate([kd, _bf16_to_f64(st.tail_k)], axis=2)
+        vd = np.concatenate([vd, _bf16_to_f64(st.tail_v)], axis=2)
+    return decode(q, kd, vd)
