@@ -39,7 +39,7 @@ typedef enum {
   QP_OK = 0,
   QP_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, Hq % Hkv != 0, w >= L, even pool ... */
   QP_ERR_UNSUPPORTED = 2, /* bits not in {2,4,8,16}, group not in {32,64,128}, D not in {64,128}, G > 8, w > 64 */
-  QP_ERR_BUDGET = 3,      /* budget gives n <= w, or n is not a whole number of groups */
+  QP_ERR_BUDGET = 3,      /* budget gives n <= w, n is not a whole number of groups, or no room to append */
   QP_ERR_WORKSPACE = 4,   /* workspace too small */
   QP_ERR_ALIGNMENT = 5,   /* a base pointer is not 16-byte aligned */
   QP_ERR_CUDA = 6         /* a launch failed */
@@ -64,9 +64,14 @@ typedef enum {
  * B = 16: k_codes / v_codes hold the gathered bf16 rows [Bt, Hkv, n, D] and the four
  * scale/zero pointers are unused (sizes 0).
  * Kept tokens are stored in ascending order of their position in the prompt.
+ *
+ * Room for tokens appended during decoding (Eq. 2): n_cap > n_keep sizes every array for n_cap
+ * tokens per KV head (read n_cap for n in the shapes above: the stride from one (batch, KV head)
+ * to the next is that of n_cap tokens), of which the first n_keep are in use.  n_cap = 0 means
+ * n_cap = n_keep (no room).  For B < 16 n_cap is a multiple of g.
  */
 typedef struct qp_cache {
-  int32_t batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep, reserved_;
+  int32_t batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep, n_cap;
   size_t k_codes_bytes, v_codes_bytes;
   size_t k_meta_bytes; /* bytes of k_scale; k_zero has the same size */
   size_t v_meta_bytes; /* bytes of v_scale; v_zero has the same size */
@@ -91,6 +96,10 @@ qp_status qp_n_keep(int64_t budget_bits, int bits, int group, int L, int w, int3
  */
 qp_status qp_cache_layout(int batch, int n_q_heads, int n_kv_heads, int head_dim, int bits, int group,
                           int n_keep, qp_cache* out /* host, out */);
+
+/* The same with room for n_cap >= n_keep tokens per KV head (see qp_cache). */
+qp_status qp_cache_layout_cap(int batch, int n_q_heads, int n_kv_heads, int head_dim, int bits, int group,
+                              int n_keep, int n_cap, qp_cache* out /* host, out */);
 
 /* Bytes of device scratch that qp_compress_layer / qp_window_scores need (0 on invalid shapes). */
 size_t qp_compress_workspace_bytes(int batch, int n_q_heads, int n_kv_heads, int head_dim, int L, int w);
@@ -170,6 +179,52 @@ qp_status qp_decode_attn(const void* q, const qp_cache* cache /* host */, void* 
  */
 qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches,
                                 void* const* out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Tokens appended during decoding that have not been quantized yet (host descriptor, caller-
+ * allocated device buffers).  Eq. 2 appends the new token's key and value to the cache; the paper
+ * does not say how a quantized cache takes single tokens in, and a key group spans g tokens, so:
+ * appended tokens wait in bf16 in this tail (fewer than g per KV head), attention runs over the
+ * packed tokens followed by the tail, and when the tail holds g tokens they are quantized by
+ * Eq. 4 exactly like g kept tokens of the prompt and become tokens n_keep .. n_keep+g-1 of the
+ * packed cache.  B = 16 needs no tail (rows go straight into the cache); the pointers may be NULL.
+ */
+typedef struct qp_tail {
+  int32_t n_tail;         /* tokens in the tail, 0 <= n_tail < group; maintained by qp_append_kv */
+  int32_t reserved_;
+  void *k_tail, *v_tail;  /* device bf16 [Bt, Hkv, group, D] each, 16-byte aligned */
+} qp_tail;
+
+/*
+ * Eq. 2 for one decode step: appends the key/value rows of the new token, k_new, v_new bf16
+ * [Bt,Hkv,D] (device), to each of n_layers caches (1 <= n_layers <= QP_MAX_LAYERS; k_new, v_new
+ * HOST arrays of device pointers; caches, tails HOST arrays, updated in place).
+ * B < 16: the rows are written to tail slot n_tail; if that fills the tail, its g tokens are
+ * quantized into key group n_keep/g and value rows n_keep.. of the cache (same arithmetic as
+ * qp_gather_quantize), n_keep grows by g and n_tail returns to 0.  B = 16: the rows are written
+ * to token n_keep of the cache and n_keep grows by 1.  One or two launches for all layers; the
+ * layers need not agree in n_keep or n_tail but must agree in shape, bits and group.
+ * QP_ERR_BUDGET, before anything is launched or changed, when a cache has no room left
+ * (n_keep + g > n_cap for a flush, n_keep + 1 > n_cap at 16 bit).
+ */
+qp_status qp_append_kv_layers(int n_layers, const void* const* k_new, const void* const* v_new,
+                              qp_cache* caches /* host, in/out */, qp_tail* tails /* host, in/out */,
+                              void* stream);
+/* The same for one layer. */
+qp_status qp_append_kv(const void* k_new, const void* v_new, qp_cache* cache /* host, in/out */,
+                       qp_tail* tail /* host, in/out */, void* stream);
+
+/*
+ * Decode attention (Eq. 3) over the packed tokens followed by the tail's tokens: the softmax runs
+ * over n_keep + n_tail tokens.  Arguments as for qp_decode_attn_layers / qp_decode_attn plus the
+ * tails (HOST array; tails[l].n_tail may be 0, tails may be NULL for "no tail anywhere").
+ * The tail is read in full precision by the merge step.
+ */
+qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const qp_cache* caches,
+                                     const qp_tail* tails, void* const* out, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+qp_status qp_decode_attn_tail(const void* q, const qp_cache* cache /* host */, const qp_tail* tail /* host */,
+                              void* out, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Decode attention without any caller-supplied scratch.  (The paper has no counterpart to this

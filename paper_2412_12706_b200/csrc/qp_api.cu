@@ -35,10 +35,11 @@ class PrevOutputs {
     auto it = prev_.find(key);
     Decision dec{!forgot_, 0};                      // a stream seen for the first time has no earlier decode kernel
     if (it != prev_.end()) {
-      dec.overlap = true;
+      dec.overlap = !it->second.barrier;
       dec.parity = it->second.parity ^ 1;
       const std::vector<Range>& w = it->second.outs;
       for (const Range& r : reads) {
+        if (!dec.overlap) break;
         const auto lo = std::lower_bound(w.begin(), w.end(), r.second,
                                          [](const Range& x, uintptr_t end) { return x.first < end; });
         if (lo != w.begin() && (lo - 1)->second > r.first) { dec.overlap = false; break; }
@@ -51,13 +52,26 @@ class PrevOutputs {
     Entry& e = prev_[key];
     e.outs.swap(writes);
     e.parity = dec.parity;
+    e.barrier = false;
     return dec;
+  }
+  // Another kernel of the library has been enqueued on this stream that writes arrays a decode call reads
+  // before it waits (a cache being filled or extended): the next decode call on the stream must be launched
+  // in plain stream order.
+  void barrier(int device, cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(mu_);
+    if (prev_.size() >= kMaxStreams && prev_.find(std::make_pair(device, st)) == prev_.end()) {
+      prev_.clear();
+      forgot_ = true;
+    }
+    prev_[std::make_pair(device, st)].barrier = true;
   }
 
  private:
   struct Entry {
     std::vector<Range> outs;
     int parity = 0;
+    bool barrier = false;
   };
   static constexpr size_t kMaxStreams = 256;
   std::mutex mu_;
@@ -69,6 +83,11 @@ PrevOutputs g_prev_outputs;
 inline PrevOutputs::Range range_of(const void* p, size_t bytes) {
   const uintptr_t b = reinterpret_cast<uintptr_t>(p);
   return {b, b + bytes};
+}
+
+void cache_written(cudaStream_t st) {
+  int device = 0;
+  if (cudaGetDevice(&device) == cudaSuccess) g_prev_outputs.barrier(device, st);
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -86,8 +105,9 @@ qp_status check_cache(const qp_cache* c, bool need_ptrs) {
   qp_status s = check_shape(c->batch, c->n_q_heads, c->n_kv_heads, c->head_dim);
   if (s != QP_OK) return s;
   if (!pow2_bits(c->bits) || !ok_group(c->group) || c->head_dim % c->group != 0) return QP_ERR_UNSUPPORTED;
-  if (c->n_keep < 1) return QP_ERR_INVALID_ARG;
+  if (c->n_keep < 1 || c->n_cap < 0) return QP_ERR_INVALID_ARG;
   if (c->bits < 16 && c->n_keep % c->group != 0) return QP_ERR_BUDGET;
+  if (c->n_cap != 0 && (c->n_cap < c->n_keep || (c->bits < 16 && c->n_cap % c->group != 0))) return QP_ERR_BUDGET;
   if (need_ptrs) {
     if (!c->k_codes || !c->v_codes) return QP_ERR_INVALID_ARG;
     if (!aligned16(c->k_codes) || !aligned16(c->v_codes)) return QP_ERR_ALIGNMENT;
@@ -130,14 +150,19 @@ qp_status qp_n_keep(int64_t budget_bits, int bits, int group, int L, int w, int3
 
 qp_status qp_cache_layout(int batch, int n_q_heads, int n_kv_heads, int head_dim, int bits, int group, int n_keep,
                           qp_cache* out) {
+  return qp_cache_layout_cap(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep, 0, out);
+}
+
+qp_status qp_cache_layout_cap(int batch, int n_q_heads, int n_kv_heads, int head_dim, int bits, int group, int n_keep,
+                              int n_cap, qp_cache* out) {
   if (!out) return QP_ERR_INVALID_ARG;
   qp_cache c;
   std::memset(&c, 0, sizeof(c));
   c.batch = batch; c.n_q_heads = n_q_heads; c.n_kv_heads = n_kv_heads; c.head_dim = head_dim;
-  c.bits = bits; c.group = group; c.n_keep = n_keep;
+  c.bits = bits; c.group = group; c.n_keep = n_keep; c.n_cap = n_cap;
   const qp_status s = check_cache(&c, false);
   if (s != QP_OK) return s;
-  const size_t elems = (size_t)batch * n_kv_heads * n_keep * head_dim;
+  const size_t elems = (size_t)batch * n_kv_heads * cache_capacity(c) * head_dim;
   if (bits == 16) {
     c.k_codes_bytes = c.v_codes_bytes = elems * 2;
   } else {
@@ -156,7 +181,7 @@ size_t qp_compress_workspace_bytes(int batch, int n_q_heads, int n_kv_heads, int
 size_t qp_decode_workspace_bytes(const qp_cache* cache) {
   if (check_cache(cache, false) != QP_OK) return 0;
   const DecDims d{cache->batch, cache->n_q_heads, cache->n_kv_heads, cache->head_dim, cache->bits, cache->group};
-  return decode_workspace_bound(d, cache->n_keep);
+  return decode_workspace_bound(d, cache_capacity(*cache));   // enough for every n_keep the arrays can hold
 }
 
 static qp_status check_score_args(const void* Q_win, const void* K, int batch, int Hq, int Hkv, int D, int L, int w,
@@ -199,6 +224,7 @@ qp_status qp_gather_quantize(const void* K, const void* V, const int32_t* kept_i
   if (s != QP_OK) return s;
   if (cache->n_keep > L) return QP_ERR_BUDGET;
   if (!aligned16(K) || !aligned16(V)) return QP_ERR_ALIGNMENT;
+  cache_written(static_cast<cudaStream_t>(stream));
   return launch_gather_quantize(K, V, kept_idx, L, *cache, static_cast<cudaStream_t>(stream)) == cudaSuccess
              ? QP_OK : QP_ERR_CUDA;
 }
@@ -223,6 +249,7 @@ qp_status qp_compress_layer(const void* K, const void* V, const void* Q_win, int
   const ScoreWorkspace sw = score_workspace(batch, n_q_heads, n_kv_heads, L, w);
   if (workspace_bytes < sw.total) return QP_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cache_written(st);
   float* pooled = reinterpret_cast<float*>(static_cast<char*>(workspace) + sw.pooled);
   const ScoreDims d{batch, n_q_heads, n_kv_heads, head_dim, L, w, pool};
   if (launch_window_scores(Q_win, K, d, pooled, workspace, st) != cudaSuccess) return QP_ERR_CUDA;
@@ -231,8 +258,8 @@ qp_status qp_compress_layer(const void* K, const void* V, const void* Q_win, int
   return QP_OK;
 }
 
-qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches, void* const* out,
-                                void* workspace, size_t workspace_bytes, void* stream) {
+qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const qp_cache* caches, const qp_tail* tails,
+                                     void* const* out, void* workspace, size_t workspace_bytes, void* stream) {
   if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !q || !caches || !out || !workspace) return QP_ERR_INVALID_ARG;
   if (!aligned16(workspace)) return QP_ERR_ALIGNMENT;
   const qp_cache& c0 = caches[0];
@@ -250,8 +277,23 @@ qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cac
     tab.l[l] = DecLayer{c.k_codes, c.v_codes,
                         static_cast<const __half*>(c.k_scale), static_cast<const __half*>(c.k_zero),
                         static_cast<const __half*>(c.v_scale), static_cast<const __half*>(c.v_zero),
-                        q[l], out[l], c.n_keep, 0, 0, 0};
+                        q[l], out[l], c.n_keep, 0, 0, cache_capacity(c)};
   }
+  // tails: only when some layer has tokens waiting (B = 16 never has)
+  bool any_tail = false;
+  if (tails && c0.bits < 16)
+    for (int l = 0; l < n_layers; ++l) {
+      const qp_tail& t = tails[l];
+      if (t.n_tail < 0 || t.n_tail >= c0.group) return QP_ERR_INVALID_ARG;
+      if (t.n_tail > 0) {
+        if (!t.k_tail || !t.v_tail) return QP_ERR_INVALID_ARG;
+        if (!aligned16(t.k_tail) || !aligned16(t.v_tail)) return QP_ERR_ALIGNMENT;
+        any_tail = true;
+      }
+    }
+  TailTable ttab;
+  if (any_tail)
+    for (int l = 0; l < n_layers; ++l) ttab.l[l] = TailLayer{tails[l].k_tail, tails[l].v_tail, tails[l].n_tail, 0};
   const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
   if (workspace_bytes < decode_plan(tab, d)) return QP_ERR_WORKSPACE;
   // everything the attention kernel reads before it waits for the stream's previous kernel, and what this
@@ -277,8 +319,72 @@ qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cac
   if (cudaGetDevice(&device) != cudaSuccess) return QP_ERR_CUDA;
   const PrevOutputs::Decision dec =
       g_prev_outputs.check_and_record(device, static_cast<cudaStream_t>(stream), reads, writes);
-  return launch_decode(tab, d, workspace, dec.parity, static_cast<cudaStream_t>(stream), dec.overlap) == cudaSuccess
+  return launch_decode(tab, d, workspace, dec.parity, static_cast<cudaStream_t>(stream), dec.overlap,
+                       any_tail ? &ttab : nullptr) == cudaSuccess
              ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches, void* const* out,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  return qp_decode_attn_tail_layers(n_layers, q, caches, nullptr, out, workspace, workspace_bytes, stream);
+}
+
+qp_status qp_decode_attn_tail(const void* q, const qp_cache* cache, const qp_tail* tail, void* out, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+  if (!cache) return QP_ERR_INVALID_ARG;
+  const void* qs[1] = {q};
+  void* os[1] = {out};
+  return qp_decode_attn_tail_layers(1, qs, cache, tail, os, workspace, workspace_bytes, stream);
+}
+
+qp_status qp_append_kv_layers(int n_layers, const void* const* k_new, const void* const* v_new, qp_cache* caches,
+                              qp_tail* tails, void* stream) {
+  if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !k_new || !v_new || !caches) return QP_ERR_INVALID_ARG;
+  const qp_cache& c0 = caches[0];
+  if (c0.bits < 16 && !tails) return QP_ERR_INVALID_ARG;
+  int flush[QP_MAX_LAYERS], n_flush = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const qp_cache& c = caches[l];
+    const qp_status s = check_cache(&c, true);
+    if (s != QP_OK) return s;
+    if (c.batch != c0.batch || c.n_q_heads != c0.n_q_heads || c.n_kv_heads != c0.n_kv_heads ||
+        c.head_dim != c0.head_dim || c.bits != c0.bits || c.group != c0.group)
+      return QP_ERR_INVALID_ARG;
+    if (!k_new[l] || !v_new[l]) return QP_ERR_INVALID_ARG;
+    if (!aligned16(k_new[l]) || !aligned16(v_new[l])) return QP_ERR_ALIGNMENT;
+    if (c.bits == 16) {
+      if (c.n_keep + 1 > cache_capacity(c)) return QP_ERR_BUDGET;
+      continue;
+    }
+    const qp_tail& t = tails[l];
+    if (t.n_tail < 0 || t.n_tail >= c.group || !t.k_tail || !t.v_tail) return QP_ERR_INVALID_ARG;
+    if (!aligned16(t.k_tail) || !aligned16(t.v_tail)) return QP_ERR_ALIGNMENT;
+    if (t.n_tail + 1 == c.group) {
+      if (c.n_keep + c.group > cache_capacity(c)) return QP_ERR_BUDGET;
+      flush[n_flush++] = l;
+    }
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (c0.bits == 16 || n_flush > 0) cache_written(st);          // arrays the next decode call reads are written
+  if (launch_append_rows(n_layers, k_new, v_new, caches, tails, st) != cudaSuccess) return QP_ERR_CUDA;
+  if (n_flush > 0 && launch_flush_tails(n_flush, flush, caches, tails, st) != cudaSuccess) return QP_ERR_CUDA;
+  for (int l = 0; l < n_layers; ++l) {
+    if (c0.bits == 16) {
+      caches[l].n_keep += 1;
+    } else if (tails[l].n_tail + 1 == c0.group) {
+      tails[l].n_tail = 0;
+      caches[l].n_keep += c0.group;
+    } else {
+      tails[l].n_tail += 1;
+    }
+  }
+  return QP_OK;
+}
+
+qp_status qp_append_kv(const void* k_new, const void* v_new, qp_cache* cache, qp_tail* tail, void* stream) {
+  const void* ks[1] = {k_new};
+  const void* vs[1] = {v_new};
+  return qp_append_kv_layers(1, ks, vs, cache, tail, stream);
 }
 
 qp_status qp_decode_attn(const void* q, const qp_cache* cache, void* out, void* workspace, size_t workspace_bytes,

@@ -83,6 +83,15 @@ cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_
 
 cudaError_t launch_gather_quantize(const void* K, const void* V, const int32_t* kept, int L, const qp_cache& c,
                                    cudaStream_t st);
+// tokens per (batch, KV head) the arrays of c are sized for
+inline int cache_capacity(const qp_cache& c) { return c.n_cap > 0 ? c.n_cap : c.n_keep; }
+
+// decode-time appends: new rows into the tail (or, at 16 bit, into the cache), and the quantization of full
+// tails into the caches' next group; each one launch over all layers
+cudaError_t launch_append_rows(int n_layers, const void* const* k_new, const void* const* v_new, const qp_cache* caches,
+                               const qp_tail* tails, cudaStream_t st);
+cudaError_t launch_flush_tails(int n_layers, const int* which, const qp_cache* caches, const qp_tail* tails,
+                               cudaStream_t st);
 
 // decode: per-layer device pointers, passed by value as a kernel parameter
 struct DecLayer {
@@ -97,7 +106,7 @@ struct DecLayer {
   int n;          // kept tokens of this layer
   int part_base;  // chunked kernel: first partial slot of this layer (in units of (bh, split) slots)
   int tile_base;  // flat-range kernel: index of this layer's first 32-token tile in the flat tile sequence
-  int reserved_;
+  int ns;         // tokens the arrays have room for per (batch, KV head): the stride between heads (>= n)
 };
 struct DecTable {
   int n_layers;
@@ -108,6 +117,15 @@ struct DecTable {
 };
 struct DecDims {
   int Bt, Hq, Hkv, D, bits, group;
+};
+// unquantized tail tokens of each layer (bf16 [Bt,Hkv,group,D]); read by the merge step only
+struct TailLayer {
+  const void* kt;
+  const void* vt;
+  int n_tail, pad_;
+};
+struct TailTable {
+  TailLayer l[QP_MAX_LAYERS];
 };
 constexpr int kMaxDecodeWorkers = 2048;
 // Chooses the decomposition for the layers in tab (n and pointers already set), fills chunk / part_base or
@@ -125,14 +143,18 @@ DecWorkspace decode_workspace_layout(const DecTable& tab, const DecDims& d);
 // parity: which half this call uses.  overlap_prev: the attention kernel may start while the stream's previous
 // kernel (an earlier decode call) still runs; the caller guarantees that this launch reads nothing that kernel
 // writes and that the earlier call used the other half.
+// tails: null, or the layers' tails (the merge step then adds their tokens to the softmax)
 cudaError_t launch_decode(const DecTable& tab, const DecDims& d, void* workspace, int parity, cudaStream_t st,
-                          bool overlap_prev);
+                          bool overlap_prev, const TailTable* tails = nullptr);
+// merge of the partial records plus the tail tokens, for either decomposition (chunked: tab.n_workers == 0)
+cudaError_t launch_merge_tail(const DecTable& tab, const DecDims& d, const float* partials, const TailTable& tails,
+                              cudaStream_t st, bool programmatic);
 int sm_count();   // SMs of the current device (cached)
 // tensor-core split-K kernel and its merge
 bool decode_mma_supported(const DecDims& d);
 int decode_mma_workers_per_sm(const DecDims& d);     // workers (see DecTable::n_workers) resident per SM
 int decode_mma_tiles_per_worker_min(const DecDims& d);   // small launches use fewer workers, not emptier ones
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
-                              bool overlap_prev);
+                              bool overlap_prev, const TailTable* tails = nullptr);
 
 }  // namespace qp

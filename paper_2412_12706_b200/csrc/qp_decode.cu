@@ -36,7 +36,7 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
   constexpr uint32_t QMAX = BITS < 16 ? (1u << BITS) - 1u : 0u;
   const int layer = blockIdx.z, bh = blockIdx.y, split = blockIdx.x;
   const DecLayer& ly = tab.l[layer];
-  const int n = ly.n, t_begin = split * tab.chunk;
+  const int n = ly.n, ns = ly.ns, t_begin = split * tab.chunk;
   if (t_begin >= n) return;
   const int t_end = min(n, t_begin + tab.chunk);
   const int D = dm.D, G = dm.Hq / dm.Hkv, g = dm.group, wpg = g * BITS / 32, ngv = D / g;
@@ -76,7 +76,7 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
     for (int h = 0; h < MAXG; ++h) lg[h] = 0.f;
     if constexpr (BITS < 16) {
       const int u = tk / g, e = tk % g;
-      const size_t base = ((size_t)bh * (n / g) + u) * D;
+      const size_t base = ((size_t)bh * (ns / g) + u) * D;
       const int wsel = e / PER, sh = (e % PER) * BITS;
       for (int d = 0; d < D; ++d) {
         const uint32_t c = (kc[(base + d) * wpg + wsel] >> sh) & QMAX;
@@ -86,7 +86,7 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
           if (h < G) lg[h] = fmaf(sq[h][d], kf, lg[h]);
       }
     } else {
-      const uint16_t* row = k16 + ((size_t)bh * n + tk) * D;
+      const uint16_t* row = k16 + ((size_t)bh * ns + tk) * D;
       for (int d = 0; d < D; ++d) {
         const float kf = bf16_bits_to_f32(row[d]);
 #pragma unroll
@@ -120,11 +120,11 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
         if (d < D) {
           if constexpr (BITS < 16) {
             const int e2 = d % g;
-            const size_t gi = ((size_t)bh * n + tok2) * ngv + d / g;
+            const size_t gi = ((size_t)bh * ns + tok2) * ngv + d / g;
             const uint32_t c = (vc[gi * wpg + e2 / PER] >> ((e2 % PER) * BITS)) & QMAX;
             vf[i] = fmaf((float)c, __half2float(ly.vs[gi]), __half2float(ly.vz[gi]));
           } else {
-            vf[i] = bf16_bits_to_f32(v16[((size_t)bh * n + tok2) * D + d]);
+            vf[i] = bf16_bits_to_f32(v16[((size_t)bh * ns + tok2) * D + d]);
           }
         }
       }
@@ -266,11 +266,12 @@ size_t decode_workspace_bound(const DecDims& d, int n_keep) {
 }
 
 cudaError_t launch_decode(const DecTable& tab, const DecDims& d, void* workspace, int parity, cudaStream_t st,
-                          bool overlap_prev) {
+                          bool overlap_prev, const TailTable* tails) {
   if (decode_mma_supported(d)) {
     const DecWorkspace ws = decode_workspace_layout(tab, d);
     unsigned char* base = static_cast<unsigned char*>(workspace);
-    return launch_decode_mma(tab, d, reinterpret_cast<float*>(base + (parity ? ws.record_bytes : 0)), st, overlap_prev);
+    return launch_decode_mma(tab, d, reinterpret_cast<float*>(base + (parity ? ws.record_bytes : 0)), st, overlap_prev,
+                             tails);
   }
   float* partials = static_cast<float*>(workspace);
   int max_splits = 1;
@@ -285,6 +286,7 @@ cudaError_t launch_decode(const DecTable& tab, const DecDims& d, void* workspace
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  if (tails) return launch_merge_tail(tab, d, partials, *tails, st, false);
   decode_merge_kernel<<<dim3(d.Bt * d.Hq, tab.n_layers), 128, 0, st>>>(tab, d, partials);
   return cudaGetLastError();
 }

@@ -126,7 +126,7 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const unsigned char *gKc, *gKm, *gVc, *gVm;
   auto set_head = [&]() {
     const DecLayer& ly = tab.l[p_li];
-    const size_t n = (size_t)ly.n, bh = (size_t)p_bh;
+    const size_t n = (size_t)ly.ns, bh = (size_t)p_bh;   // head stride: the arrays' capacity
     const int u = p_tile / GT, sub = p_tile % GT;
     // (a key group of GROUP tokens is GROUP/2 bytes per channel: a tile's 32 tokens are 16 of them)
     gKc = static_cast<const unsigned char*>(ly.kc) + bh * n * (D / 2) + (size_t)u * D * (GROUP / 2) + sub * 16 +
@@ -501,12 +501,13 @@ cudaError_t launch_decode_mma4(const DecTable& tab, const DecDims& d, float* par
 }
 
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
-                              bool overlap_prev) {
+                              bool overlap_prev, const TailTable* tails) {
   cudaError_t e = d.bits == 4   ? launch_decode_mma4(tab, d, partials, st, overlap_prev)
                   : d.bits == 8 ? launch_decode_mma8(tab, d, partials, st, overlap_prev)
                   : d.bits == 16 ? launch_decode_mma16(tab, d, partials, st, overlap_prev)
                                 : launch_decode_mma2(tab, d, partials, st, overlap_prev);
   if (e != cudaSuccess) return e;
+  if (tails) return launch_merge_tail(tab, d, partials, *tails, st, true);
   const int items = d.Bt * d.Hq * tab.n_layers;
   cudaLaunchConfig_t cfg = {};
   const int row_blocks = (items + MG_WARPS - 1) / MG_WARPS;

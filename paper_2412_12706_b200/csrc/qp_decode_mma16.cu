@@ -67,8 +67,8 @@ decode_mma16_kernel(const __grid_constant__ DecTable tab, const DecDims dm, floa
     const int rel = (int)(cur - ly.tile_base), bh = rel / tph, tile_begin = rel % tph;
     const int n_tiles = (int)min((long long)(tph - tile_begin), f_end - cur);
     const int b = bh / dm.Hkv, hk = bh % dm.Hkv;
-    const unsigned char* gK = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * n * D * 2;
-    const unsigned char* gV = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * n * D * 2;
+    const unsigned char* gK = static_cast<const unsigned char*>(ly.kc) + (size_t)bh * ly.ns * D * 2;
+    const unsigned char* gV = static_cast<const unsigned char*>(ly.vc) + (size_t)bh * ly.ns * D * 2;
 
     auto issue_tile = [&](int tile, int stage) {
       const uint32_t sb = wsm_u + stage * TL::BYTES;

@@ -146,7 +146,7 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const unsigned char *gKc, *gKm, *gVc, *gVs, *gVz;             // per-lane sources of the tile under the copy cursor
   auto set_head = [&]() {
     const DecLayer& ly = tab.l[p_li];
-    const size_t n = (size_t)ly.n, bh = (size_t)p_bh, tile = (size_t)p_tile;
+    const size_t n = (size_t)ly.ns, bh = (size_t)p_bh, tile = (size_t)p_tile;   // head stride: capacity
     gKc = static_cast<const unsigned char*>(ly.kc) + bh * n * (D / 4) + tile * D * 8 + lane * 8;
     gVc = static_cast<const unsigned char*>(ly.vc) + bh * n * (D / 4) + tile * 8 * D + lane * 8;
     gKm = reinterpret_cast<const unsigned char*>(k_arr ? ly.kz : ly.ks) + (bh * (n >> 5) + tile) * D * 2 + k_j * 16;

@@ -100,7 +100,7 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const unsigned char *gKc, *gKm, *gVc, *gVm;                   // per-lane sources of the tile under the copy cursor
   auto set_head = [&]() {
     const DecLayer& ly = tab.l[p_li];
-    const size_t n = (size_t)ly.n, bh = (size_t)p_bh;
+    const size_t n = (size_t)ly.ns, bh = (size_t)p_bh;   // head stride: the arrays' capacity
     const int u = p_tile / GT, sub = p_tile % GT;
     // (a key group of GROUP tokens is GROUP bytes per channel: a tile's 32 tokens are 32 of them, two pieces)
     gKc = static_cast<const unsigned char*>(ly.kc) + bh * n * D + (size_t)u * D * GROUP + sub * 32 +

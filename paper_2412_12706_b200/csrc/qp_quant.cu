@@ -43,19 +43,41 @@ __device__ __forceinline__ uint32_t quant_code(float x, const QParams& p, int qm
   return min((uint32_t)r, (uint32_t)qmax);
 }
 
-template <int BITS>
+// One layer's arguments.  Sources: K, V rows [BH, L, D]; kept [BH, n_idx] positions of the rows to take
+// (null: row u*g + e itself, the case of a full tail).  Destinations: group u0 + u of arrays that have room for
+// ns tokens per (batch, KV head).
+struct QuantLayer {
+  const uint16_t *K, *V;
+  const int32_t* kept;
+  uint32_t *Kc, *Vc;
+  __half *Ks, *Kz, *Vs, *Vz;
+  int L, n_idx, ns, u0;
+};
+template <int NL>
+struct QuantTable {
+  QuantLayer l[NL];
+};
+
+template <int BITS, int NL>
 __global__ void __launch_bounds__(128)
-gather_quant_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ V,
-                    const int32_t* __restrict__ kept, int L, int D, int n, int g, uint32_t* __restrict__ Kc,
-                    __half* __restrict__ Ks, __half* __restrict__ Kz, uint32_t* __restrict__ Vc,
-                    __half* __restrict__ Vs, __half* __restrict__ Vz) {
+gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   extern __shared__ __align__(16) uint16_t sK[];   // [g][D] gathered key rows
   __shared__ int sidx[128];
   constexpr int QMAX = (1 << BITS) - 1, PER = 32 / BITS;
+  const QuantLayer& ql = tab.l[blockIdx.z];
+  const uint16_t* __restrict__ K = ql.K;
+  const uint16_t* __restrict__ V = ql.V;
+  const int32_t* __restrict__ kept = ql.kept;
+  uint32_t* __restrict__ Kc = ql.Kc;
+  uint32_t* __restrict__ Vc = ql.Vc;
+  __half* __restrict__ Ks = ql.Ks; __half* __restrict__ Kz = ql.Kz;
+  __half* __restrict__ Vs = ql.Vs; __half* __restrict__ Vz = ql.Vz;
+  const int L = ql.L, n = ql.n_idx, ns = ql.ns;
   const int u = blockIdx.x, bh = blockIdx.y, tid = threadIdx.x, nthr = blockDim.x;
+  const int ud = ql.u0 + u;                        // destination group
   const int wpg = g * BITS / 32;
 
-  for (int e = tid; e < g; e += nthr) sidx[e] = kept[(size_t)bh * n + (size_t)u * g + e];
+  for (int e = tid; e < g; e += nthr) sidx[e] = kept ? kept[(size_t)bh * n + (size_t)u * g + e] : u * g + e;
   __syncthreads();
   const uint16_t* Kh = K + (size_t)bh * L * D;
   const uint16_t* Vh = V + (size_t)bh * L * D;
@@ -75,7 +97,7 @@ gather_quant_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__
       mx = fmaxf(mx, x);
     }
     const QParams p = group_params(mn, mx, QMAX);
-    const size_t gi = ((size_t)bh * (n / g) + u) * D + d;
+    const size_t gi = ((size_t)bh * (ns / g) + ud) * D + d;
     uint32_t* dst = Kc + gi * wpg;
     for (int wd = 0; wd < wpg; wd += 4) {       // wpg is 2 (B=2,g=32) or a multiple of 4
       uint32_t wv[4] = {0u, 0u, 0u, 0u};
@@ -108,7 +130,7 @@ gather_quant_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__
       }
     }
     const QParams p = group_params(mn, mx, QMAX);
-    const size_t gi = ((size_t)bh * n + (size_t)u * g + e) * ngv + v;
+    const size_t gi = ((size_t)bh * ns + (size_t)ud * g + e) * ngv + v;
     uint32_t* dst = Vc + gi * wpg;
     // second sweep over the group in 16-byte pieces (8 channels); a piece fills 8/PER words
     constexpr int WPP = PER >= 8 ? 1 : 8 / PER;                 // words completed per piece (PER 16: half a word)
@@ -145,44 +167,116 @@ gather_quant_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__
 // B = 16: plain gather of the kept bf16 rows
 __global__ void __launch_bounds__(128)
 gather_rows_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ V,
-                   const int32_t* __restrict__ kept, int L, int D, int n, uint16_t* __restrict__ Ko,
+                   const int32_t* __restrict__ kept, int L, int D, int n, int ns, uint16_t* __restrict__ Ko,
                    uint16_t* __restrict__ Vo) {
   const int bh = blockIdx.y, cpr = D / 8;            // 16-byte chunks per row
   const int rows_per_blk = blockDim.x / cpr;
   const int t = blockIdx.x * rows_per_blk + threadIdx.x / cpr, c = (threadIdx.x % cpr) * 8;
   if (t >= n || (int)threadIdx.x >= rows_per_blk * cpr) return;
   const size_t src = ((size_t)bh * L + kept[(size_t)bh * n + t]) * D + c;
-  const size_t dst = ((size_t)bh * n + t) * D + c;
+  const size_t dst = ((size_t)bh * ns + t) * D + c;   // ns: tokens the destination has room for
   *reinterpret_cast<uint4*>(Ko + dst) = *reinterpret_cast<const uint4*>(K + src);
   *reinterpret_cast<uint4*>(Vo + dst) = *reinterpret_cast<const uint4*>(V + src);
+}
+
+template <int NL>
+cudaError_t launch_quant_table(int bits, const QuantTable<NL>& tab, dim3 grid, int D, int g, cudaStream_t st) {
+  const size_t smem = (size_t)g * D * sizeof(uint16_t);
+  switch (bits) {
+    case 2: gather_quant_kernel<2, NL><<<grid, 128, smem, st>>>(tab, D, g); break;
+    case 4: gather_quant_kernel<4, NL><<<grid, 128, smem, st>>>(tab, D, g); break;
+    case 8: gather_quant_kernel<8, NL><<<grid, 128, smem, st>>>(tab, D, g); break;
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
+}
+
+// rows of the new token into the tails (or, at 16 bit, into the caches): 16 bytes per thread
+struct AppendLayer {
+  const uint16_t *k_new, *v_new;   // [BH, D]
+  uint16_t *k_dst, *v_dst;         // row of head 0; heads are head_stride elements apart
+  size_t head_stride;
+};
+struct AppendTable {
+  AppendLayer l[QP_MAX_LAYERS];
+};
+__global__ void __launch_bounds__(128)
+append_rows_kernel(const __grid_constant__ AppendTable tab, int BH, int D) {
+  const AppendLayer& a = tab.l[blockIdx.y];
+  const int cpr = D / 8;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;          // 16-byte piece of the layer's [BH, D] rows
+  if (i >= BH * cpr) return;
+  const int bh = i / cpr, c = (i % cpr) * 8;
+  *reinterpret_cast<uint4*>(a.k_dst + bh * a.head_stride + c) = *reinterpret_cast<const uint4*>(a.k_new + (size_t)bh * D + c);
+  *reinterpret_cast<uint4*>(a.v_dst + bh * a.head_stride + c) = *reinterpret_cast<const uint4*>(a.v_new + (size_t)bh * D + c);
 }
 
 }  // namespace
 
 cudaError_t launch_gather_quantize(const void* K, const void* V, const int32_t* kept, int L, const qp_cache& c,
                                    cudaStream_t st) {
-  const int BH = c.batch * c.n_kv_heads, D = c.head_dim, n = c.n_keep, g = c.group;
+  const int BH = c.batch * c.n_kv_heads, D = c.head_dim, n = c.n_keep, g = c.group, ns = cache_capacity(c);
   const uint16_t* k = static_cast<const uint16_t*>(K);
   const uint16_t* v = static_cast<const uint16_t*>(V);
   if (c.bits == 16) {
     const int rows_per_blk = 128 / (D / 8);
     gather_rows_kernel<<<dim3((n + rows_per_blk - 1) / rows_per_blk, BH), 128, 0, st>>>(
-        k, v, kept, L, D, n, static_cast<uint16_t*>(c.k_codes), static_cast<uint16_t*>(c.v_codes));
+        k, v, kept, L, D, n, ns, static_cast<uint16_t*>(c.k_codes), static_cast<uint16_t*>(c.v_codes));
     return cudaGetLastError();
   }
-  const dim3 grid(n / g, BH);
-  const size_t smem = (size_t)g * D * sizeof(uint16_t);
-  uint32_t* kc = static_cast<uint32_t*>(c.k_codes);
-  uint32_t* vc = static_cast<uint32_t*>(c.v_codes);
-  __half *ks = static_cast<__half*>(c.k_scale), *kz = static_cast<__half*>(c.k_zero);
-  __half *vs = static_cast<__half*>(c.v_scale), *vz = static_cast<__half*>(c.v_zero);
-  switch (c.bits) {
-    case 2: gather_quant_kernel<2><<<grid, 128, smem, st>>>(k, v, kept, L, D, n, g, kc, ks, kz, vc, vs, vz); break;
-    case 4: gather_quant_kernel<4><<<grid, 128, smem, st>>>(k, v, kept, L, D, n, g, kc, ks, kz, vc, vs, vz); break;
-    case 8: gather_quant_kernel<8><<<grid, 128, smem, st>>>(k, v, kept, L, D, n, g, kc, ks, kz, vc, vs, vz); break;
-    default: return cudaErrorInvalidValue;
+  QuantTable<1> tab;
+  tab.l[0] = QuantLayer{k, v, kept, static_cast<uint32_t*>(c.k_codes), static_cast<uint32_t*>(c.v_codes),
+                        static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
+                        static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, n, ns, 0};
+  return launch_quant_table<1>(c.bits, tab, dim3(n / g, BH, 1), D, g, st);
+}
+
+cudaError_t launch_append_rows(int n_layers, const void* const* k_new, const void* const* v_new, const qp_cache* caches,
+                               const qp_tail* tails, cudaStream_t st) {
+  const qp_cache& c0 = caches[0];
+  const int BH = c0.batch * c0.n_kv_heads, D = c0.head_dim;
+  AppendTable tab;
+  for (int l = 0; l < n_layers; ++l) {
+    const qp_cache& c = caches[l];
+    AppendLayer& a = tab.l[l];
+    a.k_new = static_cast<const uint16_t*>(k_new[l]);
+    a.v_new = static_cast<const uint16_t*>(v_new[l]);
+    if (c.bits == 16) {                                          // token n_keep of the cache itself
+      a.head_stride = (size_t)cache_capacity(c) * D;
+      a.k_dst = static_cast<uint16_t*>(c.k_codes) + (size_t)c.n_keep * D;
+      a.v_dst = static_cast<uint16_t*>(c.v_codes) + (size_t)c.n_keep * D;
+    } else {                                                     // slot n_tail of the tail
+      a.head_stride = (size_t)c.group * D;
+      a.k_dst = static_cast<uint16_t*>(tails[l].k_tail) + (size_t)tails[l].n_tail * D;
+      a.v_dst = static_cast<uint16_t*>(tails[l].v_tail) + (size_t)tails[l].n_tail * D;
+    }
   }
+  const int pieces = BH * (D / 8);
+  append_rows_kernel<<<dim3((pieces + 127) / 128, n_layers), 128, 0, st>>>(tab, BH, D);
   return cudaGetLastError();
+}
+
+// which[0..n_layers): indices into caches / tails of the layers whose tail is full
+cudaError_t launch_flush_tails(int n_layers, const int* which, const qp_cache* caches, const qp_tail* tails,
+                               cudaStream_t st) {
+  const qp_cache& c0 = caches[which[0]];
+  const int BH = c0.batch * c0.n_kv_heads, D = c0.head_dim, g = c0.group;
+  auto fill = [&](QuantLayer& ql, int l) {
+    const qp_cache& c = caches[l];
+    ql = QuantLayer{static_cast<const uint16_t*>(tails[l].k_tail), static_cast<const uint16_t*>(tails[l].v_tail), nullptr,
+                    static_cast<uint32_t*>(c.k_codes), static_cast<uint32_t*>(c.v_codes),
+                    static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
+                    static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero),
+                    g, g, cache_capacity(c), c.n_keep / g};
+  };
+  if (n_layers == 1) {
+    QuantTable<1> tab;
+    fill(tab.l[0], which[0]);
+    return launch_quant_table<1>(c0.bits, tab, dim3(1, BH, 1), D, g, st);
+  }
+  QuantTable<QP_MAX_LAYERS> tab;
+  for (int i = 0; i < n_layers; ++i) fill(tab.l[i], which[i]);
+  return launch_quant_table<QP_MAX_LAYERS>(c0.bits, tab, dim3(1, BH, n_layers), D, g, st);
 }
 
 }  // namespace qp

@@ -23,7 +23,9 @@ STATUS_NAMES = {0: "QP_OK", 1: "QP_ERR_INVALID_ARG", 2: "QP_ERR_UNSUPPORTED", 3:
 
 EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_workspace_bytes",
            "qp_decode_workspace_bytes", "qp_window_scores", "qp_select_topk", "qp_gather_quantize",
-           "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static"]
+           "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static",
+           "qp_cache_layout_cap", "qp_append_kv", "qp_append_kv_layers", "qp_decode_attn_tail",
+           "qp_decode_attn_tail_layers"]
 
 
 class QpError(RuntimeError):
@@ -35,12 +37,17 @@ class QpError(RuntimeError):
 class qp_cache(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("bits", ctypes.c_int32), ("group", ctypes.c_int32),
-                ("n_keep", ctypes.c_int32), ("reserved_", ctypes.c_int32),
+                ("n_keep", ctypes.c_int32), ("n_cap", ctypes.c_int32),
                 ("k_codes_bytes", ctypes.c_size_t), ("v_codes_bytes", ctypes.c_size_t),
                 ("k_meta_bytes", ctypes.c_size_t), ("v_meta_bytes", ctypes.c_size_t),
                 ("k_codes", ctypes.c_void_p), ("v_codes", ctypes.c_void_p),
                 ("k_scale", ctypes.c_void_p), ("k_zero", ctypes.c_void_p),
                 ("v_scale", ctypes.c_void_p), ("v_zero", ctypes.c_void_p)]
+
+
+class qp_tail(ctypes.Structure):
+    _fields_ = [("n_tail", ctypes.c_int32), ("reserved_", ctypes.c_int32),
+                ("k_tail", ctypes.c_void_p), ("v_tail", ctypes.c_void_p)]
 
 
 _lib = None
@@ -80,6 +87,17 @@ def lib() -> ctypes.CDLL:
         L.qp_decode_attn_layers.argtypes = [i, ctypes.POINTER(p), cp, ctypes.POINTER(p), p, sz, p]
         L.qp_decode_attn_static.restype = i
         L.qp_decode_attn_static.argtypes = [p, cp, p, p]
+        tp = ctypes.POINTER(qp_tail)
+        L.qp_cache_layout_cap.restype = i
+        L.qp_cache_layout_cap.argtypes = [i, i, i, i, i, i, i, i, cp]
+        L.qp_append_kv.restype = i
+        L.qp_append_kv.argtypes = [p, p, cp, tp, p]
+        L.qp_append_kv_layers.restype = i
+        L.qp_append_kv_layers.argtypes = [i, ctypes.POINTER(p), ctypes.POINTER(p), cp, tp, p]
+        L.qp_decode_attn_tail.restype = i
+        L.qp_decode_attn_tail.argtypes = [p, cp, tp, p, p, sz, p]
+        L.qp_decode_attn_tail_layers.restype = i
+        L.qp_decode_attn_tail_layers.argtypes = [i, ctypes.POINTER(p), cp, tp, ctypes.POINTER(p), p, sz, p]
         _lib = L
     return _lib
 
@@ -115,6 +133,14 @@ def cache_layout(batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, bit
     return c
 
 
+def cache_layout_cap(batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, bits: int, group: int,
+                     n_keep_: int, n_cap: int) -> qp_cache:
+    c = qp_cache()
+    _check(lib().qp_cache_layout_cap(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_, n_cap,
+                                     ctypes.byref(c)), "qp_cache_layout_cap")
+    return c
+
+
 def compress_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim, L, w) -> int:
     return int(lib().qp_compress_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim, L, w))
 
@@ -141,10 +167,12 @@ class Cache:
         return d.k_codes_bytes + d.v_codes_bytes + 2 * d.k_meta_bytes + 2 * d.v_meta_bytes
 
 
-def alloc_cache(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_, device="cuda") -> Cache:
-    """Allocates the buffers of ``qp_cache_layout`` with torch and fills in the pointers."""
-    d = cache_layout(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_)
-    n, D, g = n_keep_, head_dim, group
+def alloc_cache(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_, device="cuda",
+                n_cap: int = 0) -> Cache:
+    """Allocates the buffers of ``qp_cache_layout`` (``qp_cache_layout_cap`` when ``n_cap`` leaves room
+    for appended tokens) with torch and fills in the pointers."""
+    d = cache_layout_cap(batch, n_q_heads, n_kv_heads, head_dim, bits, group, n_keep_, n_cap)
+    n, D, g = (n_cap or n_keep_), head_dim, group
     if bits == 16:
         kc = torch.empty((batch, n_kv_heads, n, D), dtype=torch.bfloat16, device=device)
         vc = torch.empty_like(kc)
@@ -209,13 +237,14 @@ def gather_quantize(K: torch.Tensor, V: torch.Tensor, kept_idx: torch.Tensor, ca
 
 def compress_layer(K: torch.Tensor, V: torch.Tensor, Q_win: torch.Tensor, budget_bits: int, bits: int,
                    group: int = 32, pool: int = 7, cache: Cache | None = None,
-                   kept_idx: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
-    """qp_compress_layer: returns (cache, kept_idx).  Buffers are allocated with torch when not given."""
+                   kept_idx: torch.Tensor | None = None, workspace: torch.Tensor | None = None, n_cap: int = 0):
+    """qp_compress_layer: returns (cache, kept_idx).  Buffers are allocated with torch when not given
+    (with room for ``n_cap`` tokens per KV head when ``n_cap`` is given)."""
     _dev_bf16(K); _dev_bf16(V); _dev_bf16(Q_win)
     Bt, Hq, Hkv, D, L, w = _dims(K, Q_win)
     n = n_keep(budget_bits, bits, group, L, w)
     if cache is None:
-        cache = alloc_cache(Bt, Hq, Hkv, D, bits, group, n, K.device)
+        cache = alloc_cache(Bt, Hq, Hkv, D, bits, group, n, K.device, n_cap)
     if kept_idx is None:
         kept_idx = torch.empty((Bt, Hkv, n), dtype=torch.int32, device=K.device)
     if workspace is None:
@@ -267,6 +296,77 @@ def decode_attn_layers(batch: LayerBatch) -> None:
            "qp_decode_attn_layers")
 
 
+@dataclass
+class Tail:
+    """Device buffers of one layer's unquantized tail plus the C descriptor (host state: n_tail)."""
+    desc: qp_tail
+    k_tail: torch.Tensor | None
+    v_tail: torch.Tensor | None
+
+
+def alloc_tail(cache: Cache, device=None) -> Tail:
+    """bf16 [Bt,Hkv,group,D] buffers for the tokens that wait for a full group (none at 16 bit)."""
+    d = cache.desc
+    t = qp_tail()
+    if d.bits == 16:
+        return Tail(t, None, None)
+    device = device or cache.k_codes.device
+    kt = torch.zeros((d.batch, d.n_kv_heads, d.group, d.head_dim), dtype=torch.bfloat16, device=device)
+    vt = torch.zeros_like(kt)
+    t.k_tail, t.v_tail = _ptr(kt), _ptr(vt)
+    return Tail(t, kt, vt)
+
+
+def append_kv(k_new: torch.Tensor, v_new: torch.Tensor, cache: Cache, tail: Tail) -> None:
+    """qp_append_kv: Eq. 2 for one layer; updates cache.desc.n_keep and tail.desc.n_tail."""
+    _dev_bf16(k_new); _dev_bf16(v_new)
+    _check(lib().qp_append_kv(_ptr(k_new), _ptr(v_new), ctypes.byref(cache.desc), ctypes.byref(tail.desc),
+                              _stream()), "qp_append_kv")
+
+
+def decode_attn_tail(q: torch.Tensor, cache: Cache, tail: Tail, out: torch.Tensor | None = None,
+                     workspace: torch.Tensor | None = None) -> torch.Tensor:
+    _dev_bf16(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_decode_workspace(decode_workspace_bytes(cache), q.device)
+    _check(lib().qp_decode_attn_tail(_ptr(q), ctypes.byref(cache.desc), ctypes.byref(tail.desc), _ptr(out),
+                                     _ptr(workspace), workspace.numel(), _stream()), "qp_decode_attn_tail")
+    return out
+
+
+class GenBatch:
+    """Marshalled host arrays for a generation loop over many layers: ``qp_append_kv_layers`` followed by
+    ``qp_decode_attn_tail_layers``.  The descriptor arrays are owned here and updated in place by the
+    append call (the Cache / Tail objects passed in keep their initial descriptors)."""
+
+    def __init__(self, qs, k_news, v_news, caches: list[Cache], tails: list[Tail], outs,
+                 workspace: torch.Tensor | None = None):
+        n = len(caches)
+        assert 1 <= n <= QP_MAX_LAYERS and len(qs) == len(outs) == len(tails) == len(k_news) == len(v_news) == n
+        self.n = n
+        self.keep = (qs, k_news, v_news, caches, tails, outs)
+        arr = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+        self.q_arr, self.out_arr, self.kn_arr, self.vn_arr = arr(qs), arr(outs), arr(k_news), arr(v_news)
+        self.cache_arr = (qp_cache * n)(*[c.desc for c in caches])
+        self.tail_arr = (qp_tail * n)(*[t.desc for t in tails])
+        if workspace is None:
+            workspace = new_decode_workspace(sum(decode_workspace_bytes(c) for c in caches), qs[0].device)
+        self.workspace = workspace
+
+
+def append_kv_layers(batch: GenBatch) -> None:
+    _check(lib().qp_append_kv_layers(batch.n, batch.kn_arr, batch.vn_arr, batch.cache_arr, batch.tail_arr,
+                                     _stream()), "qp_append_kv_layers")
+
+
+def decode_attn_tail_layers(batch: GenBatch) -> None:
+    _check(lib().qp_decode_attn_tail_layers(batch.n, batch.q_arr, batch.cache_arr, batch.tail_arr, batch.out_arr,
+                                            _ptr(batch.workspace), batch.workspace.numel(), _stream()),
+           "qp_decode_attn_tail_layers")
+
+
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -300,3 +400,8 @@ qp_compress_layer = compress_layer
 qp_decode_attn = decode_attn
 qp_decode_attn_layers = decode_attn_layers
 qp_decode_attn_static = decode_attn_static
+qp_cache_layout_cap = cache_layout_cap
+qp_append_kv = append_kv
+qp_append_kv_layers = append_kv_layers
+qp_decode_attn_tail = decode_attn_tail
+qp_decode_attn_tail_layers = decode_attn_tail_layers

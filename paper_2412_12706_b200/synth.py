@@ -130,7 +130,7 @@ LLAMA70B_32K_B4 = Workload("llama3-70b-32k-b4-4bit-pyramid", 80, 4, 64, 8, 128, 
 WORKLOADS = {w.name: w for w in (TINY, LLAMA8B_8K, LLAMA8B_32K_B8, sweep_128k(16), sweep_128k(8),
                                  sweep_128k(4), sweep_128k(2), LLAMA70B_32K_B4)}
 
-_TID_K, _TID_V, _TID_QWIN, _TID_QDEC, _TID_PHASE = 1, 2, 3, 4, 5
+_TID_K, _TID_V, _TID_QWIN, _TID_QDEC, _TID_PHASE, _TID_KNEW, _TID_VNEW = 1, 2, 3, 4, 5, 6, 7
 
 
 def _outlier_channels(wl: Workload, hk: int) -> list[int]:
@@ -191,6 +191,20 @@ def make_q_dec(wl: Workload, layer: int, step: int, device="cpu") -> torch.Tenso
     n = wl.batch * wl.n_q_heads * wl.head_dim
     return _bf16(normal_f32(wl.seed, layer, _TID_QDEC + 16 * (step + 1), n, device)
                  .view(wl.batch, wl.n_q_heads, wl.head_dim))
+
+
+def make_kv_new(wl: Workload, layer: int, step: int, device="cpu"):
+    """Key and value rows [Bt,Hkv,D] bf16 of the token generated at decode step `step` (same value
+    structure as the prompt's keys: the per-head outlier channels stay outliers)."""
+    Bt, Hkv, D = wl.batch, wl.n_kv_heads, wl.head_dim
+    n = Bt * Hkv * D
+    k = normal_f32(wl.seed, layer, _TID_KNEW + 16 * (step + 1), n, device).view(Bt, Hkv, D)
+    v = normal_f32(wl.seed, layer, _TID_VNEW + 16 * (step + 1), n, device).view(Bt, Hkv, D)
+    if wl.structure == "outlier":
+        for hk in range(Hkv):
+            for d in _outlier_channels(wl, hk):
+                k[:, hk, d] *= wl.outlier_scale
+    return _bf16(k), _bf16(v)
 
 
 def bits_u16(x: torch.Tensor):

@@ -67,6 +67,50 @@ def test_cache_layout_sizes():
         assert e.value.status == code
 
 
+def test_tail_struct_and_capacity_layout():
+    assert ctypes.sizeof(qp.qp_tail) == 2 * 4 + 2 * 8
+    c = qp.cache_layout_cap(1, 32, 8, 128, 4, 32, 2048, 2048 + 256)
+    assert c.n_keep == 2048 and c.n_cap == 2304
+    assert c.k_codes_bytes == 8 * 2304 * 128 // 2 and c.k_meta_bytes == 8 * 2304 * 128 // 32 * 2
+    assert qp.cache_layout_cap(1, 32, 8, 128, 4, 32, 2048, 0).k_codes_bytes == qp.cache_layout(1, 32, 8, 128, 4, 32, 2048).k_codes_bytes
+    assert qp.cache_layout_cap(1, 32, 8, 128, 16, 32, 1000, 1001).k_codes_bytes == 8 * 1001 * 128 * 2
+    # the decode workspace covers every n_keep the arrays can hold
+    assert qp.decode_workspace_bytes(c) >= qp.decode_workspace_bytes(qp.cache_layout(1, 32, 8, 128, 4, 32, 2304))
+    for n_cap in (2047, 2048 + 16, -32):
+        with pytest.raises(qp.QpError) as e:
+            qp.cache_layout_cap(1, 32, 8, 128, 4, 32, 2048, n_cap)
+        assert e.value.status in (1, 3)
+
+
+def test_append_and_tail_arguments_are_checked_before_any_launch(lib):
+    A = 0x1000
+    c = qp.cache_layout_cap(1, 8, 2, 64, 4, 32, 512, 512 + 32)
+    c.k_codes = c.v_codes = c.k_scale = c.k_zero = c.v_scale = c.v_zero = A
+    t = qp.qp_tail()
+    t.k_tail = t.v_tail = A
+    cr, tr = ctypes.byref(c), ctypes.byref(t)
+    assert lib.qp_append_kv(None, A, cr, tr, None) == 1
+    assert lib.qp_append_kv(A, A + 4, cr, tr, None) == 5
+    assert lib.qp_append_kv(A, A, cr, None, None) == 1            # a quantized cache needs a tail
+    t.n_tail = 32
+    assert lib.qp_append_kv(A, A, cr, tr, None) == 1              # n_tail out of range
+    t.n_tail = 31
+    full = qp.cache_layout_cap(1, 8, 2, 64, 4, 32, 512, 512)
+    full.k_codes = full.v_codes = full.k_scale = full.k_zero = full.v_scale = full.v_zero = A
+    assert lib.qp_append_kv(A, A, ctypes.byref(full), tr, None) == 3   # the flush would not fit
+    assert full.n_keep == 512 and t.n_tail == 31                  # nothing changed
+    c16 = qp.cache_layout_cap(1, 8, 2, 64, 16, 32, 100, 100)
+    c16.k_codes = c16.v_codes = A
+    assert lib.qp_append_kv(A, A, ctypes.byref(c16), None, None) == 3
+    t.n_tail = 40
+    assert lib.qp_decode_attn_tail(A, cr, tr, A, A, 1 << 30, None) == 1
+    t.n_tail = 3
+    t.k_tail = None
+    assert lib.qp_decode_attn_tail(A, cr, tr, A, A, 1 << 30, None) == 1
+    t.k_tail = A + 2
+    assert lib.qp_decode_attn_tail(A, cr, tr, A, A, 1 << 30, None) == 5
+
+
 def test_workspace_sizes():
     assert qp.compress_workspace_bytes(1, 32, 8, 128, 8192, 32) > 8 * 8160 * 4
     assert qp.compress_workspace_bytes(1, 32, 8, 128, 32, 32) == 0

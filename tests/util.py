@@ -18,16 +18,20 @@ def bf16_val(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
-def cache_to_packed(cache) -> orc.Packed:
-    """Device cache (binding's Cache) -> oracle Packed with numpy arrays (copies to host)."""
-    d = cache.desc
+def cache_to_packed(cache, desc=None) -> orc.Packed:
+    """Device cache (binding's Cache) -> oracle Packed with numpy arrays (copies to host).  Only the
+    n_keep tokens in use are taken (the arrays may have room for more); `desc` overrides the cache's
+    own descriptor when another copy of it has been advanced by appends."""
+    d = desc if desc is not None else cache.desc
+    n, g = d.n_keep, d.group
     if d.bits == 16:
-        return orc.Packed(16, d.group, d.n_keep, bits_u16(cache.k_codes), bits_u16(cache.v_codes),
-                          None, None, None, None)
-    u32 = lambda t: t.detach().cpu().contiguous().numpy().view(np.uint32)
-    return orc.Packed(d.bits, d.group, d.n_keep, u32(cache.k_codes), u32(cache.v_codes),
-                      bits_u16(cache.k_scale), bits_u16(cache.k_zero),
-                      bits_u16(cache.v_scale), bits_u16(cache.v_zero))
+        return orc.Packed(16, g, n, np.ascontiguousarray(bits_u16(cache.k_codes)[:, :, :n]),
+                          np.ascontiguousarray(bits_u16(cache.v_codes)[:, :, :n]), None, None, None, None)
+    u32 = lambda t, m: np.ascontiguousarray(t.detach().cpu().contiguous().numpy().view(np.uint32)[:, :, :m])
+    h16 = lambda t, m: np.ascontiguousarray(bits_u16(t)[:, :, :m])
+    return orc.Packed(d.bits, g, n, u32(cache.k_codes, n // g), u32(cache.v_codes, n),
+                      h16(cache.k_scale, n // g), h16(cache.k_zero, n // g),
+                      h16(cache.v_scale, n), h16(cache.v_zero, n))
 
 
 def assert_packed_equal(got: orc.Packed, ref: orc.Packed) -> None:
