@@ -330,6 +330,52 @@ def run_gpu(args, wl):
         torch.cuda.synchronize()
         graph_ms = g0.elapsed_time(g1) / reps
 
+    # ---- generation loop: every decode step first appends the new token's key/value rows to every layer
+    #      (qp_append_kv_layers; full tails are quantized into the caches) and then attends over packed
+    #      tokens plus tail (qp_decode_attn_tail_layers).  Same grouping of sequences per call as above.
+    gen = None
+    if not args.no_generation:
+        g_steps = 2 * wl.group + 8 if wl.bits < 16 else 72      # two flushes of every tail on the way
+        room = 3 * wl.group if wl.bits < 16 else g_steps + 8
+        gen_groups = []
+        for g0 in range(0, n_seq, per_call):
+            members = seqs[g0:g0 + per_call]
+            caches, tails, kn, vn = [], [], [], []
+            for i, m in enumerate(members):
+                wls = synth.dataclasses.replace(wl, seed=shard.sequence_seed(wl.seed, rank, n_seq, g0 + i))
+                for l in range(n_layers):
+                    c, _ = qp.compress_layer(m["K"][l], m["V"][l], m["Qw"][l], wl.layer_budget_bits(l), wl.bits,
+                                             wl.group, wl.pool, workspace=ws_c, n_cap=wl.n_keep(l) + room)
+                    caches.append(c); tails.append(qp.alloc_tail(c))
+                    a, b_ = synth.make_kv_new(wls, l, 0, device=dev)
+                    kn.append(a); vn.append(b_)
+            gen_groups.append(qp.GenBatch([m["qdec"][0, l] for m in members for l in range(n_layers)], kn, vn, caches,
+                                          tails, [m["out"][l] for m in members for l in range(n_layers)]))
+        gen_bytes0 = sum(gb.cache_arr[i].n_keep for gb in gen_groups for i in range(gb.n))
+
+        def gen_step():
+            for gb in gen_groups:
+                qp.append_kv_layers(gb)
+                qp.decode_attn_tail_layers(gb)
+        for _ in range(4):
+            gen_step()
+        e0, e1 = ev(), ev()
+        e0.record(stream)
+        for _ in range(g_steps - 4):
+            gen_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        gen_ms = e0.elapsed_time(e1) / ((g_steps - 4) * len(gen_groups))
+        gen_bytes1 = sum(gb.cache_arr[i].n_keep for gb in gen_groups for i in range(gb.n))
+        # packed bytes a call reads, averaged over the loop (the caches grow by a group at every flush)
+        per_tok = Bt * Hkv * D * 2 * (2.0 if wl.bits == 16 else (wl.bits + 32 // wl.group) / 8)
+        gen_call_bytes = 0.5 * (gen_bytes0 + gen_bytes1) * per_tok / len(gen_groups)
+        gen = {"note": "per decode step and group of sequences: qp_append_kv_layers (new rows into the bf16 tails; "
+                       "full tails quantized into the caches) + qp_decode_attn_tail_layers (packed tokens + tail)",
+               "steps": g_steps - 4, "us_per_step_call": gen_ms * 1e3, "GB/s": gen_call_bytes / (gen_ms * 1e-3) / 1e9,
+               "launches_per_step_call": "3 (4 on the steps that flush)"}
+        del gen_groups
+
     # ---- end to end: host buffers in, host buffers out, through the same calls
     input_bytes = 2 * n_seq * n_layers * Bt * Hkv * L * D * 2
     # the host-buffer leg pins a copy of every input; keep it to workloads whose inputs are a few GB
@@ -380,6 +426,7 @@ def run_gpu(args, wl):
             "GB/s": dec_bytes_call / per_call / (layer_ms * 1e-3) / 1e9,
             "cuda_graph_us_per_layer_call": graph_ms * 1e3 / n_layers,
             "cuda_graph_GB/s": dec_bytes_call / per_call / (graph_ms * 1e-3) / 1e9},
+        "decode_with_append": gen,
         "decode_phase_ms_per_step": dec_ms / steps,
         "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "decode attention (split-K attention kernel + merge kernel, per call)",
@@ -468,6 +515,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling: keep only the first N layers of the workload")
     ap.add_argument("--batch", type=int, default=0, help="profiling: override the workload's batch size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-generation", action="store_true", help="skip the append + decode generation-loop figure")
     ap.add_argument("--no-layer-chain", action="store_true", help="skip the layer-by-layer / CUDA-graph figures")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
