@@ -202,6 +202,11 @@ struct AppendTable {
 };
 __global__ void __launch_bounds__(128)
 append_rows_kernel(const __grid_constant__ AppendTable tab, int BH, int D) {
+  // This kernel sits between two decode calls of a generation loop and keeps their overlap alive: it passes
+  // the launch permission on at once (the next call's attention kernel reads nothing written here), and only
+  // then waits for the stream's previous kernel, whose merge step may still be reading the tail rows.
+  asm volatile("griddepcontrol.launch_dependents;\n" ::);
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
   const AppendLayer& a = tab.l[blockIdx.y];
   const int cpr = D / 8;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;          // 16-byte piece of the layer's [BH, D] rows
@@ -252,8 +257,17 @@ cudaError_t launch_append_rows(int n_layers, const void* const* k_new, const voi
     }
   }
   const int pieces = BH * (D / 8);
-  append_rows_kernel<<<dim3((pieces + 127) / 128, n_layers), 128, 0, st>>>(tab, BH, D);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((pieces + 127) / 128, n_layers);
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, append_rows_kernel, tab, BH, D);
 }
 
 // which[0..n_layers): indices into caches / tails of the layers whose tail is full
