@@ -43,11 +43,11 @@ NOMINAL_HBM_GBS = 8000.0
 # kernel sources it was taken on: {"sha256": <hash of DECODE_KERNEL_SOURCES>, "workload": name,
 # "bytes_per_launch": dram__bytes_read.sum + dram__bytes_write.sum}
 NCU_TRAFFIC: dict = {
-    "sha256": "609b774712a2b5aaa699f6564320cb6f63d83090afe2650b97132f66e5701686",
+    "sha256": "ccfbe94ce393d476547a2a485af389d1f51c95a3f7efe052ed332c7d685250f6",
     "workload": "llama3-8b-8k-b1-4bit",
-    # captured on a 2-sequence call (168.39 MB read + 4.02 MB written per launch, mean of two launches) and
+    # captured on a 2-sequence call (168.39 MB read + 4.69 MB written per launch, mean of two launches) and
     # scaled by the sequences per call: the traffic is proportional to the tiles a launch streams
-    "bytes_per_launch_per_sequence": (168390656 + 4023296) / 2,
+    "bytes_per_launch_per_sequence": (168387968 + 4691968) / 2,
 }
 
 KERNELS_PER_COMPRESS = 6      # sweep 1, row-stat merge, sweep 2, pool, top-k, gather+quantize

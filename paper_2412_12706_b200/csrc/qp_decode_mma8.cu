@@ -18,7 +18,10 @@ constexpr int D8_THREADS = D8_WARPS * 32;
 #define QP_D8_STAGES 2
 #endif
 constexpr int D8_STAGES = QP_D8_STAGES;
-constexpr int D8_MINB = 2;
+#ifndef QP_D8_MINB
+#define QP_D8_MINB 2
+#endif
+constexpr int D8_MINB = QP_D8_MINB;
 constexpr int SP8_STRIDE = 80;
 constexpr int SP8_BYTES = 8 * SP8_STRIDE;
 

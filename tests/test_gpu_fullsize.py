@@ -22,14 +22,15 @@ DEV = "cuda"
 def _slice_packed(cache, b, hk):
     """Packed arrays of one (batch, KV head) pair as an oracle Packed with Bt = Hkv = 1."""
     d = cache.desc
-    sl = lambda t: t[b:b + 1, hk:hk + 1].contiguous()
+    n, ng = d.n_keep, d.n_keep // d.group                       # tokens / key groups in use (the arrays may have room for more)
+    sl = lambda t, m: t[b:b + 1, hk:hk + 1, :m].contiguous()
     if d.bits == 16:
-        return orc.Packed(16, d.group, d.n_keep, bits_u16(sl(cache.k_codes)), bits_u16(sl(cache.v_codes)),
+        return orc.Packed(16, d.group, n, bits_u16(sl(cache.k_codes, n)), bits_u16(sl(cache.v_codes, n)),
                           None, None, None, None)
-    u32 = lambda t: sl(t).cpu().numpy().view(np.uint32)
-    return orc.Packed(d.bits, d.group, d.n_keep, u32(cache.k_codes), u32(cache.v_codes),
-                      bits_u16(sl(cache.k_scale)), bits_u16(sl(cache.k_zero)),
-                      bits_u16(sl(cache.v_scale)), bits_u16(sl(cache.v_zero)))
+    u32 = lambda t, m: sl(t, m).cpu().numpy().view(np.uint32)
+    return orc.Packed(d.bits, d.group, n, u32(cache.k_codes, ng), u32(cache.v_codes, n),
+                      bits_u16(sl(cache.k_scale, ng)), bits_u16(sl(cache.k_zero, ng)),
+                      bits_u16(sl(cache.v_scale, n)), bits_u16(sl(cache.v_zero, n)))
 
 
 def _check_structure(kept: torch.Tensor, L: int, w: int):
@@ -116,3 +117,57 @@ def test_llama70b_pyramid_first_and_last_layer():
     assert wl.n_keep(0) == 8192 and wl.n_keep(79) == 2048          # 2x .. 0.5x of the 4096-token mean
     swaps = run_fullsize(wl, layers=[0, 79], samples=[(0, 0), (3, 6)])
     assert swaps <= 4
+
+
+def test_llama8b_generation_loop_in_the_bench_configuration():
+    """Append + decode over packed tokens and tail at the benchmark's launch shape: 128 layer descriptors
+    (32 layers of 4 sequences) per qp_append_kv_layers / qp_decode_attn_tail_layers call, tails cycling
+    through a flush.  The oracle follows SAMPLED (descriptor, KV head) pairs from the GPU's own prompt caches;
+    every output is checked for finiteness and every descriptor for its counters."""
+    wl = synth.LLAMA8B_8K
+    n_seq, nl, g, D, Hkv = 4, wl.n_layers, wl.group, wl.head_dim, wl.n_kv_heads
+    G = wl.n_q_heads // Hkv
+    steps = g + 3
+    caches, tails = [], []
+    ws = torch.empty(qp.compress_workspace_bytes(wl.batch, wl.n_q_heads, Hkv, D, wl.L, wl.w), dtype=torch.uint8, device=DEV)
+    for s in range(n_seq):
+        wls = dataclasses.replace(wl, seed=wl.seed + 1000 * s)
+        for l in range(nl):
+            k, v = synth.make_kv(wls, l, device=DEV)
+            qw = synth.make_q_win(wls, l, device=DEV)
+            c, _ = qp.compress_layer(k, v, qw, wl.budget_bits, wl.bits, g, wl.pool, workspace=ws, n_cap=wl.n_keep(l) + 2 * g)
+            caches.append(c); tails.append(qp.alloc_tail(c))
+    n_desc = len(caches)
+    samples = [(0, 0), (37, 5), (n_desc - 1, 7)]                  # (descriptor, KV head)
+    torch.cuda.synchronize()
+    states = [orc.gen_state(_slice_packed(caches[i], 0, hk), D) for i, hk in samples]
+    mk = lambda *shape: [torch.empty(shape, dtype=torch.bfloat16, device=DEV) for _ in range(n_desc)]
+    kn, vn, qs, outs = mk(1, Hkv, D), mk(1, Hkv, D), mk(1, wl.n_q_heads, D), mk(1, wl.n_q_heads, D)
+    gb = qp.GenBatch(qs, kn, vn, caches, tails, outs)
+    for st in range(steps):
+        # one stream of seeded rows per step, cut into the descriptors' tensors
+        rows = synth.normal_f32(wl.seed + 77, 0, 100 + st, n_desc * (2 * Hkv + wl.n_q_heads) * D, DEV) \
+            .view(n_desc, 2 * Hkv + wl.n_q_heads, D).to(torch.bfloat16)
+        for i in range(n_desc):
+            kn[i][0].copy_(rows[i, :Hkv]); vn[i][0].copy_(rows[i, Hkv:2 * Hkv]); qs[i][0].copy_(rows[i, 2 * Hkv:])
+        qp.append_kv_layers(gb)
+        qp.decode_attn_tail_layers(gb)
+        torch.cuda.synchronize()
+        flushed = (st + 1) // g
+        assert all(gb.cache_arr[i].n_keep == wl.n_keep(i % nl) + g * flushed for i in range(n_desc))
+        assert all(gb.tail_arr[i].n_tail == (st + 1) % g for i in range(n_desc))
+        assert all(bool(torch.isfinite(o.float()).all()) for o in outs)
+        for si, (i, hk) in enumerate(samples):
+            states[si] = orc.append(states[si], bits_u16(kn[i][:, hk:hk + 1]), bits_u16(vn[i][:, hk:hk + 1]))
+            if st in (0, g - 2, g - 1, g, steps - 1):
+                ref = orc.decode_state(bits_u16(qs[i][:, hk * G:(hk + 1) * G]), states[si], D)
+                got = outs[i][:, hk * G:(hk + 1) * G].float().cpu().numpy()
+                assert np.abs(got - ref).max() <= decode_tolerance(ref), (st, i, hk)
+    for si, (i, hk) in enumerate(samples):                        # the flushed group, bit for bit
+        d = gb.cache_arr[i]
+        n, c = d.n_keep, caches[i]
+        sl = lambda t, m: t[0:1, hk:hk + 1, :m].contiguous()
+        got = orc.Packed(d.bits, g, n, sl(c.k_codes, n // g).cpu().numpy().view(np.uint32),
+                         sl(c.v_codes, n).cpu().numpy().view(np.uint32), bits_u16(sl(c.k_scale, n // g)),
+                         bits_u16(sl(c.k_zero, n // g)), bits_u16(sl(c.v_scale, n)), bits_u16(sl(c.v_zero, n)))
+        assert_packed_equal(got, states[si].packed)
