@@ -113,6 +113,7 @@ struct DecTable {
   int chunk;        // chunked kernel: tokens per split
   int total_tiles;  // flat-range kernel: tiles of all layers and heads
   int n_workers;    // flat-range kernel: workers (blocks or warps, by kernel), each owning total_tiles / n_workers consecutive tiles
+  int wide;         // flat-range kernel: 1 = the build with more resident workers per SM (long ranges), see decode_plan
   DecLayer l[QP_MAX_LAYERS];
 };
 struct DecDims {
@@ -127,7 +128,10 @@ struct TailLayer {
 struct TailTable {
   TailLayer l[QP_MAX_LAYERS];
 };
-constexpr int kMaxDecodeWorkers = 2048;
+#ifndef QP_MAX_DECODE_WORKERS
+#define QP_MAX_DECODE_WORKERS 2432
+#endif
+constexpr int kMaxDecodeWorkers = QP_MAX_DECODE_WORKERS;
 // Chooses the decomposition for the layers in tab (n and pointers already set), fills chunk / part_base or
 // tile_base / total_tiles / n_workers and returns the bytes of partial records the launch needs.
 size_t decode_plan(DecTable& tab, const DecDims& d);
@@ -154,6 +158,7 @@ int sm_count();   // SMs of the current device (cached)
 bool decode_mma_supported(const DecDims& d);
 int decode_mma_workers_per_sm(const DecDims& d);     // workers (see DecTable::n_workers) resident per SM
 int decode_mma_tiles_per_worker_min(const DecDims& d);   // small launches use fewer workers, not emptier ones
+int decode_mma_wide_workers_per_sm(const DecDims& d, int* min_tiles);
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
                               bool overlap_prev, const TailTable* tails = nullptr);
 

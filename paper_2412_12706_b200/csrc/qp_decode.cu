@@ -230,6 +230,13 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
       T += (long long)BH * ((tab.l[l].n + 31) / 32);
     }
     long long W = (long long)sm_count() * decode_mma_workers_per_sm(d);
+    tab.wide = 0;
+    int wide_min = 0;
+    const long long Ww = (long long)sm_count() * decode_mma_wide_workers_per_sm(d, &wide_min);
+    if (Ww > 0 && Ww <= kMaxDecodeWorkers && T >= Ww * wide_min) {   // long ranges: more, narrower workers
+      W = Ww;
+      tab.wide = 1;
+    }
     if (W > kMaxDecodeWorkers) W = kMaxDecodeWorkers;
     const int tmin = decode_mma_tiles_per_worker_min(d);        // at least one tile per warp
     if (W > (T + tmin - 1) / tmin) W = (T + tmin - 1) / tmin;
@@ -243,7 +250,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
   long long total_tokens = 0;
   for (int l = 0; l < tab.n_layers; ++l) total_tokens += (long long)BH * tab.l[l].n;
   tab.chunk = chunk_tokens(total_tokens);
-  tab.total_tiles = tab.n_workers = 0;
+  tab.total_tiles = tab.n_workers = tab.wide = 0;
   size_t slots = 0;
   for (int l = 0; l < tab.n_layers; ++l) {
     tab.l[l].part_base = (int)slots;

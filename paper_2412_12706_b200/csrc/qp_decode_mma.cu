@@ -33,15 +33,18 @@ namespace qp {
 
 namespace {
 
-constexpr int DM_WARPS = 4;
+#ifndef QP_DM_WARPS
+#define QP_DM_WARPS 4
+#endif
+constexpr int DM_WARPS = QP_DM_WARPS;
 constexpr int DM_THREADS = DM_WARPS * 32;
-#ifndef QP_DM_STAGES
-#define QP_DM_STAGES 3
-#endif
-#ifndef QP_DM_MINB
-#define QP_DM_MINB 3
-#endif
-constexpr int DM_STAGES = QP_DM_STAGES;
+// Two builds of the kernel.  "Deep": three copy stages, three blocks (12 warps) per SM: a warp keeps two tiles in
+// flight, which is what short ranges need (a worker with a handful of tiles is bound by the latency of its own
+// copies).  "Wide": two stages, four blocks (16 warps) per SM and at most 128 registers: with long ranges the
+// extra warps fill more issue slots than the shallower ring loses (measured: +4 % on 336 MB launches, -30 % on
+// 84 MB ones), so the launch picks by tiles per worker.
+constexpr int DM_DEEP_STAGES = 3, DM_DEEP_MINB = 3, DM_WIDE_STAGES = 2, DM_WIDE_MINB = 4;
+constexpr int DM_WIDE_MIN_TILES = 20;    // tiles per worker from which the wide build is used
 constexpr int SP_STRIDE = 80;            // bytes per column of the per-warp P buffer (8 columns)
 constexpr int SP_BYTES = 8 * SP_STRIDE;
 
@@ -64,8 +67,8 @@ constexpr uint32_t M0 = 0x000f000fu;   // code in bits 0..3 of each half: value 
 constexpr uint32_t M1 = 0x00f000f0u;   // code in bits 4..7 of each half: value c * 2^-20
 constexpr float C24 = 16777216.0f, C20 = 1048576.0f;
 
-template <int D, int GROUP>
-__global__ void __launch_bounds__(DM_THREADS, QP_DM_MINB)
+template <int D, int GROUP, int DM_STAGES, int DM_MINB>
+__global__ void __launch_bounds__(DM_THREADS, DM_MINB)
 decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials) {
   using TL = Tile4<D>;
   constexpr int NC = D / 32;       // ldmatrix.x4 calls over the channels of a key tile = value groups per token
@@ -456,8 +459,8 @@ decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, c
   }
 }
 
-template <int D>
-constexpr size_t mma4_smem_bytes() { return (size_t)DM_WARPS * (DM_STAGES * Tile4<D>::BYTES + SP_BYTES); }
+template <int D, int STAGES>
+constexpr size_t mma4_smem_bytes() { return (size_t)DM_WARPS * (STAGES * Tile4<D>::BYTES + SP_BYTES); }
 
 }  // namespace
 
@@ -470,22 +473,34 @@ bool decode_mma_supported(const DecDims& d) {
 
 // The quantized kernels' workers are warps; the 16-bit kernel's workers are blocks of four warps.
 int decode_mma_workers_per_sm(const DecDims& d) {
-  return d.bits == 4 ? QP_DM_MINB * DM_WARPS : d.bits == 8 ? decode_mma8_blocks_per_sm() * decode_mma8_warps()
+  return d.bits == 4 ? DM_DEEP_MINB * DM_WARPS : d.bits == 8 ? decode_mma8_blocks_per_sm() * decode_mma8_warps()
          : d.bits == 16 ? decode_mma16_blocks_per_sm() : decode_mma2_workers_per_sm();
 }
 // Small launches: four tiles per worker at least (a 4-bit worker is one warp, the others four warps with a tile
 // each); more, smaller records per head cost the merge kernel more than the attention kernel gains.
 int decode_mma_tiles_per_worker_min(const DecDims&) { return 4; }
+// Workers per SM of the wider build of this shape's kernel and the tiles per worker from which it pays
+// (0: the shape has one build only).
+int decode_mma_wide_workers_per_sm(const DecDims& d, int* min_tiles) {
+  if (d.bits != 4) return 0;
+  *min_tiles = DM_WIDE_MIN_TILES;
+  return DM_WIDE_MINB * DM_WARPS;
+}
 
 namespace {
+template <int D, int GROUP, int STAGES, int MINB>
+cudaError_t launch_mma4_build(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev) {
+  constexpr size_t smem = mma4_smem_bytes<D, STAGES>();
+  static unsigned char done[64] = {};
+  const cudaError_t e = allow_smem(decode_mma4_kernel<D, GROUP, STAGES, MINB>, smem, done);
+  if (e != cudaSuccess) return e;
+  return launch_attention(decode_mma4_kernel<D, GROUP, STAGES, MINB>, (tab.n_workers + DM_WARPS - 1) / DM_WARPS,
+                          DM_THREADS, smem, st, overlap_prev, tab, d, partials);
+}
 template <int D, int GROUP>
 cudaError_t launch_mma4(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev) {
-  constexpr size_t smem = mma4_smem_bytes<D>();
-  static unsigned char done[64] = {};
-  const cudaError_t e = allow_smem(decode_mma4_kernel<D, GROUP>, smem, done);
-  if (e != cudaSuccess) return e;
-  return launch_attention(decode_mma4_kernel<D, GROUP>, (tab.n_workers + DM_WARPS - 1) / DM_WARPS, DM_THREADS, smem, st,
-                          overlap_prev, tab, d, partials);
+  if (tab.wide) return launch_mma4_build<D, GROUP, DM_WIDE_STAGES, DM_WIDE_MINB>(tab, d, partials, st, overlap_prev);
+  return launch_mma4_build<D, GROUP, DM_DEEP_STAGES, DM_DEEP_MINB>(tab, d, partials, st, overlap_prev);
 }
 }  // namespace
 

@@ -118,8 +118,8 @@ def test_workspace_sizes():
     # (max, sum, acc[D]) records of G heads: the larger of one per 128-token split and one per
     # (KV head + worker block), the two decompositions the decode launch can choose from
     r256 = lambda x: (x + 255) // 256 * 256
-    # two areas of records (8 heads + 2048 workers) for alternate calls, or the chunked kernel's records
-    assert qp.decode_workspace_bytes(c) == max(8 * (2048 // 128) * 4 * 130 * 4, 2 * r256((8 + 2048) * 4 * 130 * 4))
+    # two areas of records (8 heads + 2432 workers) for alternate calls, or the chunked kernel's records
+    assert qp.decode_workspace_bytes(c) == max(8 * (2048 // 128) * 4 * 130 * 4, 2 * r256((8 + 2432) * 4 * 130 * 4))
 
 
 def test_bad_arguments_are_rejected_before_any_launch(lib):
