@@ -233,7 +233,9 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
     tab.wide = 0;
     int wide_min = 0;
     const long long Ww = (long long)sm_count() * decode_mma_wide_workers_per_sm(d, &wide_min);
-    if (Ww > 0 && Ww <= kMaxDecodeWorkers && T >= Ww * wide_min) {   // long ranges: more, narrower workers
+    const long long merge_blocks = ((long long)d.Bt * d.Hq * tab.n_layers + 3) / 4;
+    // long ranges and a merge grid too large to sit beside the attention blocks anyway: more, narrower workers
+    if (Ww > 0 && Ww <= kMaxDecodeWorkers && T >= Ww * wide_min && merge_blocks > 2 * sm_count()) {
       W = Ww;
       tab.wide = 1;
     }

@@ -41,8 +41,12 @@ constexpr int DM_THREADS = DM_WARPS * 32;
 // Two builds of the kernel.  "Deep": three copy stages, three blocks (12 warps) per SM: a warp keeps two tiles in
 // flight, which is what short ranges need (a worker with a handful of tiles is bound by the latency of its own
 // copies).  "Wide": two stages, four blocks (16 warps) per SM and at most 128 registers: with long ranges the
-// extra warps fill more issue slots than the shallower ring loses (measured: +4 % on 336 MB launches, -30 % on
-// 84 MB ones), so the launch picks by tiles per worker.
+// extra warps fill more issue slots than the shallower ring loses.  Measured, deep -> wide: 5.37 -> 5.60 TB/s on
+// 336 MB launches of 8k-context caches, 5.87 -> 6.02 TB/s on 336 MB launches of 128k-context caches, but
+// 20 -> 30 us on 84 MB launches, 5.11 -> 4.15 TB/s on a 168 MB launch whose merge grid is small enough to sit
+// beside the attention blocks (the wide build leaves it no registers), and 5.18 -> 5.06 TB/s with 8 query heads
+// per KV head.  The launch therefore takes the wide build only for 20 or more tiles per worker, at most 4 query
+// heads per KV head and a merge grid of the large kind; five blocks per SM (96 registers) were slower again.
 constexpr int DM_DEEP_STAGES = 3, DM_DEEP_MINB = 3, DM_WIDE_STAGES = 2, DM_WIDE_MINB = 4;
 constexpr int DM_WIDE_MIN_TILES = 20;    // tiles per worker from which the wide build is used
 constexpr int SP_STRIDE = 80;            // bytes per column of the per-warp P buffer (8 columns)
@@ -482,7 +486,7 @@ int decode_mma_tiles_per_worker_min(const DecDims&) { return 4; }
 // Workers per SM of the wider build of this shape's kernel and the tiles per worker from which it pays
 // (0: the shape has one build only).
 int decode_mma_wide_workers_per_sm(const DecDims& d, int* min_tiles) {
-  if (d.bits != 4) return 0;
+  if (d.bits != 4 || d.Hq / d.Hkv > 4) return 0;              // (with 8 query heads per KV head the deep build wins)
   *min_tiles = DM_WIDE_MIN_TILES;
   return DM_WIDE_MINB * DM_WARPS;
 }

@@ -135,10 +135,135 @@ topk_kernel(const float* __restrict__ scores, int L, int w, int n_keep, int32_t*
   }
 }
 
+// The same selection for P <= ITEMS * 1024 with the keys held in registers: the scores are read from memory once
+// (all loads in flight together) instead of five times, the four digit passes and the compaction run from
+// registers, and the ordered compaction needs one block-wide prefix over (chunk, warp) counts instead of one
+// per chunk.  Element j = q * 1024 + tid is item q of thread tid, so ascending position = (q, warp, lane) order.
+template <int ITEMS>
+__global__ void __launch_bounds__(TK_THREADS)
+topk_reg_kernel(const float* __restrict__ scores, int L, int w, int n_keep, int32_t* __restrict__ kept) {
+  const int P = L - w, k = n_keep - w;
+  const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* s = scores + (size_t)bh * P;
+  int32_t* out = kept + (size_t)bh * n_keep;
+
+  for (int i = tid; i < w; i += TK_THREADS) out[k + i] = P + i;   // window tokens are always kept
+  if (k >= P) {                                                    // keep everything
+    for (int j = tid; j < P; j += TK_THREADS) out[j] = j;
+    return;
+  }
+
+  __shared__ unsigned hist[256];
+  __shared__ unsigned sh_prefix, sh_need;
+  __shared__ unsigned cnt_g[ITEMS][32], cnt_e[ITEMS][32];        // per (chunk, warp): counts, then exclusive prefixes
+  __shared__ unsigned row_g[ITEMS], row_e[ITEMS];                // per chunk: totals, then exclusive prefixes
+
+  uint32_t key[ITEMS];                                           // order-preserving images; valid where j < P
+#pragma unroll
+  for (int q = 0; q < ITEMS; ++q) {
+    const int j = q * TK_THREADS + tid;
+    key[q] = order_key(j < P ? s[j] : 0.f);
+  }
+
+  unsigned prefix = 0, mask = 0, need = (unsigned)k;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < ITEMS; ++q) {
+      if (q * TK_THREADS >= P) break;
+      const bool cand = q * TK_THREADS + tid < P && (key[q] & mask) == prefix;
+      const unsigned digit = (key[q] >> shift) & 255u;
+      if (shift >= 16) {                                         // crowded digits: one atomic per distinct digit and warp
+        const unsigned peers = __match_any_sync(0xffffffffu, cand ? digit : 256u + lane);
+        if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+      } else if (cand) {
+        atomicAdd(&hist[digit], 1u);
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane l owns bins 8l .. 8l+7; find the bin where the count from the top reaches `need`
+      unsigned c[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = hist[8 * lane + i]; tot += c[i]; }
+      unsigned suf = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned v = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += v;
+      }
+      const unsigned above = suf - tot;
+      if (above < need && suf >= need) {                         // exactly one lane
+        unsigned cum = above;
+        int bsel = 7;
+        for (; bsel > 0; --bsel) {
+          if (cum + c[bsel] >= need) break;
+          cum += c[bsel];
+        }
+        sh_need = need - cum;
+        sh_prefix = prefix | ((unsigned)(8 * lane + bsel) << shift);
+      }
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    need = sh_need;
+    mask |= 0xffu << shift;
+  }
+  const uint32_t T = prefix;   // image of the k-th largest score; `need` elements equal to it are kept
+
+  // ---- ordered compaction: counts per (chunk, warp), one block-wide exclusive prefix, then the writes
+#pragma unroll
+  for (int q = 0; q < ITEMS; ++q) {
+    const bool in = q * TK_THREADS + tid < P;
+    const unsigned bg = __ballot_sync(0xffffffffu, in && key[q] > T), be = __ballot_sync(0xffffffffu, in && key[q] == T);
+    if (lane == 0) { cnt_g[q][warp] = __popc(bg); cnt_e[q][warp] = __popc(be); }
+  }
+  __syncthreads();
+  for (int q = warp; q < ITEMS; q += 32) {                       // warp q scans chunk q's 32 warp counts
+    const unsigned wg = cnt_g[q][lane], we = cnt_e[q][lane];
+    unsigned sg = wg, se = we;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned vg = __shfl_up_sync(0xffffffffu, sg, o), ve = __shfl_up_sync(0xffffffffu, se, o);
+      if (lane >= o) { sg += vg; se += ve; }
+    }
+    cnt_g[q][lane] = sg - wg;
+    cnt_e[q][lane] = se - we;
+    if (lane == 31) { row_g[q] = sg; row_e[q] = se; }
+  }
+  __syncthreads();
+  if (warp == 0) {                                               // exclusive prefix of the chunk totals (ITEMS <= 32)
+    const unsigned wg = lane < ITEMS ? row_g[lane] : 0u, we = lane < ITEMS ? row_e[lane] : 0u;
+    unsigned sg = wg, se = we;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned vg = __shfl_up_sync(0xffffffffu, sg, o), ve = __shfl_up_sync(0xffffffffu, se, o);
+      if (lane >= o) { sg += vg; se += ve; }
+    }
+    if (lane < ITEMS) { row_g[lane] = sg - wg; row_e[lane] = se - we; }
+  }
+  __syncthreads();
+  const unsigned lt_mask = (1u << lane) - 1u;
+#pragma unroll
+  for (int q = 0; q < ITEMS; ++q) {
+    if (q * TK_THREADS >= P) break;
+    const int j = q * TK_THREADS + tid;
+    const bool gt = j < P && key[q] > T, eq = j < P && key[q] == T;
+    const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+    const unsigned pg = row_g[q] + cnt_g[q][warp] + __popc(bg & lt_mask);
+    const unsigned pe = row_e[q] + cnt_e[q][warp] + __popc(be & lt_mask);
+    if (gt || (eq && pe < need)) out[pg + min(pe, need)] = j;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_keep, int32_t* kept, cudaStream_t st) {
-  topk_kernel<<<BH, TK_THREADS, 0, st>>>(scores, L, w, n_keep, kept);
+  const int P = L - w;
+  if (P <= 8 * TK_THREADS) topk_reg_kernel<8><<<BH, TK_THREADS, 0, st>>>(scores, L, w, n_keep, kept);
+  else if (P <= 32 * TK_THREADS) topk_reg_kernel<32><<<BH, TK_THREADS, 0, st>>>(scores, L, w, n_keep, kept);
+  else topk_kernel<<<BH, TK_THREADS, 0, st>>>(scores, L, w, n_keep, kept);
   return cudaGetLastError();
 }
 
