@@ -241,6 +241,15 @@ def run_gpu(args, wl):
                 qp.compress_layer(sq["K"][l], sq["V"][l], sq["Qw"][l], wl.layer_budget_bits(l), wl.bits, wl.group,
                                   wl.pool, sq["cache"][l], sq["kept"][l], ws_c)
 
+    # the same work through qp_compress_layers: all layers of a sequence per call (one launch per stage)
+    ws_cl = torch.empty(qp.compress_workspace_bytes(Bt * n_layers, Hq, Hkv, D, L, w), dtype=torch.uint8, device=dev) \
+        if Bt * n_layers * Hkv <= 65535 and not args.no_compress_layers else None
+
+    def compress_all_layers():
+        budgets = [wl.layer_budget_bits(l) for l in range(n_layers)]
+        for sq in seqs:
+            qp.compress_layers(sq["K"], sq["V"], sq["Qw"], budgets, wl.bits, wl.group, wl.pool, sq["cache"], sq["kept"], ws_cl)
+
     def decode_all():
         # no event between the calls: consecutive decode calls overlap on the GPU (the next call's attention
         # kernel fills the SMs as this call's drains), and an event record in between would forbid that
@@ -276,6 +285,18 @@ def run_gpu(args, wl):
     comp_ms = sum(a.elapsed_time(b) for a, b, c in marks)
     dec_ms = sum(b.elapsed_time(c) for a, b, c in marks)
     call_ms = dec_ms / (args.steps * n_calls_step)      # average launch duration over the timed decode phases
+
+    # ---- compression with all layers of a sequence in one qp_compress_layers call
+    comp_layers_ms = None
+    if ws_cl is not None:
+        compress_all_layers()
+        k0, k1 = ev(), ev()
+        k0.record(stream)
+        for _ in range(3):
+            compress_all_layers()
+        k1.record(stream)
+        torch.cuda.synchronize()
+        comp_layers_ms = k0.elapsed_time(k1) / 3
 
     # ---- the same decode attention with one sequence per call (context for the batched figure)
     single_ms = None
@@ -417,6 +438,10 @@ def run_gpu(args, wl):
                          f"launches read different data; compress inputs {input_bytes / 1e9:.2f} GB"},
         "compress_tokens_per_s": world * ctx_tokens_step * steps / (comp_ms * 1e-3),
         "compress_ms_per_layer": comp_ms / (steps * n_seq * n_layers),
+        "compress_layers_call": None if comp_layers_ms is None else {
+            "note": f"qp_compress_layers: the {n_layers} layers of a sequence per call, one launch per stage",
+            "ms_per_layer": comp_layers_ms / (n_seq * n_layers),
+            "tokens_per_s": world * ctx_tokens_step / (comp_layers_ms * 1e-3)},
         "decode_us_per_call": call_ms * 1e3,
         "decode_single_sequence_call": None if single_ms is None else {
             "us_per_call": single_ms * 1e3, "GB/s": dec_bytes_call / per_call / (single_ms * 1e-3) / 1e9},
@@ -515,6 +540,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling: keep only the first N layers of the workload")
     ap.add_argument("--batch", type=int, default=0, help="profiling: override the workload's batch size")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-compress-layers", action="store_true", help="skip the qp_compress_layers figure")
     ap.add_argument("--no-generation", action="store_true", help="skip the append + decode generation-loop figure")
     ap.add_argument("--no-layer-chain", action="store_true", help="skip the layer-by-layer / CUDA-graph figures")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")

@@ -157,6 +157,22 @@ qp_status qp_compress_layer(const void* K, const void* V, const void* Q_win, int
                             void* stream);
 
 /*
+ * The same prefill-side path for n_layers independent layers of one shape (1 <= n_layers <=
+ * QP_MAX_LAYERS, batch * n_layers * n_kv_heads <= 65535) with one launch per stage instead of one per
+ * stage and layer: a layer of a short prompt leaves most of the GPU idle, several at once do not
+ * (layers of different sequences at the same depth, or a measurement over synthetic layers).
+ * K, V, Q_win, kept_idx are HOST arrays of device pointers, budget_bits a HOST array (budgets and so
+ * n_keep may differ per layer), caches a HOST array; shapes, bits, group and pool are shared.
+ * workspace: qp_compress_workspace_bytes(batch * n_layers, ...) bytes.  Results are identical, bit for
+ * bit, to n_layers calls of qp_compress_layer.
+ */
+qp_status qp_compress_layers(int n_layers, const void* const* K, const void* const* V, const void* const* Q_win,
+                             int batch, int n_q_heads, int n_kv_heads, int head_dim, int L, int w,
+                             const int64_t* budget_bits /* host */, int bits, int group, int pool,
+                             const qp_cache* caches /* host */, int32_t* const* kept_idx, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/*
  * S4 + S5, decode-step attention over the packed cache (Eq. 3 on the dequantized
  * cache of Eq. 5): out[b,h,:] = softmax_t(q[b,h].K'[t] / sqrt(D)) V' over the n kept
  * tokens of KV head h / G, no mask.  q, out bf16 [Bt,Hq,D] (device).  The token

@@ -258,6 +258,45 @@ qp_status qp_compress_layer(const void* K, const void* V, const void* Q_win, int
   return QP_OK;
 }
 
+qp_status qp_compress_layers(int n_layers, const void* const* K, const void* const* V, const void* const* Q_win,
+                             int batch, int n_q_heads, int n_kv_heads, int head_dim, int L, int w,
+                             const int64_t* budget_bits, int bits, int group, int pool, const qp_cache* caches,
+                             int32_t* const* kept_idx, void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !K || !V || !Q_win || !budget_bits || !caches || !kept_idx || !workspace)
+    return QP_ERR_INVALID_ARG;
+  int n_keep[QP_MAX_LAYERS];
+  for (int l = 0; l < n_layers; ++l) {
+    if (!V[l] || !kept_idx[l]) return QP_ERR_INVALID_ARG;
+    qp_status s = check_score_args(Q_win[l], K[l], batch, n_q_heads, n_kv_heads, head_dim, L, w, pool);
+    if (s != QP_OK) return s;
+    int32_t n = 0;
+    s = qp_n_keep(budget_bits[l], bits, group, L, w, &n);
+    if (s != QP_OK) return s;
+    s = check_cache(&caches[l], true);
+    if (s != QP_OK) return s;
+    const qp_cache& c = caches[l];
+    if (c.batch != batch || c.n_q_heads != n_q_heads || c.n_kv_heads != n_kv_heads || c.head_dim != head_dim ||
+        c.bits != bits || c.group != group)
+      return QP_ERR_INVALID_ARG;
+    if (c.n_keep != n) return QP_ERR_BUDGET;
+    if (!aligned16(V[l])) return QP_ERR_ALIGNMENT;
+    n_keep[l] = n;
+  }
+  if (!aligned16(workspace)) return QP_ERR_ALIGNMENT;
+  if ((long long)batch * n_layers * n_kv_heads > 65535) return QP_ERR_UNSUPPORTED;   // one grid dimension holds them
+  const ScoreWorkspace sw = score_workspace(batch * n_layers, n_q_heads, n_kv_heads, L, w);
+  if (workspace_bytes < sw.total) return QP_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cache_written(st);
+  float* pooled = reinterpret_cast<float*>(static_cast<char*>(workspace) + sw.pooled);
+  const ScoreDims d{batch, n_q_heads, n_kv_heads, head_dim, L, w, pool};
+  if (launch_window_scores_layers(n_layers, Q_win, K, d, pooled, workspace, st) != cudaSuccess) return QP_ERR_CUDA;
+  if (launch_select_topk_layers(n_layers, pooled, batch * n_kv_heads, L, w, n_keep, kept_idx, st) != cudaSuccess)
+    return QP_ERR_CUDA;
+  if (launch_gather_quantize_layers(n_layers, K, V, kept_idx, L, caches, st) != cudaSuccess) return QP_ERR_CUDA;
+  return QP_OK;
+}
+
 qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const qp_cache* caches, const qp_tail* tails,
                                      void* const* out, void* workspace, size_t workspace_bytes, void* stream) {
   if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !q || !caches || !out || !workspace) return QP_ERR_INVALID_ARG;

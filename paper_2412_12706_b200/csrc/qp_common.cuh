@@ -72,17 +72,33 @@ struct ScoreWorkspace {
 ScoreWorkspace score_workspace(int Bt, int Hq, int Hkv, int L, int w);
 cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDims& d, float* scores, void* ws,
                                  cudaStream_t st);
+// The same for n_layers layers of one shape in one sequence of launches: the layers are stacked along the batch
+// dimension of the scratch arrays (ws: score_workspace(Bt * n_layers, ...)) and of scores [n_layers, Bt, Hkv, P].
+cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, const void* const* K, const ScoreDims& d,
+                                        float* scores, void* ws, cudaStream_t st);
+// per-layer inputs of the score sweeps, passed by value
+template <int NL>
+struct ScorePtrs {
+  const bf16* q[NL];
+  const bf16* k[NL];
+};
 
 // tcgen05 / TMEM form of the two score sweeps (same outputs as score_sweep_kernel)
 bool score_tc_supported(int D);
-cudaError_t launch_score_sweep_tc(int pass, const bf16* q, const bf16* k, const ScoreDims& d, const ScoreWorkspace& s,
-                                  float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
-                                  int* error_word, cudaStream_t st);
+cudaError_t launch_score_sweep_tc(int pass, int n_layers, const void* const* q, const void* const* k, const ScoreDims& d,
+                                  const ScoreWorkspace& s, float scale_log2, float2* stat_partial, const float2* rowstat,
+                                  float* votes_partial, int* error_word, cudaStream_t st);
 
 cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_keep, int32_t* kept, cudaStream_t st);
+// n_layers layers in one launch: scores [n_layers, BH, P]; kept[l] int32 [BH, n_keep[l]]
+cudaError_t launch_select_topk_layers(int n_layers, const float* scores, int BH, int L, int w, const int* n_keep,
+                                      int32_t* const* kept, cudaStream_t st);
 
 cudaError_t launch_gather_quantize(const void* K, const void* V, const int32_t* kept, int L, const qp_cache& c,
                                    cudaStream_t st);
+// n_layers caches of one shape (n_keep may differ) in one launch; kept[l] int32 [BH, caches[l].n_keep]
+cudaError_t launch_gather_quantize_layers(int n_layers, const void* const* K, const void* const* V,
+                                          const int32_t* const* kept, int L, const qp_cache* caches, cudaStream_t st);
 // tokens per (batch, KV head) the arrays of c are sized for
 inline int cache_capacity(const qp_cache& c) { return c.n_cap > 0 ? c.n_cap : c.n_keep; }
 

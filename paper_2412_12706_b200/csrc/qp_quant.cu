@@ -7,6 +7,8 @@
 // handled one group per thread straight from global memory.
 // Arithmetic is fp32 with explicit round-to-nearest intrinsics (no FMA contraction) so that
 // codes, scales and zeros are reproducible bit for bit.
+#include <algorithm>
+
 #include "qp_common.cuh"
 
 namespace qp {
@@ -65,6 +67,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __shared__ int sidx[128];
   constexpr int QMAX = (1 << BITS) - 1, PER = 32 / BITS;
   const QuantLayer& ql = tab.l[blockIdx.z];
+  if ((int)blockIdx.x * g >= ql.n_idx) return;     // layers of one launch may keep different numbers of tokens
   const uint16_t* __restrict__ K = ql.K;
   const uint16_t* __restrict__ V = ql.V;
   const int32_t* __restrict__ kept = ql.kept;
@@ -234,6 +237,30 @@ cudaError_t launch_gather_quantize(const void* K, const void* V, const int32_t* 
                         static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
                         static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, n, ns, 0};
   return launch_quant_table<1>(c.bits, tab, dim3(n / g, BH, 1), D, g, st);
+}
+
+cudaError_t launch_gather_quantize_layers(int n_layers, const void* const* K, const void* const* V,
+                                          const int32_t* const* kept, int L, const qp_cache* caches, cudaStream_t st) {
+  const qp_cache& c0 = caches[0];
+  if (n_layers == 1 || c0.bits == 16) {            // plain row gathers: one launch per layer
+    for (int l = 0; l < n_layers; ++l) {
+      const cudaError_t e = launch_gather_quantize(K[l], V[l], kept[l], L, caches[l], st);
+      if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+  }
+  QuantTable<QP_MAX_LAYERS> tab;
+  int max_groups = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const qp_cache& c = caches[l];
+    tab.l[l] = QuantLayer{static_cast<const uint16_t*>(K[l]), static_cast<const uint16_t*>(V[l]), kept[l],
+                          static_cast<uint32_t*>(c.k_codes), static_cast<uint32_t*>(c.v_codes),
+                          static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
+                          static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, c.n_keep, cache_capacity(c), 0};
+    max_groups = std::max(max_groups, c.n_keep / c.group);
+  }
+  return launch_quant_table<QP_MAX_LAYERS>(c0.bits, tab, dim3(max_groups, c0.batch * c0.n_kv_heads, n_layers),
+                                           c0.head_dim, c0.group, st);
 }
 
 cudaError_t launch_append_rows(int n_layers, const void* const* k_new, const void* const* v_new, const qp_cache* caches,

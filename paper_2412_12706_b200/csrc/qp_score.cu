@@ -89,31 +89,34 @@ ScoreWorkspace score_workspace(int Bt, int Hq, int Hkv, int L, int w) {
   return s;
 }
 
-cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDims& d, float* scores, void* ws,
-                                 cudaStream_t st) {
-  const ScoreWorkspace s = score_workspace(d.Bt, d.Hq, d.Hkv, d.L, d.w);
-  const int BH = d.Bt * d.Hkv, P = d.L - d.w, R = (d.Hq / d.Hkv) * d.w;
+cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, const void* const* K, const ScoreDims& d,
+                                        float* scores, void* ws, cudaStream_t st) {
+  const ScoreWorkspace s = score_workspace(d.Bt * n_layers, d.Hq, d.Hkv, d.L, d.w);
+  const int BH = d.Bt * d.Hkv * n_layers, P = d.L - d.w, R = (d.Hq / d.Hkv) * d.w;
   char* base = static_cast<char*>(ws);
   float2* stat_partial = reinterpret_cast<float2*>(base + s.stat_partial);
   float2* rowstat = reinterpret_cast<float2*>(base + s.rowstat);
   float* votes_partial = reinterpret_cast<float*>(base + s.votes_partial);
   const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)d.D));
-  const bf16* q = static_cast<const bf16*>(Qwin);
-  const bf16* k = static_cast<const bf16*>(K);
-  if (score_tc_supported(d.D)) {
-    // 5th-generation tensor-core path; the word at s.error becomes 1 if a block ever gave up on a wait
-    int* err = reinterpret_cast<int*>(base + s.error);
-    cudaError_t e = cudaMemsetAsync(err, 0, sizeof(int), st);
-    if (e != cudaSuccess) return e;
-    e = launch_score_sweep_tc(1, q, k, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st);
-    if (e != cudaSuccess) return e;
-    rowstat_merge_kernel<<<BH * s.n_rb, SC_RB * RM_SLICES, 0, st>>>(stat_partial, s.n_rb, 2 * s.n_tiles, R, rowstat);
-    e = launch_score_sweep_tc(2, q, k, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st);
-    if (e != cudaSuccess) return e;
-    pool_kernel<<<dim3((P + 255) / 256, BH), 256, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);
-    return cudaGetLastError();
-  }
-  return cudaErrorInvalidValue;   // head dimensions other than 64 and 128 are rejected before this point
+  if (!score_tc_supported(d.D)) return cudaErrorInvalidValue;   // other head dimensions are rejected before this point
+  // 5th-generation tensor-core path; the word at s.error becomes 1 if a block ever gave up on a wait
+  int* err = reinterpret_cast<int*>(base + s.error);
+  cudaError_t e = cudaMemsetAsync(err, 0, sizeof(int), st);
+  if (e != cudaSuccess) return e;
+  e = launch_score_sweep_tc(1, n_layers, Qwin, K, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st);
+  if (e != cudaSuccess) return e;
+  rowstat_merge_kernel<<<BH * s.n_rb, SC_RB * RM_SLICES, 0, st>>>(stat_partial, s.n_rb, 2 * s.n_tiles, R, rowstat);
+  e = launch_score_sweep_tc(2, n_layers, Qwin, K, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st);
+  if (e != cudaSuccess) return e;
+  pool_kernel<<<dim3((P + 255) / 256, BH), 256, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDims& d, float* scores, void* ws,
+                                 cudaStream_t st) {
+  const void* qs[1] = {Qwin};
+  const void* ks[1] = {K};
+  return launch_window_scores_layers(1, qs, ks, d, scores, ws, st);
 }
 
 }  // namespace qp

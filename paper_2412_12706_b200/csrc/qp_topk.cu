@@ -14,18 +14,28 @@ namespace {
 constexpr int TK_THREADS = 1024;
 constexpr int TK_UNROLL = 8;
 
+// Outputs of the layers of one launch: block (layer, bh) reads scores[(layer * BH + bh) * P ..] and writes
+// kept[layer][bh * n_keep[layer] ..].
+template <int NL>
+struct TopkOut {
+  int32_t* kept[NL];
+  int n_keep[NL];
+};
+
 // monotone map float -> uint32 (larger float = larger integer); -0 is treated as +0
 __device__ __forceinline__ uint32_t order_key(float f) {
   const uint32_t u = __float_as_uint(f + 0.0f);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+template <int NL>
 __global__ void __launch_bounds__(TK_THREADS)
-topk_kernel(const float* __restrict__ scores, int L, int w, int n_keep, int32_t* __restrict__ kept) {
+topk_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid_constant__ TopkOut<NL> o) {
+  const int layer = blockIdx.x / BH, n_keep = o.n_keep[layer];
   const int P = L - w, k = n_keep - w;
-  const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* s = scores + (size_t)bh * P;
-  int32_t* out = kept + (size_t)bh * n_keep;
+  const int bh = blockIdx.x % BH, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* s = scores + (size_t)blockIdx.x * P;
+  int32_t* out = o.kept[layer] + (size_t)bh * n_keep;
 
   for (int i = tid; i < w; i += TK_THREADS) out[k + i] = P + i;   // window tokens are always kept
   if (k >= P) {                                                    // keep everything
@@ -139,13 +149,14 @@ topk_kernel(const float* __restrict__ scores, int L, int w, int n_keep, int32_t*
 // (all loads in flight together) instead of five times, the four digit passes and the compaction run from
 // registers, and the ordered compaction needs one block-wide prefix over (chunk, warp) counts instead of one
 // per chunk.  Element j = q * 1024 + tid is item q of thread tid, so ascending position = (q, warp, lane) order.
-template <int ITEMS>
+template <int ITEMS, int NL>
 __global__ void __launch_bounds__(TK_THREADS)
-topk_reg_kernel(const float* __restrict__ scores, int L, int w, int n_keep, int32_t* __restrict__ kept) {
+topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid_constant__ TopkOut<NL> o) {
+  const int layer = blockIdx.x / BH, n_keep = o.n_keep[layer];
   const int P = L - w, k = n_keep - w;
-  const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* s = scores + (size_t)bh * P;
-  int32_t* out = kept + (size_t)bh * n_keep;
+  const int bh = blockIdx.x % BH, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* s = scores + (size_t)blockIdx.x * P;
+  int32_t* out = o.kept[layer] + (size_t)bh * n_keep;
 
   for (int i = tid; i < w; i += TK_THREADS) out[k + i] = P + i;   // window tokens are always kept
   if (k >= P) {                                                    // keep everything
@@ -259,12 +270,33 @@ topk_reg_kernel(const float* __restrict__ scores, int L, int w, int n_keep, int3
 
 }  // namespace
 
-cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_keep, int32_t* kept, cudaStream_t st) {
+namespace {
+template <int NL>
+cudaError_t launch_topk(const float* scores, int blocks, int BH, int L, int w, const TopkOut<NL>& o, cudaStream_t st) {
   const int P = L - w;
-  if (P <= 8 * TK_THREADS) topk_reg_kernel<8><<<BH, TK_THREADS, 0, st>>>(scores, L, w, n_keep, kept);
-  else if (P <= 32 * TK_THREADS) topk_reg_kernel<32><<<BH, TK_THREADS, 0, st>>>(scores, L, w, n_keep, kept);
-  else topk_kernel<<<BH, TK_THREADS, 0, st>>>(scores, L, w, n_keep, kept);
+  if (P <= 8 * TK_THREADS) topk_reg_kernel<8, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
+  else if (P <= 32 * TK_THREADS) topk_reg_kernel<32, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
+  else topk_kernel<NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
   return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_keep, int32_t* kept, cudaStream_t st) {
+  TopkOut<1> o;
+  o.kept[0] = kept;
+  o.n_keep[0] = n_keep;
+  return launch_topk<1>(scores, BH, BH, L, w, o, st);
+}
+
+cudaError_t launch_select_topk_layers(int n_layers, const float* scores, int BH, int L, int w, const int* n_keep,
+                                      int32_t* const* kept, cudaStream_t st) {
+  if (n_layers == 1) return launch_select_topk(scores, BH, L, w, n_keep[0], kept[0], st);
+  TopkOut<QP_MAX_LAYERS> o;
+  for (int l = 0; l < n_layers; ++l) {
+    o.kept[l] = kept[l];
+    o.n_keep[l] = n_keep[l];
+  }
+  return launch_topk<QP_MAX_LAYERS>(scores, n_layers * BH, BH, L, w, o, st);
 }
 
 }  // namespace qp

@@ -25,7 +25,7 @@ EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_work
            "qp_decode_workspace_bytes", "qp_window_scores", "qp_select_topk", "qp_gather_quantize",
            "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static",
            "qp_cache_layout_cap", "qp_append_kv", "qp_append_kv_layers", "qp_decode_attn_tail",
-           "qp_decode_attn_tail_layers"]
+           "qp_decode_attn_tail_layers", "qp_compress_layers"]
 
 
 class QpError(RuntimeError):
@@ -88,6 +88,9 @@ def lib() -> ctypes.CDLL:
         L.qp_decode_attn_static.restype = i
         L.qp_decode_attn_static.argtypes = [p, cp, p, p]
         tp = ctypes.POINTER(qp_tail)
+        L.qp_compress_layers.restype = i
+        L.qp_compress_layers.argtypes = [i, ctypes.POINTER(p), ctypes.POINTER(p), ctypes.POINTER(p), i, i, i, i, i, i,
+                                         ctypes.POINTER(i64), i, i, i, cp, ctypes.POINTER(p), p, sz, p]
         L.qp_cache_layout_cap.restype = i
         L.qp_cache_layout_cap.argtypes = [i, i, i, i, i, i, i, i, cp]
         L.qp_append_kv.restype = i
@@ -256,6 +259,32 @@ def compress_layer(K: torch.Tensor, V: torch.Tensor, Q_win: torch.Tensor, budget
     return cache, kept_idx
 
 
+def compress_layers(Ks: list[torch.Tensor], Vs: list[torch.Tensor], Q_wins: list[torch.Tensor], budget_bits: list[int],
+                    bits: int, group: int = 32, pool: int = 7, caches: list[Cache] | None = None,
+                    kept_idx: list[torch.Tensor] | None = None, workspace: torch.Tensor | None = None):
+    """qp_compress_layers: the prefill-side path of several layers of one shape, one launch per stage.
+    Returns (caches, kept_idx); buffers are allocated with torch when not given."""
+    nl = len(Ks)
+    assert 1 <= nl <= QP_MAX_LAYERS and len(Vs) == nl and len(Q_wins) == nl and len(budget_bits) == nl
+    for t in (*Ks, *Vs, *Q_wins):
+        _dev_bf16(t)
+    Bt, Hq, Hkv, D, L, w = _dims(Ks[0], Q_wins[0])
+    ns = [n_keep(b, bits, group, L, w) for b in budget_bits]
+    dev = Ks[0].device
+    if caches is None:
+        caches = [alloc_cache(Bt, Hq, Hkv, D, bits, group, n, dev) for n in ns]
+    if kept_idx is None:
+        kept_idx = [torch.empty((Bt, Hkv, n), dtype=torch.int32, device=dev) for n in ns]
+    if workspace is None:
+        workspace = torch.empty(max(16, compress_workspace_bytes(Bt * nl, Hq, Hkv, D, L, w)), dtype=torch.uint8, device=dev)
+    arr = lambda ts: (ctypes.c_void_p * nl)(*[t.data_ptr() for t in ts])
+    _check(lib().qp_compress_layers(nl, arr(Ks), arr(Vs), arr(Q_wins), Bt, Hq, Hkv, D, L, w,
+                                    (ctypes.c_int64 * nl)(*budget_bits), bits, group, pool,
+                                    (qp_cache * nl)(*[c.desc for c in caches]), arr(kept_idx), _ptr(workspace),
+                                    workspace.numel(), _stream()), "qp_compress_layers")
+    return caches, kept_idx
+
+
 def new_decode_workspace(nbytes: int, device) -> torch.Tensor:
     """Scratch for the decode calls (contents irrelevant); reuse one per stream across calls."""
     return torch.empty(max(16, nbytes), dtype=torch.uint8, device=device)
@@ -397,6 +426,7 @@ qp_window_scores = window_scores
 qp_select_topk = select_topk
 qp_gather_quantize = gather_quantize
 qp_compress_layer = compress_layer
+qp_compress_layers = compress_layers
 qp_decode_attn = decode_attn
 qp_decode_attn_layers = decode_attn_layers
 qp_decode_attn_static = decode_attn_static

@@ -225,3 +225,27 @@ def test_compress_keep_all_16bit_equals_dense_attention():
         p = np.exp(a - a.max()); p /= p.sum()
         ref = p @ V[0, h // G]
         assert np.abs(out[0, h] - ref).max() <= 2e-3 + 2.0 ** -8 * np.abs(ref).max()
+
+
+# ------------------------------------------------------------------ qp_compress_layers: many layers per launch
+
+@pytest.mark.parametrize("bits,D,L,w", [(4, 128, 1100, 32), (2, 64, 777, 8), (16, 128, 600, 64), (8, 128, 40000, 32)])
+def test_compress_layers_is_bit_identical_to_per_layer_calls(bits, D, L, w):
+    """Five layers with different budgets in one qp_compress_layers call: kept indices and every packed
+    byte equal those of five qp_compress_layer calls (which the other tests check against the oracle)."""
+    nl, group = 5, 32
+    wl = small(synth.TINY, head_dim=D, n_q_heads=8, n_kv_heads=2, L=L, w=w, batch=2, bits=bits, group=group)
+    Ks, Vs, Qs = [], [], []
+    for l in range(nl):
+        k, v, qw = make_inputs(wl, l)
+        Ks.append(k.to(DEV)); Vs.append(v.to(DEV)); Qs.append(qw.to(DEV))
+    budgets = [bits * (w + 32 * (l + 1) + (0 if bits < 16 else 5)) for l in range(nl)]
+    if bits < 16:
+        budgets = [bits * ((w + 31) // 32 * 32 + 32 * (l + 1)) for l in range(nl)]
+    caches, kepts = qp.compress_layers(Ks, Vs, Qs, budgets, bits, group, wl.pool)
+    torch.cuda.synchronize()
+    for l in range(nl):
+        ref_c, ref_k = qp.compress_layer(Ks[l], Vs[l], Qs[l], budgets[l], bits, group, wl.pool)
+        torch.cuda.synchronize()
+        assert torch.equal(kepts[l], ref_k), l
+        assert_packed_equal(cache_to_packed(caches[l]), cache_to_packed(ref_c))
