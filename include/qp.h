@@ -191,7 +191,10 @@ qp_status qp_decode_attn(const void* q, const qp_cache* cache /* host */, void* 
  * The same decode attention for n_layers independent layers in one pair of
  * launches (1 <= n_layers <= QP_MAX_LAYERS).  q, caches, out are HOST arrays of
  * length n_layers; q[l], out[l] are device pointers.  All caches must agree in
- * batch, heads, head_dim, bits and group; n_keep may differ per layer.
+ * batch, heads and head_dim; n_keep may differ per layer.  bits and group may differ too
+ * (the per-layer token/precision mixes of Sec. 5.4: some layers at 4 bit with 4x the tokens,
+ * others at 8 or 16 bit): layers of equal (bits, group) then share a launch pair and the
+ * classes run one after the other, results as for separate calls.
  */
 qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches,
                                 void* const* out, void* workspace, size_t workspace_bytes, void* stream);

@@ -297,8 +297,14 @@ qp_status qp_compress_layers(int n_layers, const void* const* K, const void* con
   return QP_OK;
 }
 
-qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const qp_cache* caches, const qp_tail* tails,
-                                     void* const* out, void* workspace, size_t workspace_bytes, void* stream) {
+}  // extern "C"
+
+namespace {
+// Decode attention over layers that agree in bits and group.  check_only: validate everything (workspace size
+// included) and return before anything is launched or recorded.
+qp_status decode_layers_uniform(int n_layers, const void* const* q, const qp_cache* caches, const qp_tail* tails,
+                                void* const* out, void* workspace, size_t workspace_bytes, void* stream,
+                                bool check_only) {
   if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !q || !caches || !out || !workspace) return QP_ERR_INVALID_ARG;
   if (!aligned16(workspace)) return QP_ERR_ALIGNMENT;
   const qp_cache& c0 = caches[0];
@@ -335,6 +341,7 @@ qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const q
     for (int l = 0; l < n_layers; ++l) ttab.l[l] = TailLayer{tails[l].k_tail, tails[l].v_tail, tails[l].n_tail, 0};
   const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
   if (workspace_bytes < decode_plan(tab, d)) return QP_ERR_WORKSPACE;
+  if (check_only) return QP_OK;
   // everything the attention kernel reads before it waits for the stream's previous kernel, and what this
   // call's merge kernel writes
   std::vector<PrevOutputs::Range> reads, writes;
@@ -361,6 +368,43 @@ qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const q
   return launch_decode(tab, d, workspace, dec.parity, static_cast<cudaStream_t>(stream), dec.overlap,
                        any_tail ? &ttab : nullptr) == cudaSuccess
              ? QP_OK : QP_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const qp_cache* caches, const qp_tail* tails,
+                                     void* const* out, void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !q || !caches || !out || !workspace) return QP_ERR_INVALID_ARG;
+  bool uniform = true;
+  for (int l = 1; l < n_layers; ++l) uniform = uniform && caches[l].bits == caches[0].bits && caches[l].group == caches[0].group;
+  if (uniform) return decode_layers_uniform(n_layers, q, caches, tails, out, workspace, workspace_bytes, stream, false);
+  // Layers of different precision or group size (a per-layer token/precision mix): one class after the other, each
+  // with the kernels of its width.  All classes are validated before the first one is launched.
+  std::vector<const void*> cq(n_layers);
+  std::vector<void*> co(n_layers);
+  std::vector<qp_cache> cc(n_layers);
+  std::vector<qp_tail> ct(n_layers);
+  std::vector<char> taken(n_layers, 0);
+  for (int pass = 0; pass < 2; ++pass) {
+    std::fill(taken.begin(), taken.end(), 0);
+    for (int first = 0; first < n_layers; ++first) {
+      if (taken[first]) continue;
+      int m = 0;
+      for (int l = first; l < n_layers; ++l)
+        if (!taken[l] && caches[l].bits == caches[first].bits && caches[l].group == caches[first].group) {
+          taken[l] = 1;
+          cq[m] = q[l]; co[m] = out[l]; cc[m] = caches[l];
+          if (tails) ct[m] = tails[l];
+          ++m;
+        }
+      const qp_status s = decode_layers_uniform(m, cq.data(), cc.data(), tails ? ct.data() : nullptr, co.data(), workspace,
+                                                workspace_bytes, stream, pass == 0);
+      if (s != QP_OK) return s;
+    }
+  }
+  return QP_OK;
 }
 
 qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches, void* const* out,

@@ -249,3 +249,28 @@ def test_compress_layers_is_bit_identical_to_per_layer_calls(bits, D, L, w):
         torch.cuda.synchronize()
         assert torch.equal(kepts[l], ref_k), l
         assert_packed_equal(cache_to_packed(caches[l]), cache_to_packed(ref_c))
+
+
+# ------------------------------------------------------------------ per-layer token / precision mixes in one decode call
+
+def test_decode_layers_with_mixed_precision_equals_separate_calls():
+    """Sec. 5.4 swaps ranges of layers between 4 bit with 4x tokens, 8 bit with 2x and 16 bit with 1x at one budget.
+    Such a mix in ONE qp_decode_attn_layers call must give, bit for bit, what a call per layer gives (and those are
+    checked against the oracle above)."""
+    wl = small(synth.TINY, head_dim=128, n_q_heads=8, n_kv_heads=2, L=2048 + 32, w=32, batch=2)
+    budget = 16 * 256                                            # 256 tokens at 16 bit = 512 at 8 = 1024 at 4 = 2048 at 2
+    plan = [(4, 32), (4, 32), (8, 32), (16, 32), (4, 64), (2, 32), (8, 32), (4, 32)]   # (bits, group) per layer
+    caches, qs = [], []
+    for l, (bits, group) in enumerate(plan):
+        k, v, qw = make_inputs(wl, l)
+        c, _ = qp.compress_layer(k.to(DEV), v.to(DEV), qw.to(DEV), budget, bits, group, wl.pool)
+        assert c.desc.n_keep * bits == budget
+        caches.append(c)
+        qs.append(synth.make_q_dec(wl, l, 0).to(DEV))
+    outs = [torch.empty_like(q) for q in qs]
+    qp.decode_attn_layers(qp.LayerBatch(qs, caches, outs))
+    torch.cuda.synchronize()
+    for l in range(len(plan)):
+        ref = qp.decode_attn(qs[l], caches[l])
+        torch.cuda.synchronize()
+        assert torch.equal(outs[l], ref), (l, plan[l])
