@@ -43,11 +43,11 @@ NOMINAL_HBM_GBS = 8000.0
 # kernel sources it was taken on: {"sha256": <hash of DECODE_KERNEL_SOURCES>, "workload": name,
 # "bytes_per_launch": dram__bytes_read.sum + dram__bytes_write.sum}
 NCU_TRAFFIC: dict = {
-    "sha256": "ccfbe94ce393d476547a2a485af389d1f51c95a3f7efe052ed332c7d685250f6",
+    "sha256": "2c00a7b52b169901b91bcd7c77cb4bd9b42d38e933335a793f64cffb6560ef6a",
     "workload": "llama3-8b-8k-b1-4bit",
-    # captured on a 2-sequence call (168.39 MB read + 4.69 MB written per launch, mean of two launches) and
-    # scaled by the sequences per call: the traffic is proportional to the tiles a launch streams
-    "bytes_per_launch_per_sequence": (168387968 + 4691968) / 2,
+    # captured on a 4-sequence call, the launch shape of the default run (336.81 MB read + 6.17 MB written per
+    # launch, mean of two launches); other group sizes scale it: the traffic is proportional to the tiles streamed
+    "bytes_per_launch_per_sequence": (336811008 + 6166912) / 4,
 }
 
 KERNELS_PER_COMPRESS = 6      # sweep 1, row-stat merge, sweep 2, pool, top-k, gather+quantize
