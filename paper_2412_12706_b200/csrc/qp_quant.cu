@@ -35,14 +35,19 @@ __device__ __forceinline__ QParams group_params(float mn, float mx, int qmax) {
 // (x - z) * (1/s), which is within 2^-22 relative (< 1e-4 absolute for codes up to 255) of it, so the
 // rounded integer can only differ when the estimate lies that close to a half-integer; only then is
 // the IEEE division done.  The result is the same integer in every case.
+// Rounding and the conversion to an integer use the 1.5 * 2^23 trick (adding that constant rounds a float
+// below 2^22 to the nearest integer, ties to even, and leaves the integer in the low mantissa bits): plain
+// additions instead of the conversion instructions, which issue at a quarter of the rate.
 __device__ __forceinline__ uint32_t quant_code(float x, const QParams& p, int qmax) {
   if (p.sf == 0.f) return 0u;
+  constexpr float kMagic = 12582912.f;                 // 1.5 * 2^23
   const float d = __fsub_rn(x, p.zf);
-  float q = __fmul_rn(d, p.inv);
-  float r = rintf(q);
-  if (fabsf(q - r) > 0.4995f) r = rintf(__fdiv_rn(d, p.sf));
-  // 0 <= r <= qmax already: x >= min >= z, and the scale was rounded up so (max - z)/s <= qmax (1 + 2^-23)
-  return min((uint32_t)r, (uint32_t)qmax);
+  const float q = __fmul_rn(d, p.inv);                 // 0 <= q <= qmax (1 + 2^-22)
+  float m = __fadd_rn(q, kMagic);
+  const float r = __fsub_rn(m, kMagic);                // rint(q)
+  if (fabsf(__fsub_rn(q, r)) > 0.4995f) m = __fadd_rn(rintf(__fdiv_rn(d, p.sf)), kMagic);
+  // 0 <= code <= qmax already: x >= min >= z, and the scale was rounded up so (max - z)/s <= qmax (1 + 2^-23)
+  return min(__float_as_uint(m) & 0x3ffu, (uint32_t)qmax);
 }
 
 // One layer's arguments.  Sources: K, V rows [BH, L, D]; kept [BH, n_idx] positions of the rows to take

@@ -5,6 +5,8 @@
 // ordered sweep emits, in ascending position, every element above the threshold plus the
 // first `need` elements equal to it, which is exactly "largest score first, lower position
 // first among equals" without sorting.  Integer work only: results are exact.
+#include <cooperative_groups.h>
+
 #include "qp_common.cuh"
 
 namespace qp {
@@ -268,14 +270,169 @@ topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __
   }
 }
 
+// The same selection for long prefixes (up to TKC_CTAS * TKC_ITEMS * 1024 positions) by a thread-block cluster per
+// (layer, batch, KV head): CTA c of the cluster holds the contiguous segment [c * S, (c + 1) * S) of the prefix in
+// registers, builds its own digit histogram in shared memory, and every CTA then sums the cluster's histograms
+// through distributed shared memory, so all of them take the same decision without any global traffic.  One
+// hardware cluster barrier per digit pass (the histograms are double-buffered) and two around the compaction.
+constexpr int TKC_CTAS = 8;
+constexpr int TKC_ITEMS = 16;
+
+template <int NL>
+__global__ void __cluster_dims__(TKC_CTAS, 1, 1) __launch_bounds__(TK_THREADS)
+topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid_constant__ TopkOut<NL> o) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int head = blockIdx.x / TKC_CTAS, crank = (int)cluster.block_rank();
+  const int layer = head / BH, n_keep = o.n_keep[layer];
+  const int P = L - w, k = n_keep - w;
+  const int bh = head % BH, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* s = scores + (size_t)head * P;
+  int32_t* out = o.kept[layer] + (size_t)bh * n_keep;
+
+  if (crank == 0)
+    for (int i = tid; i < w; i += TK_THREADS) out[k + i] = P + i;  // window tokens are always kept
+  if (k >= P) {                                                    // keep everything (the whole cluster leaves)
+    for (int j = crank * TK_THREADS + tid; j < P; j += TKC_CTAS * TK_THREADS) out[j] = j;
+    return;
+  }
+
+  __shared__ unsigned hist[2][256];                              // this CTA's histogram, alternating per pass
+  __shared__ unsigned ghist[256];                                // the cluster's histogram
+  __shared__ unsigned sh_prefix, sh_need;
+  __shared__ unsigned cnt_g[TKC_ITEMS][32], cnt_e[TKC_ITEMS][32];
+  __shared__ unsigned row_g[TKC_ITEMS], row_e[TKC_ITEMS];
+  __shared__ unsigned tot_ge[2];                                 // this CTA's kept / equal totals
+
+  const int S = (P + TKC_CTAS - 1) / TKC_CTAS;                   // positions per CTA
+  const int seg0 = crank * S, seg_n = max(0, min(S, P - seg0));  // this CTA's segment
+  uint32_t key[TKC_ITEMS];
+#pragma unroll
+  for (int q = 0; q < TKC_ITEMS; ++q) {
+    const int i = q * TK_THREADS + tid;
+    key[q] = order_key(i < seg_n ? s[seg0 + i] : 0.f);
+  }
+
+  unsigned prefix = 0, mask = 0, need = (unsigned)k;
+  int pass = 0;
+  for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
+    unsigned* h = hist[pass & 1];
+    if (tid < 256) h[tid] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < TKC_ITEMS; ++q) {
+      if (q * TK_THREADS >= seg_n) break;
+      const bool cand = q * TK_THREADS + tid < seg_n && (key[q] & mask) == prefix;
+      const unsigned digit = (key[q] >> shift) & 255u;
+      if (shift >= 16) {
+        const unsigned peers = __match_any_sync(0xffffffffu, cand ? digit : 256u + lane);
+        if (cand && lane == __ffs(peers) - 1) atomicAdd(&h[digit], (unsigned)__popc(peers));
+      } else if (cand) {
+        atomicAdd(&h[digit], 1u);
+      }
+    }
+    cluster.sync();                                              // every CTA's histogram of this pass is complete
+    if (tid < 256) {
+      unsigned sum = 0;
+#pragma unroll
+      for (int c = 0; c < TKC_CTAS; ++c) sum += cluster.map_shared_rank(h, c)[tid];
+      ghist[tid] = sum;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      unsigned c[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = ghist[8 * lane + i]; tot += c[i]; }
+      unsigned suf = tot;
+#pragma unroll
+      for (int o2 = 1; o2 < 32; o2 <<= 1) {
+        const unsigned v = __shfl_down_sync(0xffffffffu, suf, o2);
+        if (lane + o2 < 32) suf += v;
+      }
+      const unsigned above = suf - tot;
+      if (above < need && suf >= need) {                         // exactly one lane
+        unsigned cum = above;
+        int bsel = 7;
+        for (; bsel > 0; --bsel) {
+          if (cum + c[bsel] >= need) break;
+          cum += c[bsel];
+        }
+        sh_need = need - cum;
+        sh_prefix = prefix | ((unsigned)(8 * lane + bsel) << shift);
+      }
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    need = sh_need;
+    mask |= 0xffu << shift;
+  }
+  const uint32_t T = prefix;
+
+  // ---- ordered compaction: counts per (chunk, warp) inside the CTA, CTA totals across the cluster
+#pragma unroll
+  for (int q = 0; q < TKC_ITEMS; ++q) {
+    const bool in = q * TK_THREADS + tid < seg_n;
+    const unsigned bg = __ballot_sync(0xffffffffu, in && key[q] > T), be = __ballot_sync(0xffffffffu, in && key[q] == T);
+    if (lane == 0) { cnt_g[q][warp] = __popc(bg); cnt_e[q][warp] = __popc(be); }
+  }
+  __syncthreads();
+  for (int q = warp; q < TKC_ITEMS; q += 32) {
+    const unsigned wg = cnt_g[q][lane], we = cnt_e[q][lane];
+    unsigned sg = wg, se = we;
+#pragma unroll
+    for (int o2 = 1; o2 < 32; o2 <<= 1) {
+      const unsigned vg = __shfl_up_sync(0xffffffffu, sg, o2), ve = __shfl_up_sync(0xffffffffu, se, o2);
+      if (lane >= o2) { sg += vg; se += ve; }
+    }
+    cnt_g[q][lane] = sg - wg;
+    cnt_e[q][lane] = se - we;
+    if (lane == 31) { row_g[q] = sg; row_e[q] = se; }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const unsigned wg = lane < TKC_ITEMS ? row_g[lane] : 0u, we = lane < TKC_ITEMS ? row_e[lane] : 0u;
+    unsigned sg = wg, se = we;
+#pragma unroll
+    for (int o2 = 1; o2 < 32; o2 <<= 1) {
+      const unsigned vg = __shfl_up_sync(0xffffffffu, sg, o2), ve = __shfl_up_sync(0xffffffffu, se, o2);
+      if (lane >= o2) { sg += vg; se += ve; }
+    }
+    if (lane < TKC_ITEMS) { row_g[lane] = sg - wg; row_e[lane] = se - we; }
+    if (lane == 31) { tot_ge[0] = sg; tot_ge[1] = se; }
+  }
+  cluster.sync();                                                // every CTA's totals are in place
+  unsigned base_g = 0, base_e = 0;                               // kept / equal elements in the segments before this one
+  for (int c = 0; c < crank; ++c) {
+    const unsigned* t = cluster.map_shared_rank(tot_ge, c);
+    base_g += t[0];
+    base_e += t[1];
+  }
+  const unsigned lt_mask = (1u << lane) - 1u;
+#pragma unroll
+  for (int q = 0; q < TKC_ITEMS; ++q) {
+    if (q * TK_THREADS >= seg_n) break;
+    const int i = q * TK_THREADS + tid;
+    const bool gt = i < seg_n && key[q] > T, eq = i < seg_n && key[q] == T;
+    const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+    const unsigned pg = base_g + row_g[q] + cnt_g[q][warp] + __popc(bg & lt_mask);
+    const unsigned pe = base_e + row_e[q] + cnt_e[q][warp] + __popc(be & lt_mask);
+    if (gt || (eq && pe < need)) out[pg + min(pe, need)] = seg0 + i;
+  }
+  cluster.sync();                                                // no CTA leaves while another may still read its totals
+}
+
 }  // namespace
 
 namespace {
 template <int NL>
 cudaError_t launch_topk(const float* scores, int blocks, int BH, int L, int w, const TopkOut<NL>& o, cudaStream_t st) {
   const int P = L - w;
+  // a cluster per head also pays for medium prefixes when the heads alone would leave most SMs idle
+  const bool few_heads = blocks * TKC_CTAS <= sm_count();
   if (P <= 8 * TK_THREADS) topk_reg_kernel<8, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
-  else if (P <= 32 * TK_THREADS) topk_reg_kernel<32, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
+  else if (P <= 32 * TK_THREADS && !few_heads) topk_reg_kernel<32, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
+  else if (P <= TKC_CTAS * TKC_ITEMS * TK_THREADS)
+    topk_cluster_kernel<NL><<<blocks * TKC_CTAS, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
   else topk_kernel<NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
   return cudaGetLastError();
 }

@@ -34,7 +34,8 @@ def compress(wl, n_cap_extra):
 
 # (bits, group, D, G): all four tensor-core kernels, groups of 64 / 128, and shapes that take the generic kernel
 SHAPES = [(4, 32, 128, 4), (4, 64, 128, 4), (4, 128, 128, 2), (4, 32, 64, 4), (8, 32, 128, 4), (8, 64, 128, 8),
-          (2, 32, 128, 4), (2, 32, 128, 8), (2, 64, 128, 4), (16, 32, 128, 4), (16, 32, 64, 8)]
+          (2, 32, 128, 4), (2, 32, 128, 8), (2, 64, 128, 4), (16, 32, 128, 4), (16, 32, 64, 8),
+          (4, 32, 64, 3), (8, 32, 128, 1), (2, 32, 128, 3)]      # odd group sizes: a merge block's second warp may idle
 
 
 @pytest.mark.parametrize("bits,group,D,G", SHAPES)
