@@ -38,7 +38,7 @@ extern "C" {
 typedef enum {
   QP_OK = 0,
   QP_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, Hq % Hkv != 0, w >= L, even pool ... */
-  QP_ERR_UNSUPPORTED = 2, /* bits not in {2,4,8,16}, group not in {32,64,128}, D not in {64,128}, G > 8, w > 64 */
+  QP_ERR_UNSUPPORTED = 2, /* bits not in {2,4,8,16}, group not in {32,64,128}, D not in {64,128}, G > 8, w > 64, pool > 65 */
   QP_ERR_BUDGET = 3,      /* budget gives n <= w, n is not a whole number of groups, or no room to append */
   QP_ERR_WORKSPACE = 4,   /* workspace too small */
   QP_ERR_ALIGNMENT = 5,   /* a base pointer is not 16-byte aligned */
@@ -117,7 +117,7 @@ size_t qp_decode_workspace_bytes(const qp_cache* cache /* host */);
  *   vote[j] = sum_h sum_i Pr_{h,i}[j]                          j < P
  *   scores[j] = (sum_{|t| <= (pool-1)/2} vote[j+t], zero outside [0,P)) / pool
  * Q_win bf16 [Bt,Hq,w,D], K bf16 [Bt,Hkv,L,D] (device) -> scores fp32 [Bt,Hkv,P] (device).
- * pool must be odd (1 = no pooling).
+ * pool must be odd (1 = no pooling) and at most 65.
  */
 qp_status qp_window_scores(const void* Q_win, const void* K, int batch, int n_q_heads, int n_kv_heads,
                            int head_dim, int L, int w, int pool, float* scores, void* workspace,

@@ -190,7 +190,7 @@ static qp_status check_score_args(const void* Q_win, const void* K, int batch, i
   qp_status s = check_shape(batch, Hq, Hkv, D);
   if (s != QP_OK) return s;
   if (w < 1 || w >= L || pool < 1 || pool % 2 == 0) return QP_ERR_INVALID_ARG;
-  if (w > 64) return QP_ERR_UNSUPPORTED;
+  if (w > 64 || pool > 65) return QP_ERR_UNSUPPORTED;
   if (!aligned16(Q_win) || !aligned16(K)) return QP_ERR_ALIGNMENT;
   return QP_OK;
 }

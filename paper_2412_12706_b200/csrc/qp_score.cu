@@ -21,14 +21,16 @@ constexpr int SC_RB = 128;       // window-query rows per thread block (8 warps 
 __host__ __device__ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // per row: M = max over tiles, Z = sum_i s_i * 2^(m_i - M); stores (M, 1/Z); rows beyond R get 1/Z = 0.
-// One block per (batch, KV head, row block): thread (row, slice) folds tiles slice, slice+8, ... into a running
-// (max, sum) pair with coalesced reads across rows; the eight slices are then combined in a fixed order.
-constexpr int RM_SLICES = 8;
-__global__ void __launch_bounds__(SC_RB * RM_SLICES)
+// One block per (batch, KV head, row block, group of RM_ROWS rows): thread (row, slice) folds tiles slice,
+// slice + RM_SLICES, ... into a running (max, sum) pair with coalesced reads across rows; the slices are then
+// combined in a fixed order.
+constexpr int RM_SLICES = 32, RM_ROWS = 32, RM_PARTS = SC_RB / RM_ROWS;
+__global__ void __launch_bounds__(RM_ROWS * RM_SLICES)
 rowstat_merge_kernel(const float2* __restrict__ stat_partial, int n_rb, int n_tiles, int R,
                      float2* __restrict__ rowstat) {
-  __shared__ float2 part[RM_SLICES][SC_RB];
-  const int blk = blockIdx.x, rb = blk % n_rb, row = threadIdx.x % SC_RB, sl = threadIdx.x / SC_RB;
+  __shared__ float2 part[RM_SLICES][RM_ROWS];
+  const int blk = blockIdx.x / RM_PARTS, rb = blk % n_rb;
+  const int rl = threadIdx.x % RM_ROWS, sl = threadIdx.x / RM_ROWS, row = (blockIdx.x % RM_PARTS) * RM_ROWS + rl;
   const float2* p = stat_partial + (size_t)blk * n_tiles * SC_RB + row;
   float m = -INFINITY, z = 0.f;
   for (int i = sl; i < n_tiles; i += RM_SLICES) {
@@ -39,33 +41,43 @@ rowstat_merge_kernel(const float2* __restrict__ stat_partial, int n_rb, int n_ti
       m = mn;
     }
   }
-  part[sl][row] = make_float2(m, z);
+  part[sl][rl] = make_float2(m, z);
   __syncthreads();
   if (sl == 0) {
     float M = -INFINITY;
 #pragma unroll
-    for (int k = 0; k < RM_SLICES; ++k) M = fmaxf(M, part[k][row].x);
+    for (int k = 0; k < RM_SLICES; ++k) M = fmaxf(M, part[k][rl].x);
     float Z = 0.f;
 #pragma unroll
     for (int k = 0; k < RM_SLICES; ++k)
-      if (part[k][row].x != -INFINITY) Z += part[k][row].y * exp2f(part[k][row].x - M);
+      if (part[k][rl].x != -INFINITY) Z += part[k][rl].y * exp2f(part[k][rl].x - M);
     const bool valid = rb * SC_RB + row < R;
     rowstat[(size_t)blk * SC_RB + row] = make_float2(valid ? M : 0.f, valid ? __fdiv_rn(1.0f, Z) : 0.f);
   }
 }
 
-__global__ void __launch_bounds__(256)
+// scores[j] = (sum over |t| <= r of vote[j + t], zero outside [0, P)) / pool with vote = the sum of the row blocks'
+// partial votes.  A block stages the votes of its 256 outputs and their halo in shared memory.
+constexpr int PK_THREADS = 256, PK_MAX_HALO = 32;
+__global__ void __launch_bounds__(PK_THREADS)
 pool_kernel(const float* __restrict__ votes_partial, int n_rb, int P, int pool, float* __restrict__ scores) {
-  const int bh = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= P) return;
-  const int r = (pool - 1) / 2;
-  float acc = 0.f;
-  for (int dlt = -r; dlt <= r; ++dlt) {
-    const int jj = j + dlt;
-    if (jj < 0 || jj >= P) continue;
+  __shared__ float sv[PK_THREADS + 2 * PK_MAX_HALO];
+  const int bh = blockIdx.y, j0 = blockIdx.x * PK_THREADS, r = (pool - 1) / 2;
+  for (int i = threadIdx.x; i < PK_THREADS + 2 * r; i += PK_THREADS) {
+    const int jj = j0 - r + i;
     float v = 0.f;
-    for (int rb = 0; rb < n_rb; ++rb) v += votes_partial[(size_t)(bh * n_rb + rb) * P + jj];
-    acc += v;
+    if (jj >= 0 && jj < P)
+      for (int rb = 0; rb < n_rb; ++rb) v += votes_partial[(size_t)(bh * n_rb + rb) * P + jj];
+    sv[i] = v;
+  }
+  __syncthreads();
+  const int j = j0 + threadIdx.x;
+  if (j >= P) return;
+  float acc = 0.f;
+  for (int dlt = 0; dlt <= 2 * r; ++dlt) {
+    const int jj = j - r + dlt;
+    if (jj < 0 || jj >= P) continue;
+    acc += sv[threadIdx.x + dlt];
   }
   scores[(size_t)bh * P + j] = __fdiv_rn(acc, (float)pool);
 }
@@ -105,7 +117,7 @@ cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, c
   if (e != cudaSuccess) return e;
   e = launch_score_sweep_tc(1, n_layers, Qwin, K, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st);
   if (e != cudaSuccess) return e;
-  rowstat_merge_kernel<<<BH * s.n_rb, SC_RB * RM_SLICES, 0, st>>>(stat_partial, s.n_rb, 2 * s.n_tiles, R, rowstat);
+  rowstat_merge_kernel<<<BH * s.n_rb * RM_PARTS, RM_ROWS * RM_SLICES, 0, st>>>(stat_partial, s.n_rb, 2 * s.n_tiles, R, rowstat);
   e = launch_score_sweep_tc(2, n_layers, Qwin, K, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st);
   if (e != cudaSuccess) return e;
   pool_kernel<<<dim3((P + 255) / 256, BH), 256, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);

@@ -52,7 +52,7 @@ def test_gather_quantize_bit_exact(bits, group, D):
 
 @pytest.mark.parametrize("P,w,n", [(992, 32, 512), (37, 5, 6), (5000, 64, 64 + 1), (4097, 8, 8 + 4096),
                                    (70000, 32, 8192), (300, 20, 320), (131072, 64, 4096 + 64),
-                                   (140000, 32, 8192 + 32), (33000, 8, 8 + 1)])
+                                   (140000, 32, 8192 + 32), (33000, 8, 8 + 1), (20000, 32, 32 + 7000)])
 def test_select_topk_bit_exact_with_ties(P, w, n):
     L = P + w
     rng = np.random.default_rng(P + n)
