@@ -275,3 +275,44 @@ def test_decode_layers_with_mixed_precision_equals_separate_calls():
         ref = qp.decode_attn(qs[l], caches[l])
         torch.cuda.synchronize()
         assert torch.equal(outs[l], ref), (l, plan[l])
+
+
+# ------------------------------------------------------------------ determinism and memory hygiene
+
+@pytest.mark.parametrize("bits", [2, 4, 8, 16])
+def test_same_bits_every_run_and_no_write_outside_the_outputs(bits):
+    """The whole path twice on the same inputs gives identical bytes everywhere (no floating-point atomics, fixed
+    reduction orders), and guard words placed directly behind every output buffer stay untouched."""
+    wl = small(synth.TINY, head_dim=128, n_q_heads=8, n_kv_heads=2, L=1500, w=32, batch=2, bits=bits,
+               tokens16=384 * bits // 16)
+    k, v, qw = (t.to(DEV) for t in make_inputs(wl))
+    q = synth.make_q_dec(wl, 0, 0).to(DEV)
+    GUARD = 64
+    n = wl.n_keep(0)
+
+    def guarded(nbytes):
+        buf = torch.full((nbytes + GUARD,), 0xA5, dtype=torch.uint8, device=DEV)
+        return buf
+
+    def run():
+        d = qp.cache_layout(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, bits, wl.group, n)
+        sizes = [d.k_codes_bytes, d.v_codes_bytes] + ([d.k_meta_bytes] * 2 + [d.v_meta_bytes] * 2 if bits < 16 else [])
+        bufs = [guarded(sz) for sz in sizes]
+        d.k_codes, d.v_codes = bufs[0].data_ptr(), bufs[1].data_ptr()
+        if bits < 16:
+            d.k_scale, d.k_zero, d.v_scale, d.v_zero = (b.data_ptr() for b in bufs[2:])
+        cache = qp.Cache(d, *bufs[:2], *(bufs[2:] if bits < 16 else [None] * 4))
+        kept = guarded(wl.batch * wl.n_kv_heads * n * 4)
+        out = guarded(q.numel() * 2)
+        kept_t = kept[:-GUARD].view(torch.int32).view(wl.batch, wl.n_kv_heads, n)
+        out_t = out[:-GUARD].view(torch.bfloat16).view_as(q)
+        qp.compress_layer(k, v, qw, wl.budget_bits, bits, wl.group, wl.pool, cache, kept_t)
+        qp.decode_attn(q, cache, out_t)
+        torch.cuda.synchronize()
+        for b in bufs + [kept, out]:
+            assert bool((b[-GUARD:] == 0xA5).all()), "a kernel wrote past the end of an output buffer"
+        return [b[:-GUARD].clone() for b in bufs + [kept, out]]
+
+    first, second = run(), run()
+    for a, b in zip(first, second):
+        assert torch.equal(a, b)
