@@ -483,19 +483,23 @@ def run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step, per_call=1):
     hK = [[k.cpu().pin_memory() for k in sq["K"]] for sq in seqs]
     hV = [[v.cpu().pin_memory() for v in sq["V"]] for sq in seqs]
     hQ = [[q.cpu().pin_memory() for q in sq["Qw"]] for sq in seqs]
-    hq = [sq["qdec"].cpu().pin_memory() for sq in seqs]
-    hout = [torch.empty((n_dec,) + tuple(sq["out"].shape), dtype=torch.bfloat16).pin_memory() for sq in seqs]
     dK, dV, dQ = torch.empty_like(seqs[0]["K"][0]), torch.empty_like(seqs[0]["V"][0]), torch.empty_like(seqs[0]["Qw"][0])
-    dq = [torch.empty_like(sq["qdec"][0]) for sq in seqs]
+    # decode: the queries and the outputs of the sequences of one call are one contiguous block on either side,
+    # so a call costs one upload and one download
     groups = []
     for g0 in range(0, len(seqs), per_call):
         ids = list(range(g0, g0 + per_call))
+        hq_g = torch.stack([seqs[i]["qdec"] for i in ids], dim=1).cpu().pin_memory()     # [n_dec, per_call, layers, Bt, Hq, D]
+        dq_g = torch.empty_like(hq_g[0], device=dev)
+        dout_g = torch.empty_like(dq_g)
+        hout_g = torch.empty_like(hq_g).pin_memory()
         ws_g = torch.empty(sum(seqs[i]["ws_d"].numel() for i in ids), dtype=torch.uint8, device=dev)
-        groups.append((ids, qp.LayerBatch([dq[i][l] for i in ids for l in range(n_layers)],
-                                          [c for i in ids for c in seqs[i]["cache"]],
-                                          [seqs[i]["out"][l] for i in ids for l in range(n_layers)], ws_g)))
-    h2d = sum(t.numel() * 2 for per in (hK, hV, hQ) for s in per for t in s) + sum(t.numel() * 2 for t in hq)
-    d2h = sum(t.numel() * 2 for t in hout)
+        batch = qp.LayerBatch([dq_g[j, l] for j in range(per_call) for l in range(n_layers)],
+                              [c for i in ids for c in seqs[i]["cache"]],
+                              [dout_g[j, l] for j in range(per_call) for l in range(n_layers)], ws_g)
+        groups.append((hq_g, dq_g, dout_g, hout_g, batch))
+    h2d = sum(t.numel() * 2 for per in (hK, hV, hQ) for s in per for t in s) + sum(g[0].numel() * 2 for g in groups)
+    d2h = sum(g[3].numel() * 2 for g in groups)
 
     def step():
         a = torch.cuda.Event(enable_timing=True); a.record(stream)
@@ -507,12 +511,10 @@ def run_e2e(args, wl, qp, seqs, ws_c, dev, stream, dec_bytes_step, per_call=1):
                                   sq["cache"][l], sq["kept"][l], ws_c)
         b = torch.cuda.Event(enable_timing=True); b.record(stream)
         for t in range(n_dec):
-            for ids, batch in groups:
-                for i in ids:
-                    dq[i].copy_(hq[i][t], non_blocking=True)
+            for hq_g, dq_g, dout_g, hout_g, batch in groups:
+                dq_g.copy_(hq_g[t], non_blocking=True)
                 qp.decode_attn_layers(batch)
-                for i in ids:
-                    hout[i][t].copy_(seqs[i]["out"], non_blocking=True)
+                hout_g[t].copy_(dout_g, non_blocking=True)
         c = torch.cuda.Event(enable_timing=True); c.record(stream)
         return a, b, c
 
