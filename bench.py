@@ -541,6 +541,8 @@ def main():
                     help="sequences whose layers go into one qp_decode_attn_layers call")
     ap.add_argument("--layers", type=int, default=0, help="profiling: keep only the first N layers of the workload")
     ap.add_argument("--batch", type=int, default=0, help="profiling: override the workload's batch size")
+    ap.add_argument("--bits", type=int, default=0, choices=[0, 2, 4, 8, 16],
+                    help="profiling: override the workload's code width (the token budget follows: tokens x bits constant)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-compress-layers", action="store_true", help="skip the qp_compress_layers figure")
     ap.add_argument("--no-generation", action="store_true", help="skip the append + decode generation-loop figure")
@@ -548,9 +550,11 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
-    if args.layers or args.batch:      # a cut-down case of the same kernels, for ncu captures; never the bench line
+    if args.layers or args.batch or args.bits:   # a variant of the same kernels, for ncu captures; never the bench line
         wl = synth.dataclasses.replace(wl, n_layers=args.layers or wl.n_layers, batch=args.batch or wl.batch,
-                                       name=f"{wl.name}[layers={args.layers or wl.n_layers},batch={args.batch or wl.batch}]")
+                                       bits=args.bits or wl.bits,
+                                       name=f"{wl.name}[layers={args.layers or wl.n_layers},batch={args.batch or wl.batch},"
+                                            f"bits={args.bits or wl.bits}]")
     if args.impl == "reference":
         run_reference(args, wl)
     else:
