@@ -171,3 +171,31 @@ def test_llama8b_generation_loop_in_the_bench_configuration():
                          sl(c.v_codes, n).cpu().numpy().view(np.uint32), bits_u16(sl(c.k_scale, n // g)),
                          bits_u16(sl(c.k_zero, n // g)), bits_u16(sl(c.v_scale, n)), bits_u16(sl(c.v_zero, n)))
         assert_packed_equal(got, states[si].packed)
+
+
+def test_llama8b_compress_layers_in_the_bench_configuration():
+    """qp_compress_layers over the 32 layers of an 8k sequence (the call the benchmark times) leaves, bit for bit,
+    the kept indices and packed bytes of 32 qp_compress_layer calls; one sampled (layer, KV head) pair is also
+    recomputed by the oracle (indices with the near-tie rule, packed bytes on the GPU's indices)."""
+    wl = synth.LLAMA8B_8K
+    nl, G = wl.n_layers, wl.n_q_heads // wl.n_kv_heads
+    Ks, Vs, Qs = [], [], []
+    for l in range(nl):
+        k, v = synth.make_kv(wl, l, device=DEV)
+        Ks.append(k); Vs.append(v); Qs.append(synth.make_q_win(wl, l, device=DEV))
+    budgets = [wl.layer_budget_bits(l) for l in range(nl)]
+    caches, kepts = qp.compress_layers(Ks, Vs, Qs, budgets, wl.bits, wl.group, wl.pool)
+    torch.cuda.synchronize()
+    for l in range(nl):
+        ref_c, ref_k = qp.compress_layer(Ks[l], Vs[l], Qs[l], budgets[l], wl.bits, wl.group, wl.pool)
+        torch.cuda.synchronize()
+        assert torch.equal(kepts[l], ref_k), l
+        for name in ("k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero"):
+            assert torch.equal(getattr(caches[l], name), getattr(ref_c, name)), (l, name)
+    layer, hk = 17, 5
+    kb = bits_u16(Ks[layer][0:1, hk:hk + 1]); vb = bits_u16(Vs[layer][0:1, hk:hk + 1])
+    qb = bits_u16(Qs[layer][0:1, hk * G:(hk + 1) * G])
+    pooled = orc.scores(qb, kb, wl.pool)
+    kept_s = kepts[layer][0:1, hk:hk + 1].cpu().numpy()
+    assert check_kept_against_oracle(kept_s, pooled, wl.L, wl.w, kept_s.shape[-1]) <= 2
+    assert_packed_equal(_slice_packed(caches[layer], 0, hk), orc.quantize(kb, vb, kept_s, wl.bits, wl.group))
