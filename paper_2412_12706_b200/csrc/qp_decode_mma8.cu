@@ -192,6 +192,7 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       // zero-point term with swapped roles (A = query pairs as they sit in registers, B = zero-point pairs as
       // loaded; rows g of the first, rows g+8 of the second MMA are read), as in the 4-bit kernel
       float accK[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      float accK2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // second k-step of a round: a chain of its own
       float accZa[4] = {0.f, 0.f, 0.f, 0.f}, accZb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c2 = 0; c2 < NQ / 2; ++c2) {                     // two k-steps (8 channels of this lane) per round
@@ -206,10 +207,14 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         mma_f16_m16n8k16(accK[1], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), b00, b01);
         mma_f16_m16n8k16(accZa, qh2[4 * c2 + 0], qh2[4 * c2 + 1], qh2[4 * c2 + 2], qh2[4 * c2 + 3], z4.x, z4.y);
         ldmatrix_x4_trans(R0, R1, R2, R3, sb + k_plane + ((k_slot0 ^ (8 * c2 + 4)) << 4));
-        mma_f16_m16n8k16(accK[0], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), b10, b11);
-        mma_f16_m16n8k16(accK[1], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), b10, b11);
+        mma_f16_m16n8k16(accK2[0], R0 & M8, odd_bytes(R0), R1 & M8, odd_bytes(R1), b10, b11);
+        mma_f16_m16n8k16(accK2[1], R2 & M8, odd_bytes(R2), R3 & M8, odd_bytes(R3), b10, b11);
         mma_f16_m16n8k16(accZb, qh2[4 * c2 + 0], qh2[4 * c2 + 1], qh2[4 * c2 + 2], qh2[4 * c2 + 3], z4.z, z4.w);
       }
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+        for (int x = 0; x < 4; ++x) accK[hf][x] += accK2[hf][x];
       const float zq = accZa[0] + accZb[2];                     // of head g; this lane needs columns 2t, 2t+1
       const float zq_e[2] = {__shfl_sync(0xffffffffu, zq, 8 * t), __shfl_sync(0xffffffffu, zq, 8 * t + 4)};
 
