@@ -205,7 +205,7 @@ score_sweep_tc_kernel(const __grid_constant__ ScorePtrs<NL> ptrs, int BH, int Hq
     const bool ok = mbar_wait(bar0 + (j & 1) * 8, (j >> 1) & 1);
     if (!ok) give_up = 1;
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-    __syncthreads();                                    // everyone sees the verdict; stage j & 1 is free again
+    __syncthreads();                                    // everyone sees the outcome; stage j & 1 is free again
     if (give_up) break;
     if (j + 2 < n_loc) {
       const int tl = tile_lo + j + 2;
