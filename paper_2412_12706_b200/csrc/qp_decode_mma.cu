@@ -463,6 +463,65 @@ decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, c
   }
 }
 
+// S5 for launches with few output rows (at most one per SM): one block per (layer, batch, query head), its four
+// warps share the head's records (warp q takes records q, q + 4, ...), so a row's chain of dependent reads is a
+// quarter as long; the four partial sums are combined through shared memory in a fixed order.  Same launch
+// protocol as decode_merge_sk_kernel.
+__global__ void __launch_bounds__(MG_WARPS * 32, 16)
+decode_merge_rows_kernel(const __grid_constant__ DecTable tab, const DecDims dm, const float* __restrict__ partials) {
+  __shared__ float s_max[MG_WARPS];
+  __shared__ float s_part[MG_WARPS][5 * 32];                      // per warp: lane's (A0..A3, Ls)
+  const int D = dm.D, G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv, n_bq = dm.Bt * dm.Hq;
+  const int lane = threadIdx.x & 31, wq = threadIdx.x >> 5;
+  const unsigned T = (unsigned)tab.total_tiles, W = (unsigned)tab.n_workers;
+  const size_t stride = (size_t)G * (D + 2);
+  asm volatile("griddepcontrol.launch_dependents;\n" ::);
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  const int layer = blockIdx.x / n_bq, bq = blockIdx.x % n_bq;
+  const DecLayer& ly = tab.l[layer];
+  const int b = bq / dm.Hq, h = bq % dm.Hq, bh = b * dm.Hkv + h / G, hl = h % G;
+  const int tph = (ly.n + 31) >> 5;
+  const unsigned first = (unsigned)ly.tile_base + (unsigned)bh * tph;
+  const int w_lo = (int)(((first + 1u) * W - 1u) / T), w_hi = (int)(((first + tph) * W - 1u) / T);
+  const float* base = partials + (((size_t)layer * BH + bh) * G + hl) * (size_t)(D + 2);
+  // the records' reference maxima: a thread per record, then across the block
+  float M = -INFINITY;
+  for (int w = w_lo + (int)threadIdx.x; w <= w_hi; w += MG_WARPS * 32) M = fmaxf(M, base[w * stride]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  if (lane == 0) s_max[wq] = M;
+  __syncthreads();
+  M = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
+  float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
+  if (4 * lane < D)
+    for (int w = w_lo + wq; w <= w_hi; w += MG_WARPS) {
+      const float* r = base + w * stride;
+      const float2 ml = *reinterpret_cast<const float2*>(r);
+      const float2 a01 = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
+      const float2 a23 = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
+      const float f = ex2(ml.x - M);
+      Ls = fmaf(ml.y, f, Ls);
+      A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
+      A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
+    }
+  float* mine = s_part[wq] + 5 * lane;
+  mine[0] = A0; mine[1] = A1; mine[2] = A2; mine[3] = A3; mine[4] = Ls;
+  __syncthreads();
+  if (wq != 0 || 4 * lane >= D) return;
+  Ls = A0 = A1 = A2 = A3 = 0.f;
+#pragma unroll
+  for (int q = 0; q < MG_WARPS; ++q) {
+    const float* o = s_part[q] + 5 * lane;
+    A0 += o[0]; A1 += o[1]; A2 += o[2]; A3 += o[3]; Ls += o[4];
+  }
+  const float inv = __fdiv_rn(1.0f, Ls);
+  __nv_bfloat162 o01 = __floats2bfloat162_rn(A0 * inv, A1 * inv), o23 = __floats2bfloat162_rn(A2 * inv, A3 * inv);
+  uint2 packed;
+  packed.x = *reinterpret_cast<uint32_t*>(&o01);
+  packed.y = *reinterpret_cast<uint32_t*>(&o23);
+  *reinterpret_cast<uint2*>(static_cast<bf16*>(ly.out) + (size_t)bq * D + 4 * lane) = packed;
+}
+
 template <int D, int STAGES>
 constexpr size_t mma4_smem_bytes() { return (size_t)DM_WARPS * (STAGES * Tile4<D>::BYTES + SP_BYTES); }
 
@@ -539,6 +598,10 @@ cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* part
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (items <= sm_count()) {                                    // few rows: a block per row
+    cfg.gridDim = dim3(items);
+    return cudaLaunchKernelEx(&cfg, decode_merge_rows_kernel, tab, d, (const float*)partials);
+  }
   return cudaLaunchKernelEx(&cfg, decode_merge_sk_kernel, tab, d, (const float*)partials);
 }
 
