@@ -25,7 +25,11 @@ class PrevOutputs {
     int parity;     // workspace half of this call: alternates per (device, stream)
   };
   // decides for this call, then records `writes` as the stream's latest outputs
-  Decision check_and_record(int device, cudaStream_t st, const std::vector<Range>& reads, std::vector<Range>& writes) {
+  // ws_base / half_bytes: this call's partial records go to [ws_base + parity * half_bytes, + half_bytes); if that
+  // area meets the one the previous call's merge may still be reading (calls of different sizes place their halves
+  // differently), the call must not overlap the previous one either
+  Decision check_and_record(int device, cudaStream_t st, const std::vector<Range>& reads, std::vector<Range>& writes,
+                            uintptr_t ws_base, size_t half_bytes) {
     std::sort(writes.begin(), writes.end());
     // after sorting by begin, writes[i].second becomes the largest end among writes[0..i]: a read [b, e) meets
     // one of the writes that begin before e exactly when that running maximum exceeds b
@@ -50,6 +54,9 @@ class PrevOutputs {
       dec.overlap = false;
     }
     Entry& e = prev_[key];
+    const Range mine{ws_base + (dec.parity ? half_bytes : 0), ws_base + (dec.parity ? half_bytes : 0) + half_bytes};
+    if (mine.first < e.scratch.second && e.scratch.first < mine.second) dec.overlap = false;
+    e.scratch = mine;
     e.outs.swap(writes);
     e.parity = dec.parity;
     e.barrier = false;
@@ -70,6 +77,7 @@ class PrevOutputs {
  private:
   struct Entry {
     std::vector<Range> outs;
+    Range scratch{0, 0};     // where the last call's partial records live
     int parity = 0;
     bool barrier = false;
   };
@@ -340,8 +348,10 @@ qp_status decode_layers_uniform(int n_layers, const void* const* q, const qp_cac
   if (any_tail)
     for (int l = 0; l < n_layers; ++l) ttab.l[l] = TailLayer{tails[l].k_tail, tails[l].v_tail, tails[l].n_tail, 0};
   const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
-  if (workspace_bytes < decode_plan(tab, d)) return QP_ERR_WORKSPACE;
+  const size_t need = decode_plan(tab, d);
+  if (workspace_bytes < need) return QP_ERR_WORKSPACE;
   if (check_only) return QP_OK;
+  const size_t half_bytes = decode_mma_supported(d) ? decode_workspace_layout(tab, d).record_bytes : need;
   // everything the attention kernel reads before it waits for the stream's previous kernel, and what this
   // call's merge kernel writes
   std::vector<PrevOutputs::Range> reads, writes;
@@ -364,7 +374,8 @@ qp_status decode_layers_uniform(int n_layers, const void* const* q, const qp_cac
   int device = 0;
   if (cudaGetDevice(&device) != cudaSuccess) return QP_ERR_CUDA;
   const PrevOutputs::Decision dec =
-      g_prev_outputs.check_and_record(device, static_cast<cudaStream_t>(stream), reads, writes);
+      g_prev_outputs.check_and_record(device, static_cast<cudaStream_t>(stream), reads, writes,
+                                      reinterpret_cast<uintptr_t>(workspace), half_bytes);
   return launch_decode(tab, d, workspace, dec.parity, static_cast<cudaStream_t>(stream), dec.overlap,
                        any_tail ? &ttab : nullptr) == cudaSuccess
              ? QP_OK : QP_ERR_CUDA;

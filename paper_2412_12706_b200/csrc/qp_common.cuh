@@ -173,7 +173,7 @@ int sm_count();   // SMs of the current device (cached)
 // tensor-core split-K kernel and its merge
 bool decode_mma_supported(const DecDims& d);
 int decode_mma_workers_per_sm(const DecDims& d);     // workers (see DecTable::n_workers) resident per SM
-int decode_mma_tiles_per_worker_min(const DecDims& d);   // small launches use fewer workers, not emptier ones
+int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles);   // small launches: fewer workers, not emptier ones
 int decode_mma_wide_workers_per_sm(const DecDims& d, int* min_tiles);
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
                               bool overlap_prev, const TailTable* tails = nullptr);

@@ -240,8 +240,8 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
       tab.wide = 1;
     }
     if (W > kMaxDecodeWorkers) W = kMaxDecodeWorkers;
-    const int tmin = decode_mma_tiles_per_worker_min(d);        // at least one tile per warp
-    if (W > (T + tmin - 1) / tmin) W = (T + tmin - 1) / tmin;
+    const int tmin = decode_mma_tiles_per_worker_min(d, T);
+    if (!tab.wide && W > (T + tmin - 1) / tmin) W = (T + tmin - 1) / tmin;
     if (W < 1) W = 1;
     while (W > 1 && T * W >= (1ll << 31)) W /= 2;               // the merge kernel's range arithmetic is 32-bit
     tab.total_tiles = (int)T;

@@ -539,9 +539,17 @@ int decode_mma_workers_per_sm(const DecDims& d) {
   return d.bits == 4 ? DM_DEEP_MINB * DM_WARPS : d.bits == 8 ? decode_mma8_blocks_per_sm() * decode_mma8_warps()
          : d.bits == 16 ? decode_mma16_blocks_per_sm() : decode_mma2_workers_per_sm();
 }
-// Small launches: four tiles per worker at least (a 4-bit worker is one warp, the others four warps with a tile
-// each); more, smaller records per head cost the merge kernel more than the attention kernel gains.
-int decode_mma_tiles_per_worker_min(const DecDims&) { return 4; }
+// Launches that do not fill every worker slot with a long range use fewer workers, not emptier ones: a worker's
+// ramp and its partial record (which the merge step has to read) are costs per worker.  Measured for the 4-bit
+// kernel on caches of 64 tiles per head: per-layer calls (512 tiles) from a CUDA graph take 9.8 / 6.4 / 4.0 / 3.6 /
+// 3.3 / 3.8 us with at least 1 / 2 / 4 / 8 / 16 / 32 tiles per worker, 84 MB calls (16384 tiles) 20.4 us with the
+// 1776 workers of a full grid, 19.5 us with 16 tiles per worker and 17.5 us with 32 (512 workers, two per head,
+// ranges aligned with the heads), 26.6 us with 64.  So: 32 tiles where that still leaves 256 workers, else 16.
+// The other kernels keep four tiles per worker.
+int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles) {
+  if (d.bits != 4) return 4;
+  return total_tiles / 32 >= 256 ? 32 : 16;
+}
 // Workers per SM of the wider build of this shape's kernel and the tiles per worker from which it pays
 // (0: the shape has one build only).
 int decode_mma_wide_workers_per_sm(const DecDims& d, int* min_tiles) {
