@@ -545,9 +545,11 @@ int decode_mma_workers_per_sm(const DecDims& d) {
 // 3.3 / 3.8 us with at least 1 / 2 / 4 / 8 / 16 / 32 tiles per worker, 84 MB calls (16384 tiles) 20.4 us with the
 // 1776 workers of a full grid, 19.5 us with 16 tiles per worker and 17.5 us with 32 (512 workers, two per head,
 // ranges aligned with the heads), 26.6 us with 64.  So: 32 tiles where that still leaves 256 workers, else 16.
-// The other kernels keep four tiles per worker.
+// The 8-bit kernel behaves alike (151 MB calls of 16384 tiles: 4.22 / 4.02 / 5.08 / 2.76 TB/s with 4 / 16 / 32 / 64);
+// the 2-bit and 16-bit kernels showed no gain (4.96 / 4.78 / 4.87 / 4.65 and 5.60 / 5.61 / 5.60 / 4.81 TB/s) and keep
+// four tiles per worker.
 int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles) {
-  if (d.bits != 4) return 4;
+  if (d.bits != 4 && d.bits != 8) return 4;
   return total_tiles / 32 >= 256 ? 32 : 16;
 }
 // Workers per SM of the wider build of this shape's kernel and the tiles per worker from which it pays
