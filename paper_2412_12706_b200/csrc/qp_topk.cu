@@ -427,9 +427,11 @@ namespace {
 template <int NL>
 cudaError_t launch_topk(const float* scores, int blocks, int BH, int L, int w, const TopkOut<NL>& o, cudaStream_t st) {
   const int P = L - w;
-  // a cluster per head also pays for medium prefixes when the heads alone would leave most SMs idle
+  // a cluster per head also pays for shorter prefixes (above 2048 positions) when the heads alone would leave most
+  // SMs idle: eight CTAs with one or two keys per thread beat one CTA with eight
   const bool few_heads = blocks * TKC_CTAS <= sm_count();
-  if (P <= 8 * TK_THREADS) topk_reg_kernel<8, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
+  if (P <= 8 * TK_THREADS && !(few_heads && P > 2 * TK_THREADS))
+    topk_reg_kernel<8, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
   else if (P <= 32 * TK_THREADS && !few_heads) topk_reg_kernel<32, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
   else if (P <= TKC_CTAS * TKC_ITEMS * TK_THREADS)
     topk_cluster_kernel<NL><<<blocks * TKC_CTAS, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
