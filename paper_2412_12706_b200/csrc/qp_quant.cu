@@ -1,7 +1,7 @@
 // S3: fused gather + asymmetric min/max group quantization + packing.
 //
-// One thread block per (batch, KV head, run of g kept tokens).  The g kept key rows are
-// gathered into shared memory with 16-byte loads; thread d then owns channel d of the key
+// Two thread blocks per (batch, KV head, run of g kept tokens): one for the key group, one for the
+// value rows.  The g kept key rows are gathered into shared memory with 16-byte loads; thread d then owns channel d of the key
 // group (g tokens, per-channel quantization) and writes its g*B/32 packed words, scale and
 // zero; the value groups of the same g tokens (per-token quantization, g channels each) are
 // handled one group per thread straight from global memory.
@@ -72,7 +72,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __shared__ int sidx[128];
   constexpr int QMAX = (1 << BITS) - 1, PER = 32 / BITS;
   const QuantLayer& ql = tab.l[blockIdx.z];
-  if ((int)blockIdx.x * g >= ql.n_idx) return;     // layers of one launch may keep different numbers of tokens
+  if ((int)(blockIdx.x >> 1) * g >= ql.n_idx) return;   // layers of one launch may keep different numbers of tokens
   const uint16_t* __restrict__ K = ql.K;
   const uint16_t* __restrict__ V = ql.V;
   const int32_t* __restrict__ kept = ql.kept;
@@ -81,7 +81,10 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __half* __restrict__ Ks = ql.Ks; __half* __restrict__ Kz = ql.Kz;
   __half* __restrict__ Vs = ql.Vs; __half* __restrict__ Vz = ql.Vz;
   const int L = ql.L, n = ql.n_idx, ns = ql.ns;
-  const int u = blockIdx.x, bh = blockIdx.y, tid = threadIdx.x, nthr = blockDim.x;
+  // two blocks per run of g kept tokens: an even block quantizes its key group, the odd one its value rows (each has
+  // a shorter chain of dependent memory round trips than one block doing both)
+  const int u = blockIdx.x >> 1, bh = blockIdx.y, tid = threadIdx.x, nthr = blockDim.x;
+  const bool key_part = (blockIdx.x & 1) == 0;
   const int ud = ql.u0 + u;                        // destination group
   const int wpg = g * BITS / 32;
 
@@ -89,7 +92,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __syncthreads();
   const uint16_t* Kh = K + (size_t)bh * L * D;
   const uint16_t* Vh = V + (size_t)bh * L * D;
-  for (int c = tid; c < g * (D / 8); c += nthr) {
+  for (int c = tid; key_part && c < g * (D / 8); c += nthr) {
     const int e = c / (D / 8), col = (c % (D / 8)) * 8;
     *reinterpret_cast<uint4*>(sK + e * D + col) =
         *reinterpret_cast<const uint4*>(Kh + (size_t)sidx[e] * D + col);
@@ -97,7 +100,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __syncthreads();
 
   // keys: channel d, tokens e = 0..g-1
-  for (int d = tid; d < D; d += nthr) {
+  for (int d = tid; key_part && d < D; d += nthr) {
     float mn = bf16_bits_to_f32(sK[d]), mx = mn;
     for (int e = 1; e < g; ++e) {
       const float x = bf16_bits_to_f32(sK[e * D + d]);
@@ -123,7 +126,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
 
   // values: token e, channel group v
   const int ngv = D / g;
-  for (int it = tid; it < g * ngv; it += nthr) {
+  for (int it = tid; !key_part && it < g * ngv; it += nthr) {
     const int e = it / ngv, v = it % ngv;
     const uint16_t* src = Vh + (size_t)sidx[e] * D + (size_t)v * g;
     float mn = INFINITY, mx = -INFINITY;
@@ -241,7 +244,7 @@ cudaError_t launch_gather_quantize(const void* K, const void* V, const int32_t* 
   tab.l[0] = QuantLayer{k, v, kept, static_cast<uint32_t*>(c.k_codes), static_cast<uint32_t*>(c.v_codes),
                         static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
                         static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, n, ns, 0};
-  return launch_quant_table<1>(c.bits, tab, dim3(n / g, BH, 1), D, g, st);
+  return launch_quant_table<1>(c.bits, tab, dim3(2 * (n / g), BH, 1), D, g, st);
 }
 
 cudaError_t launch_gather_quantize_layers(int n_layers, const void* const* K, const void* const* V,
@@ -264,7 +267,7 @@ cudaError_t launch_gather_quantize_layers(int n_layers, const void* const* K, co
                           static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, c.n_keep, cache_capacity(c), 0};
     max_groups = std::max(max_groups, c.n_keep / c.group);
   }
-  return launch_quant_table<QP_MAX_LAYERS>(c0.bits, tab, dim3(max_groups, c0.batch * c0.n_kv_heads, n_layers),
+  return launch_quant_table<QP_MAX_LAYERS>(c0.bits, tab, dim3(2 * max_groups, c0.batch * c0.n_kv_heads, n_layers),
                                            c0.head_dim, c0.group, st);
 }
 
@@ -318,11 +321,11 @@ cudaError_t launch_flush_tails(int n_layers, const int* which, const qp_cache* c
   if (n_layers == 1) {
     QuantTable<1> tab;
     fill(tab.l[0], which[0]);
-    return launch_quant_table<1>(c0.bits, tab, dim3(1, BH, 1), D, g, st);
+    return launch_quant_table<1>(c0.bits, tab, dim3(2, BH, 1), D, g, st);
   }
   QuantTable<QP_MAX_LAYERS> tab;
   for (int i = 0; i < n_layers; ++i) fill(tab.l[i], which[i]);
-  return launch_quant_table<QP_MAX_LAYERS>(c0.bits, tab, dim3(1, BH, n_layers), D, g, st);
+  return launch_quant_table<QP_MAX_LAYERS>(c0.bits, tab, dim3(2, BH, n_layers), D, g, st);
 }
 
 }  // namespace qp
