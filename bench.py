@@ -301,8 +301,8 @@ def run_gpu(args, wl):
     # ---- the same decode attention with one sequence per call (context for the batched figure)
     single_ms = None
     if per_call > 1:
-        reps = 64
-        for r in range(8):
+        reps = 512
+        for r in range(32):
             qp.decode_attn_layers(seqs[r % n_seq]["batches"][r % 8])
         s0, s1 = ev(), ev()
         s0.record(stream)
