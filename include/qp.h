@@ -181,8 +181,9 @@ qp_status qp_compress_layers(int n_layers, const void* const* K, const void* con
  * stream may overlap on the GPU: the library starts a call's first kernel before the
  * previous call has finished when this call reads none of the previous call's out
  * buffers (it checks q and the cache arrays against them), and alternates between
- * two halves of the workspace.  Results are as if the calls ran one after the other;
- * calls on different streams must not share a workspace.
+ * two halves of the workspace (calls of different sizes may share one workspace: where
+ * their halves would meet, the later call simply waits).  Results are as if the calls ran
+ * one after the other; calls on different streams must not share a workspace.
  */
 qp_status qp_decode_attn(const void* q, const qp_cache* cache /* host */, void* out, void* workspace,
                          size_t workspace_bytes, void* stream);
