@@ -250,6 +250,116 @@ def test_quantizer_error_bound_and_code_range(bits, g):
     assert np.all(f16_val(pk.k_zero) <= kmin)
 
 
+# The three tests below pin the stored-precision rules of one quantization group (Eq. 4 with
+# the scale and the zero point held in fp16): each fails if the oracle rounds the scale down or
+# to nearest, rounds the zero point up or to nearest, or breaks rounding ties away from zero.
+
+def _group_views(kb, vb, g):
+    """bf16 bit arrays [Bt,Hkv,L,D] -> float64 values per group, last axis = the group's elements:
+    keys [Bt,Hkv,L/g,D,g] (per channel over g tokens), values [Bt,Hkv,L,D/g,g] (per token)."""
+    Bt, Hkv, L, D = kb.shape
+    kg = bf16_val(kb).reshape(Bt, Hkv, L // g, g, D).transpose(0, 1, 2, 4, 3)
+    vg = bf16_val(vb).reshape(Bt, Hkv, L, D // g, g)
+    return kg, vg
+
+
+def _f16_floor(x: np.ndarray) -> np.ndarray:
+    """largest fp16 <= x (x float64), from numpy's own float16 rounding and nextafter"""
+    near = x.astype(np.float16)
+    lower = np.nextafter(near, np.float16(-np.inf))
+    return np.where(near.astype(np.float64) <= x, near, lower)
+
+
+def _f16_ceil(x: np.ndarray) -> np.ndarray:
+    near = x.astype(np.float16)
+    upper = np.nextafter(near, np.float16(np.inf))
+    return np.where(near.astype(np.float64) >= x, near, upper)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_stored_scale_is_smallest_fp16_not_below_the_exact_quotient(bits):
+    g, D, L = 32, 64, 256
+    k = RNG.standard_normal((1, 2, L, D)) * 3.0
+    v = RNG.standard_normal((1, 2, L, D))
+    pk, kb, vb, _ = _quant(k, v, bits, g)
+    kg, vg = _group_views(kb, vb, g)
+    qmax = (1 << bits) - 1
+    checked = 0
+    for vals, scale, zero in ((kg, pk.k_scale, pk.k_zero), (vg, pk.v_scale, pk.v_zero)):
+        quot = (vals.max(-1) - f16_val(zero)) / qmax          # float64, from the STORED zero point
+        want = _f16_ceil(quot)
+        got = scale.view(np.float16)
+        # a quotient within fp32 rounding of an fp16 value may legitimately land on either side
+        gap = np.abs(quot - want.astype(np.float64))
+        clear = (gap == 0) | (gap > 4e-7 * quot)          # exactly representable quotients are clear too
+        checked += int(clear.sum())
+        assert np.array_equal(got[clear], want[clear])
+        # never below the quotient (beyond fp32 rounding): the top element must not clip
+        assert np.all(got.astype(np.float64) >= quot * (1 - 2e-7))
+        # and strictly above it somewhere by a good part of an fp16 step: not round-to-nearest
+        assert np.any(got.astype(np.float64) > quot * (1 + 6e-4))
+    assert checked > 0.99 * (kg.shape[:-1][2] * kg.shape[3] * 2 + vg.shape[2] * vg.shape[3] * 2)
+
+
+@pytest.mark.parametrize("magnitude", [1e-6, 1e-7, 1e-9])
+def test_stored_zero_is_largest_fp16_not_above_the_minimum(magnitude):
+    # minima in and below the fp16 subnormal range (spacing 2^-24 = 6e-8): bf16 holds them
+    # exactly, fp16 does not, so the direction of the zero point's rounding shows
+    bits, g, D, L = 4, 32, 32, 64
+    k = RNG.standard_normal((1, 1, L, D)) * magnitude
+    v = RNG.standard_normal((1, 1, L, D)) * magnitude
+    k[0, 0, :, 0] = np.abs(k[0, 0, :, 0]) + magnitude        # an all-positive group: zero must not exceed min
+    pk, kb, vb, _ = _quant(k, v, bits, g)
+    kg, vg = _group_views(kb, vb, g)
+    inexact = 0
+    for vals, zero in ((kg, pk.k_zero), (vg, pk.v_zero)):
+        mn = vals.min(-1)
+        want = _f16_floor(mn)
+        got = zero.view(np.float16)
+        assert np.array_equal(got.view(np.uint16), want.view(np.uint16))     # bit patterns: -0.0 vs 0.0 too
+        assert np.all(got.astype(np.float64) <= mn)
+        inexact += int((got.astype(np.float64) < mn).sum())
+    assert inexact > 0          # the case really exercises the rounding
+    # scale and codes are computed from the STORED zero point, not from the exact minimum (the two
+    # differ by up to one fp16 subnormal step here, a good part of a scale step)
+    qmax = (1 << bits) - 1
+    for vals, codes, scale, zero in ((kg, unpack(pk.k_codes, bits, g), pk.k_scale, pk.k_zero),
+                                     (vg, unpack(pk.v_codes, bits, g), pk.v_scale, pk.v_zero)):
+        zf, sf = f16_val(zero), f16_val(scale)
+        quot = (vals.max(-1) - zf) / qmax
+        gap = np.abs(quot - _f16_ceil(quot).astype(np.float64))
+        clear = (gap == 0) | (gap > 4e-7 * quot)
+        assert np.array_equal(scale.view(np.float16)[clear], _f16_ceil(quot)[clear])
+        live = sf > 0
+        ratio = (vals - zf[..., None])[live] / sf[live][:, None]
+        want = np.clip(np.rint(ratio), 0, qmax)
+        off_tie = np.abs(ratio - np.floor(ratio) - 0.5) > 1e-4
+        assert np.array_equal(codes[live][off_tie], want[off_tie].astype(np.uint32))
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_codes_round_half_to_even(bits):
+    # a group holding 0 and 2^B - 1 has zero 0 and scale 1 exactly; its other elements are the
+    # half-integers 0.5, 1.5, 2.5, ... (bf16-exact below 128), whose quotients are exact ties
+    g, D, L = 32, 32, 32
+    qmax = (1 << bits) - 1
+    halves = (np.arange(g - 2) % qmax) + 0.5                 # 0.5 .. qmax - 0.5, cyclic
+    if bits == 8:
+        halves = (np.arange(g - 2) * 4 % 127) + 0.5          # stay below 128 where x.5 is bf16-exact
+    elems = np.concatenate([[0.0, float(qmax)], halves])
+    assert np.array_equal(bf16_val(bf16_bits(elems)), elems)
+    k = np.broadcast_to(elems[:, None], (1, 1, L, D)).copy()       # key groups run along tokens
+    v = np.broadcast_to(elems[None, :], (1, 1, L, D)).copy()       # value groups run along channels
+    pk, _, _, _ = _quant(k, v, bits, g)
+    assert np.all(f16_val(pk.k_scale) == 1.0) and np.all(f16_val(pk.k_zero) == 0.0)
+    want = np.concatenate([[0, qmax], 2 * np.floor((halves + 0.5) / 2)]).astype(np.uint32)   # nearest even
+    assert np.any(want[2:] != np.floor(halves) + 1)          # differs from ties-away somewhere
+    kc = unpack(pk.k_codes, bits, g)                         # [1,1,1,D,g]
+    vc = unpack(pk.v_codes, bits, g)                         # [1,1,L,1,g]
+    assert np.array_equal(kc[0, 0, 0], np.broadcast_to(want, (D, g)))
+    assert np.array_equal(vc[0, 0, :, 0], np.broadcast_to(want, (L, g)))
+
+
 def test_quantizer_dequant_formula_against_independent_unpack():
     bits, g, D = 4, 32, 64
     k = RNG.standard_normal((1, 1, 64, D)); v = RNG.standard_normal((1, 1, 64, D))
