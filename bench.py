@@ -193,6 +193,7 @@ def run_gpu(args, wl):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     qp.lib()
+    qp.decode_overlap(not args.no_overlap)     # the decode steps are independent and nothing else runs between them
 
     n_seq, n_layers, n_dec = args.sequences, wl.n_layers, wl.decode_steps
     # sequences whose layers share one qp_decode_attn_layers call (independent problems, as in continuous batching)
@@ -337,6 +338,7 @@ def run_gpu(args, wl):
         side.wait_stream(stream)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
+            qp.decode_overlap(not args.no_overlap)
             chain()
             torch.cuda.synchronize()
             with torch.cuda.graph(graph, stream=side):
@@ -547,6 +549,7 @@ def main():
     ap.add_argument("--no-compress-layers", action="store_true", help="skip the qp_compress_layers figure")
     ap.add_argument("--no-generation", action="store_true", help="skip the append + decode generation-loop figure")
     ap.add_argument("--no-layer-chain", action="store_true", help="skip the layer-by-layer / CUDA-graph figures")
+    ap.add_argument("--no-overlap", action="store_true", help="decode calls in plain stream order")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]

@@ -14,7 +14,12 @@
  *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream)
  *     and buffers must stay alive until the stream has passed that point.
  *   - bf16 / fp16 tensors are raw 16-bit patterns, row-major and contiguous, base
- *     addresses 16-byte aligned.  Inputs must be finite with |x| <= 65504.
+ *     addresses 16-byte aligned.  Inputs must be finite.  Magnitudes: K, V and Q_win of the
+ *     prefill-side calls up to 65504 (the fp16 range of the stored scale and zero).  The decode
+ *     calls multiply in fp16 on the tensor cores (query x key scale, softmax weight x value scale)
+ *     and need   max|q| * max|K| <= 2^19   and   max|V| <= 4096   over the tensors of a call, K and V
+ *     being the values that were quantized into the cache (at 16 bit: max|q| <= 65504 only).
+ *     Beyond that a product may overflow fp16 and the output holds inf or NaN; nothing checks it.
  *   - Host-checkable errors are returned before anything is launched and leave
  *     the outputs untouched.  Launch failures are reported as QP_ERR_CUDA from
  *     cudaGetLastError() without synchronising.
@@ -118,6 +123,12 @@ size_t qp_decode_workspace_bytes(const qp_cache* cache /* host */);
  *   scores[j] = (sum_{|t| <= (pool-1)/2} vote[j+t], zero outside [0,P)) / pool
  * Q_win bf16 [Bt,Hq,w,D], K bf16 [Bt,Hkv,L,D] (device) -> scores fp32 [Bt,Hkv,P] (device).
  * pool must be odd (1 = no pooling) and at most 65.
+ * Error word: the score sweeps wait on hardware barriers (copies into shared memory, tensor-core
+ * completion) with a bounded number of polls.  A block whose wait runs out stops, and the 32-bit
+ * word at byte offset qp_compress_workspace_bytes(...) - 256 of the workspace becomes 1; the
+ * scores (and everything qp_compress_layer derives from them) are then invalid.  The word is
+ * cleared at the start of every qp_window_scores / qp_compress_layer(s) call (stream-ordered) and
+ * can be read by the caller once the stream has passed the call.  It is 0 in every correct run.
  */
 qp_status qp_window_scores(const void* Q_win, const void* K, int batch, int n_q_heads, int n_kv_heads,
                            int head_dim, int L, int w, int pool, float* scores, void* workspace,
@@ -177,16 +188,33 @@ qp_status qp_compress_layers(int n_layers, const void* const* K, const void* con
  * cache of Eq. 5): out[b,h,:] = softmax_t(q[b,h].K'[t] / sqrt(D)) V' over the n kept
  * tokens of KV head h / G, no mask.  q, out bf16 [Bt,Hq,D] (device).  The token
  * range is split across workers and the partial results merged; workspace (device,
- * 16-byte aligned, contents irrelevant) holds the partials.  Consecutive calls on one
- * stream may overlap on the GPU: the library starts a call's first kernel before the
- * previous call has finished when this call reads none of the previous call's out
- * buffers (it checks q and the cache arrays against them), and alternates between
- * two halves of the workspace (calls of different sizes may share one workspace: where
- * their halves would meet, the later call simply waits).  Results are as if the calls ran
- * one after the other; calls on different streams must not share a workspace.
+ * 16-byte aligned, contents irrelevant) holds the partials.  Calls run in stream order
+ * unless qp_decode_overlap has been enabled for the stream (below).  Calls on different
+ * streams must not share a workspace.
  */
 qp_status qp_decode_attn(const void* q, const qp_cache* cache /* host */, void* out, void* workspace,
                          size_t workspace_bytes, void* stream);
+
+/*
+ * Lets consecutive decode calls on `stream` overlap on the GPU (enable != 0) or returns the stream
+ * to plain stream order (0, the default).  No counterpart in the paper: a launch-level measure.
+ * Enabled, a decode call's attention kernel is launched so that it may begin while the previous
+ * decode call's merge step still runs, which hides the launch gap and the merge step between the
+ * calls of a decode loop.  The library keeps this safe against its own calls: it starts a call early
+ * only if the call reads none of the previous decode call's out buffers (q and the cache arrays are
+ * checked against them), alternates between two halves of the workspace (calls of different sizes
+ * may share one workspace: where their halves would meet, the later call simply waits), and falls
+ * back to stream order after any of its calls that writes a cache.  Its kernels guarantee that at
+ * most two consecutive decode calls are in flight at a time.  Results are as if the calls ran one
+ * after the other.
+ * What the caller promises while it is enabled: whatever ELSE is enqueued on the stream between two
+ * decode calls (kernels or copies that are not calls of this library) writes nothing that the later
+ * call reads (its q, its cache arrays).  A loop that computes each layer's q just before attending
+ * with it must leave the setting off.  Host call, takes effect from the next decode call on the
+ * stream; the setting is per (device, stream) and is forgotten, falling back to the default, if more
+ * than 256 streams are in use.
+ */
+qp_status qp_decode_overlap(void* stream, int enable);
 
 /*
  * The same decode attention for n_layers independent layers in one pair of

@@ -13,9 +13,11 @@ using namespace qp;
 
 namespace {
 
-// What the last decode call on each (device, stream) wrote through its merge kernel.  The attention kernel of
-// the next call on that stream is allowed to start while that merge kernel still runs (programmatic dependent
-// launch) only if none of its inputs overlaps those outputs; otherwise it is launched in plain stream order.
+// What the last decode call on each (device, stream) wrote through its merge kernel.  On a stream for which the
+// caller has enabled it (qp_decode_overlap), the attention kernel of the next call is allowed to start while that
+// merge kernel still runs (programmatic dependent launch) if none of its inputs overlaps those outputs; otherwise,
+// and on every other stream, it is launched in plain stream order.  The kernels' own protocol (pdl_gate in
+// qp_mma.cuh) guarantees that only the previous call can still be running then, so one call of history is enough.
 // Host bookkeeping only: a few sorted address ranges per stream.
 class PrevOutputs {
  public:
@@ -28,8 +30,11 @@ class PrevOutputs {
   // ws_base / half_bytes: this call's partial records go to [ws_base + parity * half_bytes, + half_bytes); if that
   // area meets the one the previous call's merge may still be reading (calls of different sizes place their halves
   // differently), the call must not overlap the previous one either
+  // two_halves: the launch is of the kind that alternates between workspace halves and takes part in the
+  // overlap; the other kind (the chunked kernels) always writes [ws_base, ws_base + half_bytes), runs in plain
+  // stream order, and so does the call after it
   Decision check_and_record(int device, cudaStream_t st, const std::vector<Range>& reads, std::vector<Range>& writes,
-                            uintptr_t ws_base, size_t half_bytes) {
+                            uintptr_t ws_base, size_t half_bytes, bool two_halves) {
     std::sort(writes.begin(), writes.end());
     // after sorting by begin, writes[i].second becomes the largest end among writes[0..i]: a read [b, e) meets
     // one of the writes that begin before e exactly when that running maximum exceeds b
@@ -37,10 +42,10 @@ class PrevOutputs {
     std::lock_guard<std::mutex> lock(mu_);
     const auto key = std::make_pair(device, st);
     auto it = prev_.find(key);
-    Decision dec{!forgot_, 0};                      // a stream seen for the first time has no earlier decode kernel
+    Decision dec{false, 0};                         // overlap is opt-in per stream
     if (it != prev_.end()) {
-      dec.overlap = !it->second.barrier;
-      dec.parity = it->second.parity ^ 1;
+      dec.overlap = it->second.allow && !it->second.barrier && two_halves;
+      dec.parity = two_halves ? it->second.parity ^ 1 : 0;
       const std::vector<Range>& w = it->second.outs;
       for (const Range& r : reads) {
         if (!dec.overlap) break;
@@ -48,10 +53,8 @@ class PrevOutputs {
                                          [](const Range& x, uintptr_t end) { return x.first < end; });
         if (lo != w.begin() && (lo - 1)->second > r.first) { dec.overlap = false; break; }
       }
-    } else if (prev_.size() >= kMaxStreams) {       // bounded memory: forget, and stop trusting absence
+    } else if (prev_.size() >= kMaxStreams) {       // bounded memory: forget (the opt-ins too: plain order is always safe)
       prev_.clear();
-      forgot_ = true;
-      dec.overlap = false;
     }
     Entry& e = prev_[key];
     const Range mine{ws_base + (dec.parity ? half_bytes : 0), ws_base + (dec.parity ? half_bytes : 0) + half_bytes};
@@ -59,7 +62,7 @@ class PrevOutputs {
     e.scratch = mine;
     e.outs.swap(writes);
     e.parity = dec.parity;
-    e.barrier = false;
+    e.barrier = !two_halves;
     return dec;
   }
   // Another kernel of the library has been enqueued on this stream that writes arrays a decode call reads
@@ -67,11 +70,20 @@ class PrevOutputs {
   // in plain stream order.
   void barrier(int device, cudaStream_t st) {
     std::lock_guard<std::mutex> lock(mu_);
-    if (prev_.size() >= kMaxStreams && prev_.find(std::make_pair(device, st)) == prev_.end()) {
-      prev_.clear();
-      forgot_ = true;
-    }
+    if (prev_.size() >= kMaxStreams && prev_.find(std::make_pair(device, st)) == prev_.end()) prev_.clear();
     prev_[std::make_pair(device, st)].barrier = true;
+  }
+  bool allowed(int device, cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(mu_);
+    const auto it = prev_.find(std::make_pair(device, st));
+    return it != prev_.end() && it->second.allow;
+  }
+  void allow(int device, cudaStream_t st, bool on) {
+    std::lock_guard<std::mutex> lock(mu_);
+    if (prev_.size() >= kMaxStreams && prev_.find(std::make_pair(device, st)) == prev_.end()) prev_.clear();
+    Entry& e = prev_[std::make_pair(device, st)];
+    e.allow = on;
+    e.barrier = true;                               // whatever was enqueued before the switch is unknown
   }
 
  private:
@@ -80,11 +92,11 @@ class PrevOutputs {
     Range scratch{0, 0};     // where the last call's partial records live
     int parity = 0;
     bool barrier = false;
+    bool allow = false;      // the caller's qp_decode_overlap setting for this stream
   };
   static constexpr size_t kMaxStreams = 256;
   std::mutex mu_;
   std::map<std::pair<int, cudaStream_t>, Entry> prev_;
-  bool forgot_ = false;
 };
 PrevOutputs g_prev_outputs;
 
@@ -348,10 +360,14 @@ qp_status decode_layers_uniform(int n_layers, const void* const* q, const qp_cac
   if (any_tail)
     for (int l = 0; l < n_layers; ++l) ttab.l[l] = TailLayer{tails[l].k_tail, tails[l].v_tail, tails[l].n_tail, 0};
   const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
-  const size_t need = decode_plan(tab, d);
+  int device = 0;
+  const bool have_device = cudaGetDevice(&device) == cudaSuccess;   // (size checks below work without one)
+  const size_t need = decode_plan(tab, d, have_device && g_prev_outputs.allowed(device, static_cast<cudaStream_t>(stream)));
   if (workspace_bytes < need) return QP_ERR_WORKSPACE;
   if (check_only) return QP_OK;
-  const size_t half_bytes = decode_mma_supported(d) ? decode_workspace_layout(tab, d).record_bytes : need;
+  if (!have_device) return QP_ERR_CUDA;
+  const bool two_halves = decode_mma_supported(d);
+  const size_t half_bytes = two_halves ? decode_workspace_layout(tab, d).record_bytes : need;
   // everything the attention kernel reads before it waits for the stream's previous kernel, and what this
   // call's merge kernel writes
   std::vector<PrevOutputs::Range> reads, writes;
@@ -371,11 +387,9 @@ qp_status decode_layers_uniform(int n_layers, const void* const* q, const qp_cac
     }
     writes.push_back(range_of(out[l], qo_bytes));
   }
-  int device = 0;
-  if (cudaGetDevice(&device) != cudaSuccess) return QP_ERR_CUDA;
   const PrevOutputs::Decision dec =
       g_prev_outputs.check_and_record(device, static_cast<cudaStream_t>(stream), reads, writes,
-                                      reinterpret_cast<uintptr_t>(workspace), half_bytes);
+                                      reinterpret_cast<uintptr_t>(workspace), half_bytes, two_halves);
   return launch_decode(tab, d, workspace, dec.parity, static_cast<cudaStream_t>(stream), dec.overlap,
                        any_tail ? &ttab : nullptr) == cudaSuccess
              ? QP_OK : QP_ERR_CUDA;
@@ -421,6 +435,13 @@ qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const q
 qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches, void* const* out,
                                 void* workspace, size_t workspace_bytes, void* stream) {
   return qp_decode_attn_tail_layers(n_layers, q, caches, nullptr, out, workspace, workspace_bytes, stream);
+}
+
+qp_status qp_decode_overlap(void* stream, int enable) {
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) return QP_ERR_CUDA;
+  g_prev_outputs.allow(device, static_cast<cudaStream_t>(stream), enable != 0);
+  return QP_OK;
 }
 
 qp_status qp_decode_attn_tail(const void* q, const qp_cache* cache, const qp_tail* tail, void* out, void* workspace,

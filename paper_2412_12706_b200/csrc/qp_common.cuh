@@ -150,7 +150,9 @@ struct TailTable {
 constexpr int kMaxDecodeWorkers = QP_MAX_DECODE_WORKERS;
 // Chooses the decomposition for the layers in tab (n and pointers already set), fills chunk / part_base or
 // tile_base / total_tiles / n_workers and returns the bytes of partial records the launch needs.
-size_t decode_plan(DecTable& tab, const DecDims& d);
+// paired: the stream lets consecutive calls overlap (two calls share the GPU most of the time), so a small launch
+// does better with fewer, longer-lived workers; alone on the GPU it wants as many as it can feed.
+size_t decode_plan(DecTable& tab, const DecDims& d, bool paired);
 // Upper bound of decode_plan's result for one layer of n_keep tokens, whatever else is in the launch.
 size_t decode_workspace_bound(const DecDims& d, int n_keep);
 // Workspace of the tensor-core kernels: two areas of partial records, used by alternate calls (parity), so that
@@ -173,7 +175,7 @@ int sm_count();   // SMs of the current device (cached)
 // tensor-core split-K kernel and its merge
 bool decode_mma_supported(const DecDims& d);
 int decode_mma_workers_per_sm(const DecDims& d);     // workers (see DecTable::n_workers) resident per SM
-int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles);   // small launches: fewer workers, not emptier ones
+int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles, bool paired);   // small launches: fewer workers, not emptier ones
 int decode_mma_wide_workers_per_sm(const DecDims& d, int* min_tiles);
 cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st,
                               bool overlap_prev, const TailTable* tails = nullptr);

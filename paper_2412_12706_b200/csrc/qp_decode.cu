@@ -220,7 +220,7 @@ int chunk_tokens(long long total_tokens) {
 
 }  // namespace
 
-size_t decode_plan(DecTable& tab, const DecDims& d) {
+size_t decode_plan(DecTable& tab, const DecDims& d, bool paired) {
   const int BH = d.Bt * d.Hkv;
   if (decode_mma_supported(d)) {
     long long T = 0;
@@ -240,7 +240,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d) {
       tab.wide = 1;
     }
     if (W > kMaxDecodeWorkers) W = kMaxDecodeWorkers;
-    const int tmin = decode_mma_tiles_per_worker_min(d, T);
+    const int tmin = decode_mma_tiles_per_worker_min(d, T, paired);
     if (!tab.wide && W > (T + tmin - 1) / tmin) W = (T + tmin - 1) / tmin;
     if (W < 1) W = 1;
     while (W > 1 && T * W >= (1ll << 31)) W /= 2;               // the merge kernel's range arithmetic is 32-bit

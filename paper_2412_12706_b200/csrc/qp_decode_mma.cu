@@ -84,7 +84,6 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);       // provably warp-uniform: cursors stay in uniform registers
   const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
-  asm volatile("griddepcontrol.launch_dependents;\n" ::);     // the merge grid may start to become resident
   // Every warp is a worker of its own: a contiguous range of the flat tile sequence, a private copy ring,
   // one partial record per head it touches.  Warps of a block share nothing and never synchronise.
   const int wk = blockIdx.x * DM_WARPS + warp;
@@ -197,8 +196,10 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   };
   clear_state();
   bool fresh = true;
+  const int gate = gate_tile(total);
 
   for (int it = 0; it < total; ++it) {
+    if (it == gate) pdl_gate();                                 // see qp_mma.cuh: wait, then let the merge grid in
     if (fresh) {
       fresh = false;
       const DecLayer& ly = tab.l[c_li];
@@ -400,10 +401,8 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
     }
   }
   // This kernel may have started while the previous call's merge kernel was still reading its records: alternate
-  // calls use alternate halves of the workspace, so nothing here had to wait for it.  The call after this one
-  // uses the previous call's half again; it starts its writes only after this grid has ended, and waiting here
-  // makes that imply that the previous call's merge has ended as well.
-  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  // calls use alternate halves of the workspace, and the call before the previous one had ended before this
+  // kernel could start (pdl_gate), so no record store had to wait.
 }
 
 // S5 for the decomposition above: head (layer, batch, KV head) was touched by the blocks
@@ -412,7 +411,7 @@ decode_mma4_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
 // programmatic dependent of the attention kernel: its blocks may become resident while that kernel
 // drains and wait at griddepcontrol.wait until its records are complete and visible.  It passes the
 // permission on at once, so that the next call's attention kernel can fill the machine while this
-// one runs; that kernel reads none of this one's outputs and waits before it overwrites the records.
+// one runs; that kernel reads none of this one's outputs and writes the other half of the workspace.
 constexpr int MG_WARPS = 4;
 // At most 32 registers per thread, so that a block fits beside the resident blocks of the attention kernel.  A
 // small launch (up to two blocks of work per SM) uses at most one block per SM: the whole grid is then resident
@@ -548,9 +547,19 @@ int decode_mma_workers_per_sm(const DecDims& d) {
 // The 8-bit kernel behaves alike (151 MB calls of 16384 tiles: 4.22 / 4.02 / 5.08 / 2.76 TB/s with 4 / 16 / 32 / 64);
 // the 2-bit and 16-bit kernels showed no gain (4.96 / 4.78 / 4.87 / 4.65 and 5.60 / 5.61 / 5.60 / 4.81 TB/s) and keep
 // four tiles per worker.
-int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles) {
+#ifndef QP_TMIN_BIG
+#define QP_TMIN_BIG 32
+#endif
+#ifndef QP_TMIN_SMALL
+#define QP_TMIN_SMALL 16
+#endif
+#ifndef QP_TMIN_SOLO
+#define QP_TMIN_SOLO 4
+#endif
+int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles, bool paired) {
+  if (!paired) return QP_TMIN_SOLO;
   if (d.bits != 4 && d.bits != 8) return 4;
-  return total_tiles / 32 >= 256 ? 32 : 16;
+  return total_tiles / QP_TMIN_BIG >= 256 ? QP_TMIN_BIG : QP_TMIN_SMALL;
 }
 // Workers per SM of the wider build of this shape's kernel and the tiles per worker from which it pays
 // (0: the shape has one build only).

@@ -45,7 +45,6 @@ decode_mma16_kernel(const __grid_constant__ DecTable tab, const DecDims dm, floa
   const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
   const SkOwner sk{tab.total_tiles, tab.n_workers};
   const int cta = blockIdx.x;
-  asm volatile("griddepcontrol.launch_dependents;\n" ::);
   long long cur = sk.start(cta);
   const long long f_end = sk.start(cta + 1);
 
@@ -109,7 +108,9 @@ decode_mma16_kernel(const __grid_constant__ DecTable tab, const DecDims dm, floa
 #pragma unroll
       for (int x = 0; x < 4; ++x) accO[j][x] = 0.f;
 
+    const bool last_seg = cur + n_tiles >= f_end;
     for (int it = 0; it < n_my; ++it) {
+      if (last_seg && it == n_my - 1) pdl_gate();               // see qp_mma.cuh (a warp without tiles leaves it to the others)
       __syncwarp();
       if (it + D16_STAGES - 1 < n_my)
         issue_tile(tile_begin + warp + D16_WARPS * (it + D16_STAGES - 1), (it + D16_STAGES - 1) % D16_STAGES);
@@ -210,9 +211,6 @@ decode_mma16_kernel(const __grid_constant__ DecTable tab, const DecDims dm, floa
     cur += n_tiles;
     if (bh == BH - 1 && tile_begin + n_tiles == tph) ++li;
   }
-  // (see the 4-bit kernel: a call may start before the previous call's merge kernel has ended; the call after it
-  // relies on this grid not ending before that kernel has)
-  asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
 template <int D>

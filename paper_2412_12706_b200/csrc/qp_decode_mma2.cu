@@ -91,7 +91,6 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const int e = g >> 2, o = g & 3;                              // variant bit and unit index of this lane's MMA rows
   const bool lane_valid = e == (t >> 1);                        // this lane's accumulator entries are an e = e' block
   const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
-  asm volatile("griddepcontrol.launch_dependents;\n" ::);
   const int wk = blockIdx.x * D2_WARPS + warp;
   if (wk >= tab.n_workers) return;
   const SkOwner sk{tab.total_tiles, tab.n_workers};
@@ -216,9 +215,13 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
         for (int x = 0; x < 4; ++x) accO[v][mt][x] = 0.f;
   };
   clear_state();
-  bool fresh = true;
+  bool fresh = true, gated = false;
 
   while (c_left > 0) {
+    if (!gated && c_left <= total - gate_tile(total)) {
+      gated = true;
+      pdl_gate();
+    }
     if (fresh) {
       fresh = false;
       const DecLayer& ly = tab.l[c_li];
@@ -425,9 +428,6 @@ decode_mma2_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       }
     }
   }
-  // (see the 4-bit kernel: a call may start before the previous call's merge kernel has ended; the call after it
-  // relies on this grid not ending before that kernel has)
-  asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
 template <int D>

@@ -54,7 +54,6 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);       // provably warp-uniform
   const int G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv;
-  asm volatile("griddepcontrol.launch_dependents;\n" ::);
   // every warp is a worker of its own (see the 4-bit kernel): contiguous tile range, private copy ring
   const int wk = blockIdx.x * D8_WARPS + warp;
   if (wk >= tab.n_workers) return;
@@ -162,8 +161,10 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
   };
   clear_state();
   bool fresh = true;
+  const int gate = gate_tile(total);
 
   for (int it = 0; it < total; ++it) {
+    if (it == gate) pdl_gate();                                 // see qp_mma.cuh
     if (fresh) {
       fresh = false;
       const DecLayer& ly = tab.l[c_li];
@@ -348,9 +349,6 @@ decode_mma8_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float
       }
     }
   }
-  // (see the 4-bit kernel: a call may start before the previous call's merge kernel has ended; the call after it
-  // relies on this grid not ending before that kernel has)
-  asm volatile("griddepcontrol.wait;\n" ::: "memory");
 }
 
 template <int D>

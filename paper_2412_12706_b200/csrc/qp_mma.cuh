@@ -40,6 +40,35 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Order of consecutive decode calls on one stream when they are allowed to overlap (programmatic dependent
+// launch).  Kernels of a stream: A_N (attention of call N), M_N (its merge), optionally P (rows of an appended
+// token), A_{N+1}, ...  Every kernel executes griddepcontrol.wait before it ends, so "X has ended" implies
+// "everything before X has ended".  The merge and append kernels pass the launch permission on as soon as they
+// start; an attention kernel passes it on only AFTER its own wait has returned (pdl_gate), a few tiles before
+// its range ends.  So A_{N+1} can begin only when some thread of A_N is past its wait, i.e. when the kernel
+// before A_N (M_{N-1}, or an append after it) and with it everything of call N-1 and earlier has ended:
+// at most A_N, M_N (and an append) and A_{N+1} are in flight together, however small the grids are.  A_{N+1}
+// therefore needs to be checked only against call N (the host does: it reads none of call N's outputs) and
+// writes the workspace half that call N-1, which has ended, used.
+__device__ __forceinline__ void pdl_gate() {
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+}
+// the gate sits this many tiles before the end of a worker's range (or at its start, for shorter ranges): late
+// enough that the previous call's merge has normally ended by then, early enough to hide the next launches
+#ifndef QP_GATE_TILES
+#define QP_GATE_TILES 2
+#endif
+#ifndef QP_GATE_EIGHTHS
+#define QP_GATE_EIGHTHS 4
+#endif
+constexpr int kGateTiles = QP_GATE_TILES;
+// first tile a worker computes AFTER its gate, for a range of `total` tiles
+__device__ __forceinline__ int gate_tile(int total) {
+  const int lead = max(kGateTiles, (total * QP_GATE_EIGHTHS) >> 3);
+  return total > lead ? total - lead : 0;
+}
+
 // Work decomposition ("stream-K" over tokens): the 32-token tiles of all (layer, batch, KV head)
 // triples form one flat sequence of T tiles; block w of W owns the contiguous range
 // [w*T/W, (w+1)*T/W), so every block streams the same number of bytes (+-1 tile), the grid is one

@@ -3,6 +3,9 @@
 // The split-K decode kernels need scratch for the per-split partial results.  The other
 // entry points take that scratch from the caller; this one keeps it in a fixed array that is
 // part of the library image, so the caller passes only inputs and outputs.
+#include <algorithm>
+#include <atomic>
+
 #include "qp_common.cuh"
 
 namespace {
@@ -14,17 +17,18 @@ static __device__ __align__(256) unsigned char g_static_scratch[QP_STATIC_SCRATC
 constexpr int kMaxDevices = 64;
 // Device address of g_static_scratch per CUDA device.  The array's name is only a host-side
 // handle in host code; the address a kernel can use must be asked for, with that device current.
-void* g_scratch_addr[kMaxDevices] = {};
+// Filled on the first call on each device; host threads that race on a first call all store the same value.
+std::atomic<void*> g_scratch_addr[kMaxDevices] = {};
 
 qp_status static_scratch(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return QP_ERR_CUDA;
-  if (!g_scratch_addr[dev]) {
-    void* p = nullptr;
+  void* p = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return QP_ERR_CUDA;
-    g_scratch_addr[dev] = p;
+    g_scratch_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return QP_OK;
 }
 
@@ -40,7 +44,8 @@ extern "C" qp_status qp_decode_attn_static(const void* q, const qp_cache* cache,
   qp::DecTable plan;
   plan.n_layers = 1;
   plan.l[0].n = cache->n_keep;
-  const size_t need = qp::decode_plan(plan, d);   // the same plan qp_decode_attn makes for this cache
+  // the plans qp_decode_attn may make for this cache (it depends on the stream's overlap setting)
+  const size_t need = std::max(qp::decode_plan(plan, d, false), qp::decode_plan(plan, d, true));
   if (need > (size_t)QP_STATIC_SCRATCH_BYTES) return QP_ERR_WORKSPACE;
   void* scratch = nullptr;
   const qp_status s = static_scratch(&scratch);

@@ -25,7 +25,7 @@ EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_work
            "qp_decode_workspace_bytes", "qp_window_scores", "qp_select_topk", "qp_gather_quantize",
            "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static",
            "qp_cache_layout_cap", "qp_append_kv", "qp_append_kv_layers", "qp_decode_attn_tail",
-           "qp_decode_attn_tail_layers", "qp_compress_layers"]
+           "qp_decode_attn_tail_layers", "qp_compress_layers", "qp_decode_overlap"]
 
 
 class QpError(RuntimeError):
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.qp_decode_attn_tail.argtypes = [p, cp, tp, p, p, sz, p]
         L.qp_decode_attn_tail_layers.restype = i
         L.qp_decode_attn_tail_layers.argtypes = [i, ctypes.POINTER(p), cp, tp, ctypes.POINTER(p), p, sz, p]
+        L.qp_decode_overlap.restype = i
+        L.qp_decode_overlap.argtypes = [p, i]
         _lib = L
     return _lib
 
@@ -302,6 +304,12 @@ def decode_attn(q: torch.Tensor, cache: Cache, out: torch.Tensor | None = None,
     return out
 
 
+def decode_overlap(enable: bool) -> None:
+    """qp_decode_overlap for torch's current stream: let consecutive decode calls on it overlap on the GPU
+    (see include/qp.h for what the caller promises while it is on).  Off by default."""
+    _check(lib().qp_decode_overlap(_stream(), 1 if enable else 0), "qp_decode_overlap")
+
+
 class LayerBatch:
     """Marshalled host arrays for ``qp_decode_attn_layers`` (built once, reused every step)."""
 
@@ -430,6 +438,7 @@ qp_compress_layers = compress_layers
 qp_decode_attn = decode_attn
 qp_decode_attn_layers = decode_attn_layers
 qp_decode_attn_static = decode_attn_static
+qp_decode_overlap = decode_overlap
 qp_cache_layout_cap = cache_layout_cap
 qp_append_kv = append_kv
 qp_append_kv_layers = append_kv_layers

@@ -318,10 +318,11 @@ def test_same_bits_every_run_and_no_write_outside_the_outputs(bits):
         assert torch.equal(a, b)
 
 
-def test_calls_of_different_sizes_may_share_one_workspace():
-    """Consecutive decode calls on one stream overlap on the GPU and alternate between two halves of the workspace,
-    whose boundary depends on the call's size: calls of different sizes on ONE workspace must still give the results
-    of calls with workspaces of their own."""
+@pytest.mark.parametrize("overlap", [False, True])
+def test_calls_of_different_sizes_may_share_one_workspace(overlap):
+    """Consecutive decode calls on one stream may overlap on the GPU (when enabled) and alternate between two halves
+    of the workspace, whose boundary depends on the call's size: calls of different sizes on ONE workspace must still
+    give the results of calls with workspaces of their own."""
     shapes = [(4, 2048), (2, 512), (8, 1024), (4, 256), (16, 512), (4, 4096)]
     caches, qs, refs = [], [], []
     for i, (bits, n) in enumerate(shapes):
@@ -331,14 +332,18 @@ def test_calls_of_different_sizes_may_share_one_workspace():
         c, _ = qp.compress_layer(k.to(DEV), v.to(DEV), qw.to(DEV), wl.budget_bits, bits, wl.group, wl.pool)
         caches.append(c)
         qs.append(synth.make_q_dec(wl, i, 0).to(DEV))
+        qp.decode_overlap(overlap)            # (a call's split over workers depends on the setting)
         refs.append(qp.decode_attn(qs[-1], c))
         torch.cuda.synchronize()
+        qp.decode_overlap(False)
     ws = qp.new_decode_workspace(max(qp.decode_workspace_bytes(c) for c in caches), DEV)
     outs = [[torch.empty_like(q) for q in qs] for _ in range(5)]
+    qp.decode_overlap(overlap)
     for rep in range(5):                                         # back to back, no synchronisation in between
         for i in range(len(shapes)):
             qp.decode_attn(qs[i], caches[i], outs[rep][i], ws)
     torch.cuda.synchronize()
+    qp.decode_overlap(False)
     for rep in range(5):
         for i in range(len(shapes)):
             assert torch.equal(outs[rep][i], refs[i]), (rep, i, shapes[i])

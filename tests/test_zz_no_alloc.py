@@ -41,6 +41,8 @@ def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
 
 
 def test_static_scratch_rejects_oversized_cache_without_launching():
+    # 8 query heads per KV head at 2 bits take the chunked kernel, whose scratch is one record per
+    # (batch x KV head, token split, query head of the group):
     # 1024 (batch x KV head) pairs x 2 splits x 8 heads x 130 floats = 8.5 MB > 4 MiB
     c = qp.cache_layout(128, 64, 8, 128, 2, 32, 4096)
     fake = 0x10000   # aligned, never dereferenced: the size check comes before any launch
