@@ -129,6 +129,7 @@ struct DecTable {
   int chunk;        // chunked kernel: tokens per split
   int total_tiles;  // flat-range kernel: tiles of all layers and heads
   int n_workers;    // flat-range kernel: workers (blocks or warps, by kernel), each owning total_tiles / n_workers consecutive tiles
+  int paired;       // flat-range kernel: 1 = planned for a stream on which consecutive calls overlap (see decode_plan)
   int wide;         // flat-range kernel: 1 = the build with more resident workers per SM (long ranges), see decode_plan
   DecLayer l[QP_MAX_LAYERS];
 };

@@ -231,6 +231,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d, bool paired) {
     }
     long long W = (long long)sm_count() * decode_mma_workers_per_sm(d);
     tab.wide = 0;
+    tab.paired = paired ? 1 : 0;
     int wide_min = 0;
     const long long Ww = (long long)sm_count() * decode_mma_wide_workers_per_sm(d, &wide_min);
     const long long merge_blocks = ((long long)d.Bt * d.Hq * tab.n_layers + 3) / 4;
@@ -252,7 +253,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d, bool paired) {
   long long total_tokens = 0;
   for (int l = 0; l < tab.n_layers; ++l) total_tokens += (long long)BH * tab.l[l].n;
   tab.chunk = chunk_tokens(total_tokens);
-  tab.total_tiles = tab.n_workers = tab.wide = 0;
+  tab.total_tiles = tab.n_workers = tab.wide = tab.paired = 0;
   size_t slots = 0;
   for (int l = 0; l < tab.n_layers; ++l) {
     tab.l[l].part_base = (int)slots;

@@ -34,3 +34,51 @@ def max_over_ranks(x: float, dist=None, device=None) -> float:
 def whole_job_throughput(units_per_rank: float, world: int, slowest_seconds: float) -> float:
     """Aggregate throughput of a weak-scaled job: all ranks' units over the slowest rank's time."""
     return units_per_rank * world / slowest_seconds
+
+
+def init_ranks(backend: str = "nccl"):
+    """Reads RANK / WORLD_SIZE / LOCAL_RANK / MASTER_* from the environment (as torch.distributed.run sets them) and
+    joins the process group when there is more than one rank.  Returns (dist or None, rank, world, local_rank).
+    The group exists only for the barrier and the max over ranks of the timings: the data path has no collective."""
+    import os
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world == 1:
+        return None, rank, world, local
+    import torch
+    import torch.distributed as dist
+    if backend == "nccl":
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        dist.init_process_group(backend)
+    return dist, rank, world, local
+
+
+def finish_ranks(dist) -> None:
+    if dist is not None and dist.is_initialized():
+        dist.destroy_process_group()
+
+
+def spawn_ranks(n_ranks: int, script_and_args: list[str], port: int | None = None, timeout: float | None = None) -> int:
+    """Starts `n_ranks` local processes of `script_and_args` under torch.distributed.run (one per GPU for the
+    benchmark), rendezvous on 127.0.0.1, and returns the launcher's exit code.  The ranks inherit stdout, so
+    rank 0's result line appears on the caller's."""
+    import socket
+    import subprocess
+    import sys
+    if port is None:
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port)] + list(script_and_args)
+    return subprocess.run(cmd, timeout=timeout).returncode
+
+
+def job_line(metric: str, unit: str, units_per_rank: float, world: int, slowest_seconds: float, **more) -> dict:
+    """The fields of a result line that depend on the number of ranks."""
+    line = {"metric": metric, "value": whole_job_throughput(units_per_rank, world, slowest_seconds), "unit": unit,
+            "n_gpus": world, "scaling": "weak"}
+    line.update(more)
+    return line

@@ -52,3 +52,19 @@ def test_two_gloo_ranks_agree():
         assert sorted(gathered[0] + gathered[1]) == list(range(5))
         assert not set(gathered[0]) & set(gathered[1])
     assert shard.whole_job_throughput(10.0, 2, 2.0) == 10.0
+
+
+def test_spawned_ranks_print_one_line_for_the_whole_job(capfd):
+    """The spawn code bench.py uses for --gpus N (torch.distributed.run on 127.0.0.1) with two gloo ranks on CPU:
+    rank 0's line reports both ranks, the slowest rank's time and disjoint units."""
+    import json
+    worker = os.path.join(os.path.dirname(os.path.abspath(__file__)), "rank_worker.py")
+    rc = shard.spawn_ranks(2, [worker], timeout=300)
+    out = capfd.readouterr().out
+    assert rc == 0
+    lines = [json.loads(l) for l in out.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak"
+    assert line["value"] == 10.0 * 2 / 1.0                            # all ranks' units over the slowest rank's second
+    assert sorted(line["units"][0] + line["units"][1]) == list(range(7))
