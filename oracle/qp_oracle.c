@@ -219,13 +219,19 @@ void qpo_select(const double* pooled, int Bt, int Hkv, int L, int w, int n_keep,
  *   range = mx - zf; s32 = range / (2^b - 1); s16 = fp16 round-up(s32);
  *   sf = float(s16); code = clamp(rint((x - zf)/sf), 0, 2^b - 1), 0 if sf == 0.
  * x points at the first element, consecutive elements are `stride` apart. */
-static void quant_group(const float* x, int stride, int g, int bits, uint32_t* codes,
-                        uint16_t* s16_out, uint16_t* z16_out) {
-  float mn = x[0], mx = x[0];
-  for (int e = 1; e < g; ++e) {
+static void quant_group_thr(const float* x, int stride, int g, int bits, float thr, uint32_t* codes,
+                            uint16_t* s16_out, uint16_t* z16_out) {
+  /* thr: elements with |x| > thr are outliers (Sec. 5.3 "Quantization methods", Appendix B: numbers whose
+   * absolute value exceeds 6 are excluded from quantization).  They take no part in min/max, get code 0 and
+   * are kept exactly elsewhere.  thr = +inf: no filtering.  A group made of outliers only has z = s = 0. */
+  float mn = 0.0f, mx = 0.0f;
+  int seen = 0;
+  for (int e = 0; e < g; ++e) {
     float v = x[(size_t)e * stride];
-    if (v < mn) mn = v;
-    if (v > mx) mx = v;
+    if (fabsf(v) > thr) continue;
+    if (!seen || v < mn) mn = v;
+    if (!seen || v > mx) mx = v;
+    seen = 1;
   }
   const int qmax = (1 << bits) - 1;
   uint16_t z16 = f32_to_f16_dir(mn, -1);
@@ -236,7 +242,7 @@ static void quant_group(const float* x, int stride, int g, int bits, uint32_t* c
   volatile float sf = f16_to_f32(s16);
   for (int e = 0; e < g; ++e) {
     uint32_t c = 0;
-    if (sf != 0.0f) {
+    if (sf != 0.0f && !(fabsf(x[(size_t)e * stride]) > thr)) {
       volatile float diff = x[(size_t)e * stride] - zf;
       volatile float qf = diff / sf;
       float rf = rintf(qf);                 /* round half to even */
@@ -248,6 +254,11 @@ static void quant_group(const float* x, int stride, int g, int bits, uint32_t* c
   }
   *s16_out = s16;
   *z16_out = z16;
+}
+
+static void quant_group(const float* x, int stride, int g, int bits, uint32_t* codes,
+                        uint16_t* s16_out, uint16_t* z16_out) {
+  quant_group_thr(x, stride, g, bits, INFINITY, codes, s16_out, z16_out);
 }
 
 /* element e of a group -> word e / (32/b), bit offset (e mod (32/b)) * b */
@@ -388,5 +399,116 @@ void qpo_decode(const uint16_t* q, const double* Kd, const double* Vd, int Bt, i
       }
     }
     free(a);
+  }
+}
+
+/* ---------- other quantization strategies of the ablation (Sec. 5.3 "Quantization methods") ----------- */
+/*
+ * k_axis = 0: keys per channel over g kept tokens (KIVI, as qpo_quantize).
+ * k_axis = 1: keys grouped like the values, g consecutive channels of one token ("FlexGen": both caches
+ *             quantized along the token dimension, i.e. token by token; Sec. 5.3).  Layout then
+ *             Kc [Bt,Hkv,n,D/g,wpg], Ks,Kz [Bt,Hkv,n,D/g].
+ * thr: outlier threshold (Appendix B: |x| > 6 is excluded from quantization); +inf = no filtering.
+ * Outliers of a (batch, KV head) are listed in ascending order of t*D + d (t = index among the kept
+ * tokens): side_idx [Bt*Hkv, cap] int32, side_val [Bt*Hkv, cap] bf16 bits, side_cnt [Bt*Hkv]
+ * (-1 if more than cap).  One list for keys, one for values.  bits < 16 only.
+ */
+void qpo_quantize_ex(const uint16_t* K, const uint16_t* V, const int32_t* kept, int Bt, int Hkv,
+                     int D, int L, int n, int bits, int g, int k_axis, float thr, uint32_t* Kc,
+                     uint16_t* Ks, uint16_t* Kz, uint32_t* Vc, uint16_t* Vs, uint16_t* Vz,
+                     int32_t* k_side_idx, uint16_t* k_side_val, int32_t* k_side_cnt,
+                     int32_t* v_side_idx, uint16_t* v_side_val, int32_t* v_side_cnt, int cap) {
+#pragma omp parallel for schedule(dynamic)
+  for (int bh = 0; bh < Bt * Hkv; ++bh) {
+    const uint16_t* Kh = K + (size_t)bh * L * D;
+    const uint16_t* Vh = V + (size_t)bh * L * D;
+    const int32_t* idx = kept + (size_t)bh * n;
+    const int wpg = g * bits / 32;
+    float* Ke = (float*)malloc(sizeof(float) * (size_t)n * D);
+    float* Ve = (float*)malloc(sizeof(float) * (size_t)n * D);
+    uint32_t* codes = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)g);
+    int kc = 0, vc = 0;
+    for (int t = 0; t < n; ++t)
+      for (int d = 0; d < D; ++d) {
+        const uint16_t kb = Kh[(size_t)idx[t] * D + d], vb = Vh[(size_t)idx[t] * D + d];
+        Ke[(size_t)t * D + d] = bf16_to_f32(kb);
+        Ve[(size_t)t * D + d] = bf16_to_f32(vb);
+        if (fabsf(bf16_to_f32(kb)) > thr) {              /* ascending t*D + d by construction */
+          if (kc < cap) { k_side_idx[(size_t)bh * cap + kc] = t * D + d; k_side_val[(size_t)bh * cap + kc] = kb; }
+          ++kc;
+        }
+        if (fabsf(bf16_to_f32(vb)) > thr) {
+          if (vc < cap) { v_side_idx[(size_t)bh * cap + vc] = t * D + d; v_side_val[(size_t)bh * cap + vc] = vb; }
+          ++vc;
+        }
+      }
+    if (k_side_cnt) k_side_cnt[bh] = kc <= cap ? kc : -1;
+    if (v_side_cnt) v_side_cnt[bh] = vc <= cap ? vc : -1;
+    if (k_axis == 0) {
+      uint32_t* Kcb = Kc + (size_t)bh * (n / g) * D * wpg;
+      for (int u = 0; u < n / g; ++u)
+        for (int d = 0; d < D; ++d) {
+          size_t gi = (size_t)u * D + d;
+          quant_group_thr(Ke + (size_t)u * g * D + d, D, g, bits, thr, codes,
+                          Ks + (size_t)bh * (n / g) * D + gi, Kz + (size_t)bh * (n / g) * D + gi);
+          pack_group(codes, g, bits, Kcb + gi * wpg);
+        }
+    } else {
+      uint32_t* Kcb = Kc + (size_t)bh * n * (D / g) * wpg;
+      for (int t = 0; t < n; ++t)
+        for (int v = 0; v < D / g; ++v) {
+          size_t gi = (size_t)t * (D / g) + v;
+          quant_group_thr(Ke + (size_t)t * D + (size_t)v * g, 1, g, bits, thr, codes,
+                          Ks + (size_t)bh * n * (D / g) + gi, Kz + (size_t)bh * n * (D / g) + gi);
+          pack_group(codes, g, bits, Kcb + gi * wpg);
+        }
+    }
+    uint32_t* Vcb = Vc + (size_t)bh * n * (D / g) * wpg;
+    for (int t = 0; t < n; ++t)
+      for (int v = 0; v < D / g; ++v) {
+        size_t gi = (size_t)t * (D / g) + v;
+        quant_group_thr(Ve + (size_t)t * D + (size_t)v * g, 1, g, bits, thr, codes,
+                        Vs + (size_t)bh * n * (D / g) + gi, Vz + (size_t)bh * n * (D / g) + gi);
+        pack_group(codes, g, bits, Vcb + gi * wpg);
+      }
+    free(Ke);
+    free(Ve);
+    free(codes);
+  }
+}
+
+/* Eq. 5 for the layouts of qpo_quantize_ex; a listed outlier is reconstructed as its stored 16-bit value. */
+void qpo_dequantize_ex(const uint32_t* Kc, const uint16_t* Ks, const uint16_t* Kz, const uint32_t* Vc,
+                       const uint16_t* Vs, const uint16_t* Vz, int Bt, int Hkv, int D, int n, int bits,
+                       int g, int k_axis, const int32_t* k_side_idx, const uint16_t* k_side_val,
+                       const int32_t* k_side_cnt, const int32_t* v_side_idx, const uint16_t* v_side_val,
+                       const int32_t* v_side_cnt, int cap, double* Kd, double* Vd) {
+  const int per = 32 / bits, wpg = g * bits / 32;
+  const uint32_t mask = (1u << bits) - 1u;
+  for (int bh = 0; bh < Bt * Hkv; ++bh) {
+    for (int t = 0; t < n; ++t)
+      for (int d = 0; d < D; ++d) {
+        size_t o = ((size_t)bh * n + t) * D + d;
+        {
+          size_t gi;
+          int e;
+          if (k_axis == 0) { gi = ((size_t)bh * (n / g) + t / g) * D + d; e = t % g; }
+          else { gi = ((size_t)bh * n + t) * (D / g) + d / g; e = d % g; }
+          uint32_t c = (Kc[gi * wpg + e / per] >> ((e % per) * bits)) & mask;
+          Kd[o] = (double)c * (double)f16_to_f32(Ks[gi]) + (double)f16_to_f32(Kz[gi]);
+        }
+        {
+          size_t gi = ((size_t)bh * n + t) * (D / g) + d / g;
+          int e = d % g;
+          uint32_t c = (Vc[gi * wpg + e / per] >> ((e % per) * bits)) & mask;
+          Vd[o] = (double)c * (double)f16_to_f32(Vs[gi]) + (double)f16_to_f32(Vz[gi]);
+        }
+      }
+    if (k_side_cnt)
+      for (int i = 0; i < k_side_cnt[bh]; ++i)
+        Kd[(size_t)bh * n * D + k_side_idx[(size_t)bh * cap + i]] = (double)bf16_to_f32(k_side_val[(size_t)bh * cap + i]);
+    if (v_side_cnt)
+      for (int i = 0; i < v_side_cnt[bh]; ++i)
+        Vd[(size_t)bh * n * D + v_side_idx[(size_t)bh * cap + i]] = (double)bf16_to_f32(v_side_val[(size_t)bh * cap + i]);
   }
 }

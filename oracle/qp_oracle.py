@@ -49,6 +49,10 @@ def lib() -> ctypes.CDLL:
         L.qpo_dequantize.argtypes = [p, p, p, p, p, p, i, i, i, i, i, i, p, p]
         L.qpo_decode.restype = None
         L.qpo_decode.argtypes = [p, p, p, i, i, i, i, i, p]
+        L.qpo_quantize_ex.restype = None
+        L.qpo_quantize_ex.argtypes = [p, p, p, i, i, i, i, i, i, i, i, ctypes.c_float] + [p] * 12 + [i]
+        L.qpo_dequantize_ex.restype = None
+        L.qpo_dequantize_ex.argtypes = [p] * 6 + [i] * 7 + [p] * 6 + [i, p, p]
         L.qpo_f32_to_f16_down.restype = ctypes.c_uint16
         L.qpo_f32_to_f16_down.argtypes = [ctypes.c_float]
         L.qpo_f32_to_f16_up.restype = ctypes.c_uint16
@@ -125,6 +129,18 @@ class Packed:
     k_zero: np.ndarray | None
     v_scale: np.ndarray | None  # u16(fp16) [Bt,Hkv,n,D/g]
     v_zero: np.ndarray | None
+    # the other strategies of Sec. 5.3 (qpo_quantize_ex); defaults = the method's own (KIVI axes, no filtering)
+    k_axis: int = 0                     # 1: keys grouped per token like the values: k_codes [Bt,Hkv,n,D/g,wpg]
+    k_side: "Side | None" = None        # outliers kept in 16 bit, keys / values
+    v_side: "Side | None" = None
+
+
+@dataclass
+class Side:
+    """Outliers of every (batch, KV head), ascending in t*D + d (t = index among the kept tokens)."""
+    idx: np.ndarray    # int32 [Bt,Hkv,cap]
+    val: np.ndarray    # u16(bf16) [Bt,Hkv,cap]
+    cnt: np.ndarray    # int32 [Bt,Hkv]
 
 
 def quantize(k: np.ndarray, v: np.ndarray, kept: np.ndarray, bits: int, group: int) -> Packed:
@@ -150,11 +166,51 @@ def quantize(k: np.ndarray, v: np.ndarray, kept: np.ndarray, bits: int, group: i
     return Packed(bits, group, n, kc, vc, ks, kz, vs, vz)
 
 
+def quantize_ex(k: np.ndarray, v: np.ndarray, kept: np.ndarray, bits: int, group: int, k_axis: int = 0,
+                outlier_threshold: float | None = None, cap: int | None = None) -> Packed:
+    """The quantization strategies of Sec. 5.3: key grouping axis and outlier filtering (bits < 16)."""
+    k, v, kept = _c(k, np.uint16), _c(v, np.uint16), _c(kept, np.int32)
+    Bt, Hkv, L, D = k.shape
+    n = kept.shape[-1]
+    assert bits < 16 and D % group == 0 and (k_axis == 1 or n % group == 0)
+    wpg = group * bits // 32
+    if k_axis == 0:
+        kc = np.empty((Bt, Hkv, n // group, D, wpg), np.uint32)
+        ks = np.empty((Bt, Hkv, n // group, D), np.uint16)
+    else:
+        kc = np.empty((Bt, Hkv, n, D // group, wpg), np.uint32)
+        ks = np.empty((Bt, Hkv, n, D // group), np.uint16)
+    kz = np.empty_like(ks)
+    vc = np.empty((Bt, Hkv, n, D // group, wpg), np.uint32)
+    vs = np.empty((Bt, Hkv, n, D // group), np.uint16)
+    vz = np.empty_like(vs)
+    filt = outlier_threshold is not None
+    cap = (n * D if cap is None else cap) if filt else 1
+    sides = [Side(np.zeros((Bt, Hkv, cap), np.int32), np.zeros((Bt, Hkv, cap), np.uint16),
+                  np.zeros((Bt, Hkv), np.int32)) for _ in range(2)]
+    lib().qpo_quantize_ex(_p(k), _p(v), _p(kept), Bt, Hkv, D, L, n, bits, group, k_axis,
+                          float(outlier_threshold) if filt else float("inf"),
+                          _p(kc), _p(ks), _p(kz), _p(vc), _p(vs), _p(vz),
+                          _p(sides[0].idx), _p(sides[0].val), _p(sides[0].cnt),
+                          _p(sides[1].idx), _p(sides[1].val), _p(sides[1].cnt), cap)
+    return Packed(bits, group, n, kc, vc, ks, kz, vs, vz, k_axis, sides[0] if filt else None,
+                  sides[1] if filt else None)
+
+
 def dequantize(pk: Packed, D: int):
     """-> (K', V') fp64 [Bt,Hkv,n,D]  (Eq. 5)."""
     Bt, Hkv = pk.k_codes.shape[:2]
     kd = np.empty((Bt, Hkv, pk.n, D), np.float64)
     vd = np.empty_like(kd)
+    if pk.k_axis != 0 or pk.k_side is not None:
+        ksd, vsd = pk.k_side, pk.v_side
+        cap = ksd.idx.shape[-1] if ksd is not None else 1
+        lib().qpo_dequantize_ex(_p(pk.k_codes), _p(pk.k_scale), _p(pk.k_zero), _p(pk.v_codes), _p(pk.v_scale),
+                                _p(pk.v_zero), Bt, Hkv, D, pk.n, pk.bits, pk.group, pk.k_axis,
+                                _p(ksd.idx) if ksd else None, _p(ksd.val) if ksd else None,
+                                _p(ksd.cnt) if ksd else None, _p(vsd.idx) if vsd else None,
+                                _p(vsd.val) if vsd else None, _p(vsd.cnt) if vsd else None, cap, _p(kd), _p(vd))
+        return kd, vd
     lib().qpo_dequantize(_p(pk.k_codes), _p(pk.k_scale), _p(pk.k_zero), _p(pk.v_codes),
                          _p(pk.v_scale), _p(pk.v_zero), Bt, Hkv, D, pk.n, pk.bits, pk.group,
                          _p(kd), _p(vd))
