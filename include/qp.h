@@ -275,6 +275,46 @@ qp_status qp_decode_attn_tail(const void* q, const qp_cache* cache /* host */, c
                               void* out, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The other quantization strategies of the paper's ablation (Sec. 5.3 "Quantization methods"; Appendix B
+ * "KV quantization").  The method's own arrangement is KIVI's (keys per channel, values per token, no
+ * filtering); the ablation also runs
+ *   - the FlexGen arrangement: keys AND values quantized token by token, g consecutive channels of one
+ *     token per group (k_axis = 1; the paper's FlexGen runs use g = 64), and
+ *   - outlier filtering for either arrangement: numbers with |x| > outlier_threshold (6 in the paper,
+ *     about 1 % of the cache) are left out of their group's min/max, get code 0, and are kept in 16 bit in
+ *     a side list; reconstruction takes the listed value instead of code * scale + zero.  A group that
+ *     consists of outliers only has scale = zero = 0.
+ * With k_axis = 1 the key arrays of qp_cache have the value arrays' shapes: k_codes [Bt,Hkv,n,D/g,wpg],
+ * k_scale, k_zero [Bt,Hkv,n,D/g] (same byte sizes as before).
+ * Side list of one tensor (device arrays, caller-allocated): for every (batch, KV head) the outliers in
+ * ascending order of t*D + d (t = index among the kept tokens, d = channel):
+ *   idx int32 [Bt,Hkv,cap], val bf16 [Bt,Hkv,cap], cnt int32 [Bt,Hkv] (-1: more than cap outliers, list invalid),
+ *   tile_ptr int32 [Bt,Hkv,ceil(n/32)+1]: the entries of tokens 32i..32i+31 are [tile_ptr[i], tile_ptr[i+1]).
+ * outlier_threshold <= 0 or +inf: no filtering (the side lists are ignored and may be zeroed structs).
+ */
+typedef struct qp_side {
+  int32_t cap, reserved_;
+  int32_t* idx;
+  void* val;
+  int32_t* cnt;
+  int32_t* tile_ptr;
+} qp_side;
+typedef struct qp_strategy {
+  int32_t k_axis;            /* 0: keys per channel (KIVI); 1: keys per token (FlexGen) */
+  float outlier_threshold;   /* <= 0 or inf: off */
+  qp_side k_side, v_side;
+} qp_strategy;
+
+/* S3 under a strategy: as qp_gather_quantize (bits < 16), plus the side lists when filtering is on. */
+qp_status qp_gather_quantize_ex(const void* K, const void* V, const int32_t* kept_idx, int L,
+                                const qp_cache* cache /* host */, const qp_strategy* strategy /* host */,
+                                void* stream);
+/* S4 + S5 under a strategy: as qp_decode_attn for a cache written by qp_gather_quantize_ex with the same
+ * strategy.  Runs in plain stream order.  workspace: qp_decode_workspace_bytes(cache) bytes. */
+qp_status qp_decode_attn_ex(const void* q, const qp_cache* cache /* host */, const qp_strategy* strategy /* host */,
+                            void* out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Decode attention without any caller-supplied scratch.  (The paper has no counterpart to this
  * call; it exists for integration reasons only.)  Some hosts of this library cannot give it
  * scratch memory: a serving process that hands all device memory to its own arena at start-up,

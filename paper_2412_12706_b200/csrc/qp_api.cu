@@ -1,6 +1,7 @@
 // C ABI of the library: argument checks, workspace carving and launches.  No allocation,
 // no synchronisation, no host copies.
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -435,6 +436,68 @@ qp_status qp_decode_attn_tail_layers(int n_layers, const void* const* q, const q
 qp_status qp_decode_attn_layers(int n_layers, const void* const* q, const qp_cache* caches, void* const* out,
                                 void* workspace, size_t workspace_bytes, void* stream) {
   return qp_decode_attn_tail_layers(n_layers, q, caches, nullptr, out, workspace, workspace_bytes, stream);
+}
+
+static qp_status check_strategy(const qp_strategy* s, const qp_cache* c, bool* filter) {
+  if (!s) return QP_ERR_INVALID_ARG;
+  if (s->k_axis != 0 && s->k_axis != 1) return QP_ERR_INVALID_ARG;
+  if (c->bits == 16) return QP_ERR_UNSUPPORTED;                 // nothing is quantized at 16 bit
+  *filter = s->outlier_threshold > 0.f && s->outlier_threshold < INFINITY;
+  if (*filter)
+    for (const qp_side* q : {&s->k_side, &s->v_side}) {
+      if (!q->idx || !q->val || !q->cnt || !q->tile_ptr || q->cap < 1) return QP_ERR_INVALID_ARG;
+      if ((reinterpret_cast<uintptr_t>(q->idx) | reinterpret_cast<uintptr_t>(q->cnt) |
+           reinterpret_cast<uintptr_t>(q->tile_ptr)) & 3u) return QP_ERR_ALIGNMENT;
+      if (reinterpret_cast<uintptr_t>(q->val) & 1u) return QP_ERR_ALIGNMENT;
+    }
+  return QP_OK;
+}
+
+qp_status qp_gather_quantize_ex(const void* K, const void* V, const int32_t* kept_idx, int L, const qp_cache* cache,
+                                const qp_strategy* strategy, void* stream) {
+  if (!K || !V || !kept_idx || L < 1) return QP_ERR_INVALID_ARG;
+  qp_status s = check_cache(cache, true);
+  if (s != QP_OK) return s;
+  bool filter = false;
+  s = check_strategy(strategy, cache, &filter);
+  if (s != QP_OK) return s;
+  if (cache->n_keep > L) return QP_ERR_BUDGET;
+  if (!aligned16(K) || !aligned16(V)) return QP_ERR_ALIGNMENT;
+  cache_written(static_cast<cudaStream_t>(stream));
+  return launch_gather_quantize_ex(K, V, kept_idx, L, *cache, *strategy, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_decode_attn_ex(const void* q, const qp_cache* cache, const qp_strategy* strategy, void* out,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+  if (!q || !out || !workspace) return QP_ERR_INVALID_ARG;
+  qp_status s = check_cache(cache, true);
+  if (s != QP_OK) return s;
+  bool filter = false;
+  s = check_strategy(strategy, cache, &filter);
+  if (s != QP_OK) return s;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return QP_ERR_ALIGNMENT;
+  const qp_cache& c = *cache;
+  DecTable tab;
+  tab.n_layers = 1;
+  tab.l[0] = DecLayer{c.k_codes, c.v_codes, static_cast<const __half*>(c.k_scale), static_cast<const __half*>(c.k_zero),
+                      static_cast<const __half*>(c.v_scale), static_cast<const __half*>(c.v_zero), q, out, c.n_keep, 0, 0,
+                      cache_capacity(c)};
+  const DecDims d{c.batch, c.n_q_heads, c.n_kv_heads, c.head_dim, c.bits, c.group};
+  if (workspace_bytes < decode_plan_chunked(tab, d)) return QP_ERR_WORKSPACE;
+  DecEx ex{};
+  ex.k_axis = strategy->k_axis;
+  ex.has_side = filter ? 1 : 0;
+  if (filter) {
+    const int n_tiles = (c.n_keep + 31) / 32;
+    auto side = [&](const qp_side& x) {
+      return SideList{x.idx, static_cast<const uint16_t*>(x.val), x.cnt, x.tile_ptr, x.cap, n_tiles};
+    };
+    ex.k = side(strategy->k_side);
+    ex.v = side(strategy->v_side);
+  }
+  cache_written(static_cast<cudaStream_t>(stream));           // plain stream order here and for the next decode call
+  return launch_decode_ex(tab, d, ex, workspace, static_cast<cudaStream_t>(stream)) == cudaSuccess ? QP_OK : QP_ERR_CUDA;
 }
 
 qp_status qp_decode_overlap(void* stream, int enable) {

@@ -109,6 +109,24 @@ cudaError_t launch_append_rows(int n_layers, const void* const* k_new, const voi
 cudaError_t launch_flush_tails(int n_layers, const int* which, const qp_cache* caches, const qp_tail* tails,
                                cudaStream_t st);
 
+// The other quantization strategies (qp_strategy): key grouping axis and outlier side lists, device pointers.
+struct SideList {
+  const int32_t* idx;       // [BH, cap] ascending t*D + d
+  const uint16_t* val;      // [BH, cap] bf16
+  const int32_t* cnt;       // [BH]
+  const int32_t* tile_ptr;  // [BH, n_tiles + 1]: entries of tokens 32i .. 32i+31 are [tile_ptr[i], tile_ptr[i+1])
+  int cap, n_tiles;
+};
+struct DecEx {
+  int k_axis;               // 0: key groups per channel over g tokens; 1: per token over g channels
+  int has_side;
+  SideList k, v;
+};
+cudaError_t launch_gather_quantize_ex(const void* K, const void* V, const int32_t* kept, int L, const qp_cache& c,
+                                      const qp_strategy& s, cudaStream_t st);
+cudaError_t launch_decode_ex(const struct DecTable& tab, const struct DecDims& d, const DecEx& ex, void* workspace,
+                             cudaStream_t st);
+
 // decode: per-layer device pointers, passed by value as a kernel parameter
 struct DecLayer {
   const void* kc;
@@ -154,6 +172,7 @@ constexpr int kMaxDecodeWorkers = QP_MAX_DECODE_WORKERS;
 // paired: the stream lets consecutive calls overlap (two calls share the GPU most of the time), so a small launch
 // does better with fewer, longer-lived workers; alone on the GPU it wants as many as it can feed.
 size_t decode_plan(DecTable& tab, const DecDims& d, bool paired);
+size_t decode_plan_chunked(DecTable& tab, const DecDims& d);   // the chunked decomposition, whatever the shape
 // Upper bound of decode_plan's result for one layer of n_keep tokens, whatever else is in the launch.
 size_t decode_workspace_bound(const DecDims& d, int n_keep);
 // Workspace of the tensor-core kernels: two areas of partial records, used by alternate calls (parity), so that

@@ -29,9 +29,13 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Reference-shaped kernel: any supported (B, g, D, G).  One lane per token on the key side,
 // one lane per channel (stride 32) on the value side.
+// ex: key grouping axis and outlier side lists of the other quantization strategies (single layer); a listed
+// element was stored with code 0, so the dense arithmetic sees its group's zero point z there and the listed
+// value x enters as a correction x - z, applied in list order (fixed order of additions).
 template <int BITS>
 __global__ void __launch_bounds__(DG_THREADS)
-decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials) {
+decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, float* __restrict__ partials,
+                      const DecEx ex) {
   constexpr int PER = BITS < 16 ? 32 / BITS : 1;
   constexpr uint32_t QMAX = BITS < 16 ? (1u << BITS) - 1u : 0u;
   const int layer = blockIdx.z, bh = blockIdx.y, split = blockIdx.x;
@@ -75,15 +79,50 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
 #pragma unroll
     for (int h = 0; h < MAXG; ++h) lg[h] = 0.f;
     if constexpr (BITS < 16) {
-      const int u = tk / g, e = tk % g;
-      const size_t base = ((size_t)bh * (ns / g) + u) * D;
-      const int wsel = e / PER, sh = (e % PER) * BITS;
-      for (int d = 0; d < D; ++d) {
-        const uint32_t c = (kc[(base + d) * wpg + wsel] >> sh) & QMAX;
-        const float kf = fmaf((float)c, __half2float(ly.ks[base + d]), __half2float(ly.kz[base + d]));
+      if (ex.k_axis == 1) {                                     // this lane's token: D/g groups of g channels
+        const size_t row = ((size_t)bh * ns + tk) * ngv;
+        for (int v = 0; v < ngv; ++v) {
+          const float sc = __half2float(ly.ks[row + v]), zr = __half2float(ly.kz[row + v]);
+          const uint32_t* wp = kc + (row + v) * wpg;
+          for (int wd = 0; wd < wpg; ++wd) {
+            const uint32_t word = wp[wd];
 #pragma unroll
-        for (int h = 0; h < MAXG; ++h)
-          if (h < G) lg[h] = fmaf(sq[h][d], kf, lg[h]);
+            for (int i = 0; i < PER; ++i) {
+              const float kf = fmaf((float)((word >> (i * BITS)) & QMAX), sc, zr);
+              const int d = v * g + wd * PER + i;
+#pragma unroll
+              for (int h = 0; h < MAXG; ++h)
+                if (h < G) lg[h] = fmaf(sq[h][d], kf, lg[h]);
+            }
+          }
+        }
+      } else {
+        const int u = tk / g, e = tk % g;
+        const size_t base = ((size_t)bh * (ns / g) + u) * D;
+        const int wsel = e / PER, sh = (e % PER) * BITS;
+        for (int d = 0; d < D; ++d) {
+          const uint32_t c = (kc[(base + d) * wpg + wsel] >> sh) & QMAX;
+          const float kf = fmaf((float)c, __half2float(ly.ks[base + d]), __half2float(ly.kz[base + d]));
+#pragma unroll
+          for (int h = 0; h < MAXG; ++h)
+            if (h < G) lg[h] = fmaf(sq[h][d], kf, lg[h]);
+        }
+      }
+      if (ex.has_side) {                                        // key outliers of this tile, in list order
+        const int32_t* tp = ex.k.tile_ptr + (size_t)bh * (ex.k.n_tiles + 1) + (tile >> 5);
+        const int32_t* sidx = ex.k.idx + (size_t)bh * ex.k.cap;
+        const uint16_t* sval = ex.k.val + (size_t)bh * ex.k.cap;
+        for (int i = tp[0]; i < tp[1]; ++i) {
+          const int fi = sidx[i], t2 = fi / D, d = fi % D;      // warp-uniform
+          if (t2 == tok) {
+            const size_t gi = ex.k_axis == 1 ? ((size_t)bh * ns + t2) * ngv + d / g
+                                             : ((size_t)bh * (ns / g) + t2 / g) * D + d;
+            const float delta = bf16_bits_to_f32(sval[i]) - __half2float(ly.kz[gi]);
+#pragma unroll
+            for (int h = 0; h < MAXG; ++h)
+              if (h < G) lg[h] = fmaf(sq[h][d], delta, lg[h]);
+          }
+        }
       }
     } else {
       const uint16_t* row = k16 + ((size_t)bh * ns + tk) * D;
@@ -135,6 +174,28 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
 #pragma unroll
           for (int i = 0; i < 4; ++i) acc[h][i] = fmaf(ph, vf[i], acc[h][i]);
         }
+    }
+    if constexpr (BITS < 16) {
+      if (ex.has_side) {                                        // value outliers of this tile, in list order
+        const int32_t* tp = ex.v.tile_ptr + (size_t)bh * (ex.v.n_tiles + 1) + (tile >> 5);
+        const int32_t* sidx = ex.v.idx + (size_t)bh * ex.v.cap;
+        const uint16_t* sval = ex.v.val + (size_t)bh * ex.v.cap;
+        for (int i = tp[0]; i < tp[1]; ++i) {
+          const int fi = sidx[i], t2 = fi / D, d = fi % D;      // warp-uniform
+          const size_t gi = ((size_t)bh * ns + t2) * ngv + d / g;
+          const float delta = bf16_bits_to_f32(sval[i]) - __half2float(ly.vz[gi]);
+#pragma unroll
+          for (int h = 0; h < MAXG; ++h)
+            if (h < G) {
+              const float ph = __shfl_sync(0xffffffffu, p[h], t2 - tile);
+              if ((d & 31) == lane) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  if (j == (d >> 5)) acc[h][j] = fmaf(ph, delta, acc[h][j]);
+              }
+            }
+        }
+      }
     }
   }
 
@@ -250,17 +311,7 @@ size_t decode_plan(DecTable& tab, const DecDims& d, bool paired) {
     tab.chunk = 0;
     return decode_workspace_layout(tab, d).total_bytes();
   }
-  long long total_tokens = 0;
-  for (int l = 0; l < tab.n_layers; ++l) total_tokens += (long long)BH * tab.l[l].n;
-  tab.chunk = chunk_tokens(total_tokens);
-  tab.total_tiles = tab.n_workers = tab.wide = tab.paired = 0;
-  size_t slots = 0;
-  for (int l = 0; l < tab.n_layers; ++l) {
-    tab.l[l].part_base = (int)slots;
-    tab.l[l].tile_base = 0;
-    slots += (size_t)BH * ((tab.l[l].n + tab.chunk - 1) / tab.chunk);
-  }
-  return slots * record_bytes(d);
+  return decode_plan_chunked(tab, d);
 }
 
 DecWorkspace decode_workspace_layout(const DecTable& tab, const DecDims& d) {
@@ -287,11 +338,12 @@ cudaError_t launch_decode(const DecTable& tab, const DecDims& d, void* workspace
   int max_splits = 1;
   for (int l = 0; l < tab.n_layers; ++l) max_splits = max(max_splits, (tab.l[l].n + tab.chunk - 1) / tab.chunk);
   const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
+  const DecEx none{};
   switch (d.bits) {
-    case 2: decode_generic_kernel<2><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
-    case 4: decode_generic_kernel<4><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
-    case 8: decode_generic_kernel<8><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
-    case 16: decode_generic_kernel<16><<<grid, DG_THREADS, 0, st>>>(tab, d, partials); break;
+    case 2: decode_generic_kernel<2><<<grid, DG_THREADS, 0, st>>>(tab, d, partials, none); break;
+    case 4: decode_generic_kernel<4><<<grid, DG_THREADS, 0, st>>>(tab, d, partials, none); break;
+    case 8: decode_generic_kernel<8><<<grid, DG_THREADS, 0, st>>>(tab, d, partials, none); break;
+    case 16: decode_generic_kernel<16><<<grid, DG_THREADS, 0, st>>>(tab, d, partials, none); break;
     default: return cudaErrorInvalidValue;
   }
   cudaError_t e = cudaGetLastError();
@@ -299,6 +351,40 @@ cudaError_t launch_decode(const DecTable& tab, const DecDims& d, void* workspace
   if (tails) return launch_merge_tail(tab, d, partials, *tails, st, false);
   decode_merge_kernel<<<dim3(d.Bt * d.Hq, tab.n_layers), 128, 0, st>>>(tab, d, partials);
   return cudaGetLastError();
+}
+
+// One layer under a quantization strategy: the chunked kernel with the strategy's key axis and side lists, then
+// the chunked merge.  tab: planned with decode_plan_chunked.
+cudaError_t launch_decode_ex(const DecTable& tab, const DecDims& d, const DecEx& ex, void* workspace, cudaStream_t st) {
+  float* partials = static_cast<float*>(workspace);
+  int max_splits = 1;
+  for (int l = 0; l < tab.n_layers; ++l) max_splits = max(max_splits, (tab.l[l].n + tab.chunk - 1) / tab.chunk);
+  const dim3 grid(max_splits, d.Bt * d.Hkv, tab.n_layers);
+  switch (d.bits) {
+    case 2: decode_generic_kernel<2><<<grid, DG_THREADS, 0, st>>>(tab, d, partials, ex); break;
+    case 4: decode_generic_kernel<4><<<grid, DG_THREADS, 0, st>>>(tab, d, partials, ex); break;
+    case 8: decode_generic_kernel<8><<<grid, DG_THREADS, 0, st>>>(tab, d, partials, ex); break;
+    default: return cudaErrorInvalidValue;
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  decode_merge_kernel<<<dim3(d.Bt * d.Hq, tab.n_layers), 128, 0, st>>>(tab, d, partials);
+  return cudaGetLastError();
+}
+
+size_t decode_plan_chunked(DecTable& tab, const DecDims& d) {
+  const int BH = d.Bt * d.Hkv;
+  long long total_tokens = 0;
+  for (int l = 0; l < tab.n_layers; ++l) total_tokens += (long long)BH * tab.l[l].n;
+  tab.chunk = chunk_tokens(total_tokens);
+  tab.total_tiles = tab.n_workers = tab.wide = tab.paired = 0;
+  size_t slots = 0;
+  for (int l = 0; l < tab.n_layers; ++l) {
+    tab.l[l].part_base = (int)slots;
+    tab.l[l].tile_base = 0;
+    slots += (size_t)BH * ((tab.l[l].n + tab.chunk - 1) / tab.chunk);
+  }
+  return slots * record_bytes(d);
 }
 
 }  // namespace qp

@@ -50,6 +50,10 @@ __device__ __forceinline__ uint32_t quant_code(float x, const QParams& p, int qm
   return min(__float_as_uint(m) & 0x3ffu, (uint32_t)qmax);
 }
 
+__device__ __forceinline__ uint32_t code_or_zero(float x, const QParams& p, int qmax, float thr) {
+  return fabsf(x) > thr ? 0u : quant_code(x, p, qmax);
+}
+
 // One layer's arguments.  Sources: K, V rows [BH, L, D]; kept [BH, n_idx] positions of the rows to take
 // (null: row u*g + e itself, the case of a full tail).  Destinations: group u0 + u of arrays that have room for
 // ns tokens per (batch, KV head).
@@ -59,6 +63,8 @@ struct QuantLayer {
   uint32_t *Kc, *Vc;
   __half *Ks, *Kz, *Vs, *Vz;
   int L, n_idx, ns, u0;
+  int k_axis = 0;          // 1: key groups run over g channels of one token, like the values
+  float thr = INFINITY;    // |x| > thr: outlier, left out of min/max, code 0
 };
 template <int NL>
 struct QuantTable {
@@ -81,6 +87,8 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __half* __restrict__ Ks = ql.Ks; __half* __restrict__ Kz = ql.Kz;
   __half* __restrict__ Vs = ql.Vs; __half* __restrict__ Vz = ql.Vz;
   const int L = ql.L, n = ql.n_idx, ns = ql.ns;
+  const float thr = ql.thr;
+  const bool k_rows = ql.k_axis == 1;              // keys token by token: the value loop below, run on K
   // two blocks per run of g kept tokens: an even block quantizes its key group, the odd one its value rows (each has
   // a shorter chain of dependent memory round trips than one block doing both)
   const int u = blockIdx.x >> 1, bh = blockIdx.y, tid = threadIdx.x, nthr = blockDim.x;
@@ -92,7 +100,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __syncthreads();
   const uint16_t* Kh = K + (size_t)bh * L * D;
   const uint16_t* Vh = V + (size_t)bh * L * D;
-  for (int c = tid; key_part && c < g * (D / 8); c += nthr) {
+  for (int c = tid; key_part && !k_rows && c < g * (D / 8); c += nthr) {
     const int e = c / (D / 8), col = (c % (D / 8)) * 8;
     *reinterpret_cast<uint4*>(sK + e * D + col) =
         *reinterpret_cast<const uint4*>(Kh + (size_t)sidx[e] * D + col);
@@ -100,13 +108,15 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __syncthreads();
 
   // keys: channel d, tokens e = 0..g-1
-  for (int d = tid; key_part && d < D; d += nthr) {
-    float mn = bf16_bits_to_f32(sK[d]), mx = mn;
-    for (int e = 1; e < g; ++e) {
+  for (int d = tid; key_part && !k_rows && d < D; d += nthr) {
+    float mn = INFINITY, mx = -INFINITY;
+    for (int e = 0; e < g; ++e) {
       const float x = bf16_bits_to_f32(sK[e * D + d]);
+      if (fabsf(x) > thr) continue;
       mn = fminf(mn, x);
       mx = fmaxf(mx, x);
     }
+    if (mn > mx) mn = mx = 0.f;                     // outliers only
     const QParams p = group_params(mn, mx, QMAX);
     const size_t gi = ((size_t)bh * (ns / g) + ud) * D + d;
     uint32_t* dst = Kc + gi * wpg;
@@ -116,7 +126,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
       for (int i = 0; i < nw; ++i)
 #pragma unroll
         for (int c = 0; c < PER; ++c)
-          wv[i] |= quant_code(bf16_bits_to_f32(sK[((wd + i) * PER + c) * D + d]), p, QMAX) << (c * BITS);
+          wv[i] |= code_or_zero(bf16_bits_to_f32(sK[((wd + i) * PER + c) * D + d]), p, QMAX, thr) << (c * BITS);
       if (nw == 4) *reinterpret_cast<uint4*>(dst + wd) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
       else *reinterpret_cast<uint2*>(dst + wd) = make_uint2(wv[0], wv[1]);
     }
@@ -126,9 +136,13 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
 
   // values: token e, channel group v
   const int ngv = D / g;
-  for (int it = tid; !key_part && it < g * ngv; it += nthr) {
+  const uint16_t* Rh = key_part ? Kh : Vh;          // rows quantized token by token by this block
+  uint32_t* __restrict__ Rc = key_part ? Kc : Vc;
+  __half* __restrict__ Rs = key_part ? Ks : Vs;
+  __half* __restrict__ Rz = key_part ? Kz : Vz;
+  for (int it = tid; (!key_part || k_rows) && it < g * ngv; it += nthr) {
     const int e = it / ngv, v = it % ngv;
-    const uint16_t* src = Vh + (size_t)sidx[e] * D + (size_t)v * g;
+    const uint16_t* src = Rh + (size_t)sidx[e] * D + (size_t)v * g;
     float mn = INFINITY, mx = -INFINITY;
     for (int c8 = 0; c8 < g; c8 += 8) {
       const uint4 q = *reinterpret_cast<const uint4*>(src + c8);
@@ -136,13 +150,14 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const float x0 = bf16lo(ww[i]), x1 = bf16hi(ww[i]);
-        mn = fminf(mn, fminf(x0, x1));
-        mx = fmaxf(mx, fmaxf(x0, x1));
+        if (!(fabsf(x0) > thr)) { mn = fminf(mn, x0); mx = fmaxf(mx, x0); }
+        if (!(fabsf(x1) > thr)) { mn = fminf(mn, x1); mx = fmaxf(mx, x1); }
       }
     }
+    if (mn > mx) mn = mx = 0.f;                     // outliers only
     const QParams p = group_params(mn, mx, QMAX);
     const size_t gi = ((size_t)bh * ns + (size_t)ud * g + e) * ngv + v;
-    uint32_t* dst = Vc + gi * wpg;
+    uint32_t* dst = Rc + gi * wpg;
     // second sweep over the group in 16-byte pieces (8 channels); a piece fills 8/PER words
     constexpr int WPP = PER >= 8 ? 1 : 8 / PER;                 // words completed per piece (PER 16: half a word)
     uint32_t word = 0;
@@ -152,8 +167,8 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
       uint32_t codes[8];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        codes[2 * i] = quant_code(bf16lo(ww[i]), p, QMAX);
-        codes[2 * i + 1] = quant_code(bf16hi(ww[i]), p, QMAX);
+        codes[2 * i] = code_or_zero(bf16lo(ww[i]), p, QMAX, thr);
+        codes[2 * i + 1] = code_or_zero(bf16hi(ww[i]), p, QMAX, thr);
       }
       if constexpr (PER == 16) {                                // 2-bit: two pieces per word
         const int sh = (c8 & 8) ? 16 : 0;
@@ -170,8 +185,77 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
         }
       }
     }
-    Vs[gi] = p.s16;
-    Vz[gi] = p.z16;
+    Rs[gi] = p.s16;
+    Rz[gi] = p.z16;
+  }
+}
+
+// Side list of one tensor (keys or values) of one (batch, KV head): the elements with |x| > thr of the n kept
+// rows, in ascending order of t*D + d, plus the first entry of every 32-token tile.  One block walks the head
+// in chunks of blockDim.x * 8 elements and compacts in order (ballot counts, one block-wide prefix per chunk),
+// so the list is the same in every run.
+constexpr int SL_THREADS = 256;
+__global__ void __launch_bounds__(SL_THREADS)
+side_list_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ V, const int32_t* __restrict__ kept, int L,
+                 int D, int n, float thr, SideList k_out, SideList v_out) {
+  __shared__ int s_warp[SL_THREADS / 32];
+  __shared__ int s_base;
+  const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint16_t* X = (blockIdx.y == 0 ? K : V) + (size_t)bh * L * D;
+  const SideList& o = blockIdx.y == 0 ? k_out : v_out;
+  int32_t* idx = const_cast<int32_t*>(o.idx) + (size_t)bh * o.cap;
+  uint16_t* val = const_cast<uint16_t*>(o.val) + (size_t)bh * o.cap;
+  int32_t* tile_ptr = const_cast<int32_t*>(o.tile_ptr) + (size_t)bh * (o.n_tiles + 1);
+  const int32_t* kp = kept ? kept + (size_t)bh * n : nullptr;
+  const int total8 = n * D / 8;                                   // 16-byte pieces
+  if (tid == 0) s_base = 0;
+  __syncthreads();
+  for (int c0 = 0; c0 < total8; c0 += SL_THREADS) {
+    const int c = c0 + tid;
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    int t = 0, d0 = 0;
+    if (c < total8) {
+      t = (c * 8) / D; d0 = (c * 8) % D;
+      const uint4 q = *reinterpret_cast<const uint4*>(X + (size_t)(kp ? kp[t] : t) * D + d0);
+      w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
+    }
+    unsigned mask = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (fabsf(bf16lo(w[i])) > thr) mask |= 1u << (2 * i);
+      if (fabsf(bf16hi(w[i])) > thr) mask |= 1u << (2 * i + 1);
+    }
+    if (c >= total8) mask = 0;
+    const int mine = __popc(mask);
+    int incl = mine;                                              // inclusive prefix within the warp
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, s);
+      if (lane >= s) incl += y;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int before = s_base;
+    for (int q = 0; q < warp; ++q) before += s_warp[q];
+    int pos = before + incl - mine;
+    // a piece that starts a 32-token tile records where the tile's entries begin
+    if (c < total8 && d0 == 0 && (t & 31) == 0) tile_ptr[t >> 5] = pos;
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      if (mask >> e & 1u) {
+        if (pos < o.cap) {
+          idx[pos] = t * D + d0 + e;
+          val[pos] = (uint16_t)((e & 1) ? w[e >> 1] >> 16 : w[e >> 1] & 0xffffu);
+        }
+        ++pos;
+      }
+    __syncthreads();
+    if (tid == SL_THREADS - 1) s_base = before + incl;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    tile_ptr[o.n_tiles] = s_base;
+    const_cast<int32_t*>(o.cnt)[bh] = s_base <= o.cap ? s_base : -1;
   }
 }
 
@@ -245,6 +329,28 @@ cudaError_t launch_gather_quantize(const void* K, const void* V, const int32_t* 
                         static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
                         static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, n, ns, 0};
   return launch_quant_table<1>(c.bits, tab, dim3(2 * (n / g), BH, 1), D, g, st);
+}
+
+cudaError_t launch_gather_quantize_ex(const void* K, const void* V, const int32_t* kept, int L, const qp_cache& c,
+                                      const qp_strategy& s, cudaStream_t st) {
+  const int BH = c.batch * c.n_kv_heads, D = c.head_dim, n = c.n_keep, g = c.group, ns = cache_capacity(c);
+  const uint16_t* k = static_cast<const uint16_t*>(K);
+  const uint16_t* v = static_cast<const uint16_t*>(V);
+  const bool filter = s.outlier_threshold > 0.f && s.outlier_threshold < INFINITY;
+  QuantTable<1> tab;
+  tab.l[0] = QuantLayer{k, v, kept, static_cast<uint32_t*>(c.k_codes), static_cast<uint32_t*>(c.v_codes),
+                        static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
+                        static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, n, ns, 0,
+                        s.k_axis, filter ? s.outlier_threshold : INFINITY};
+  cudaError_t e = launch_quant_table<1>(c.bits, tab, dim3(2 * (n / g), BH, 1), D, g, st);
+  if (e != cudaSuccess || !filter) return e;
+  const int n_tiles = (n + 31) / 32;
+  auto side = [&](const qp_side& q) {
+    return SideList{q.idx, static_cast<const uint16_t*>(q.val), q.cnt, q.tile_ptr, q.cap, n_tiles};
+  };
+  side_list_kernel<<<dim3(BH, 2), SL_THREADS, 0, st>>>(k, v, kept, L, D, n, s.outlier_threshold, side(s.k_side),
+                                                      side(s.v_side));
+  return cudaGetLastError();
 }
 
 cudaError_t launch_gather_quantize_layers(int n_layers, const void* const* K, const void* const* V,

@@ -25,7 +25,8 @@ EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_work
            "qp_decode_workspace_bytes", "qp_window_scores", "qp_select_topk", "qp_gather_quantize",
            "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static",
            "qp_cache_layout_cap", "qp_append_kv", "qp_append_kv_layers", "qp_decode_attn_tail",
-           "qp_decode_attn_tail_layers", "qp_compress_layers", "qp_decode_overlap"]
+           "qp_decode_attn_tail_layers", "qp_compress_layers", "qp_decode_overlap", "qp_gather_quantize_ex",
+           "qp_decode_attn_ex"]
 
 
 class QpError(RuntimeError):
@@ -43,6 +44,16 @@ class qp_cache(ctypes.Structure):
                 ("k_codes", ctypes.c_void_p), ("v_codes", ctypes.c_void_p),
                 ("k_scale", ctypes.c_void_p), ("k_zero", ctypes.c_void_p),
                 ("v_scale", ctypes.c_void_p), ("v_zero", ctypes.c_void_p)]
+
+
+class qp_side(ctypes.Structure):
+    _fields_ = [("cap", ctypes.c_int32), ("reserved_", ctypes.c_int32), ("idx", ctypes.c_void_p),
+                ("val", ctypes.c_void_p), ("cnt", ctypes.c_void_p), ("tile_ptr", ctypes.c_void_p)]
+
+
+class qp_strategy(ctypes.Structure):
+    _fields_ = [("k_axis", ctypes.c_int32), ("outlier_threshold", ctypes.c_float),
+                ("k_side", qp_side), ("v_side", qp_side)]
 
 
 class qp_tail(ctypes.Structure):
@@ -101,6 +112,11 @@ def lib() -> ctypes.CDLL:
         L.qp_decode_attn_tail.argtypes = [p, cp, tp, p, p, sz, p]
         L.qp_decode_attn_tail_layers.restype = i
         L.qp_decode_attn_tail_layers.argtypes = [i, ctypes.POINTER(p), cp, tp, ctypes.POINTER(p), p, sz, p]
+        sp = ctypes.POINTER(qp_strategy)
+        L.qp_gather_quantize_ex.restype = i
+        L.qp_gather_quantize_ex.argtypes = [p, p, p, i, cp, sp, p]
+        L.qp_decode_attn_ex.restype = i
+        L.qp_decode_attn_ex.argtypes = [p, cp, sp, p, p, sz, p]
         L.qp_decode_overlap.restype = i
         L.qp_decode_overlap.argtypes = [p, i]
         _lib = L
@@ -424,6 +440,55 @@ def decode_attn_static(q: torch.Tensor, cache: Cache, out: torch.Tensor | None =
     return out
 
 
+@dataclass
+class Strategy:
+    """A quantization strategy of Sec. 5.3 (qp_strategy) with torch-owned side-list buffers."""
+    desc: qp_strategy
+    bufs: list
+
+
+def make_strategy(cache: Cache, k_axis: int = 0, outlier_threshold: float | None = None, cap: int | None = None) -> Strategy:
+    """Fills a qp_strategy; with filtering on, allocates the two side lists for `cache` (cap entries per
+    (batch, KV head), default 4 % of the head's elements)."""
+    d = cache.desc
+    s = qp_strategy()
+    s.k_axis = k_axis
+    s.outlier_threshold = float(outlier_threshold) if outlier_threshold else 0.0
+    bufs = []
+    if outlier_threshold:
+        n = d.n_cap or d.n_keep
+        cap = cap or max(64, n * d.head_dim // 25)
+        dev = cache.k_codes.device
+        for side in (s.k_side, s.v_side):
+            idx = torch.zeros((d.batch, d.n_kv_heads, cap), dtype=torch.int32, device=dev)
+            val = torch.zeros((d.batch, d.n_kv_heads, cap), dtype=torch.bfloat16, device=dev)
+            cnt = torch.zeros((d.batch, d.n_kv_heads), dtype=torch.int32, device=dev)
+            tp = torch.zeros((d.batch, d.n_kv_heads, (n + 31) // 32 + 1), dtype=torch.int32, device=dev)
+            side.cap, side.idx, side.val, side.cnt, side.tile_ptr = cap, _ptr(idx), _ptr(val), _ptr(cnt), _ptr(tp)
+            bufs.append((idx, val, cnt, tp))
+    return Strategy(s, bufs)
+
+
+def gather_quantize_ex(K: torch.Tensor, V: torch.Tensor, kept_idx: torch.Tensor, cache: Cache, strategy: Strategy) -> Cache:
+    _dev_bf16(K); _dev_bf16(V)
+    assert kept_idx.is_cuda and kept_idx.dtype == torch.int32 and kept_idx.is_contiguous()
+    _check(lib().qp_gather_quantize_ex(_ptr(K), _ptr(V), _ptr(kept_idx), K.shape[2], ctypes.byref(cache.desc),
+                                       ctypes.byref(strategy.desc), _stream()), "qp_gather_quantize_ex")
+    return cache
+
+
+def decode_attn_ex(q: torch.Tensor, cache: Cache, strategy: Strategy, out: torch.Tensor | None = None,
+                   workspace: torch.Tensor | None = None) -> torch.Tensor:
+    _dev_bf16(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_decode_workspace(decode_workspace_bytes(cache), q.device)
+    _check(lib().qp_decode_attn_ex(_ptr(q), ctypes.byref(cache.desc), ctypes.byref(strategy.desc), _ptr(out),
+                                   _ptr(workspace), workspace.numel(), _stream()), "qp_decode_attn_ex")
+    return out
+
+
 # the C entry points under their own names
 qp_status_string = status_string
 qp_n_keep = n_keep
@@ -439,6 +504,8 @@ qp_decode_attn = decode_attn
 qp_decode_attn_layers = decode_attn_layers
 qp_decode_attn_static = decode_attn_static
 qp_decode_overlap = decode_overlap
+qp_gather_quantize_ex = gather_quantize_ex
+qp_decode_attn_ex = decode_attn_ex
 qp_cache_layout_cap = cache_layout_cap
 qp_append_kv = append_kv
 qp_append_kv_layers = append_kv_layers
