@@ -315,6 +315,34 @@ qp_status qp_decode_attn_ex(const void* q, const qp_cache* cache /* host */, con
                             void* out, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Head-level token budgets: the KV heads of a layer share the layer's budget and keep different numbers of
+ * tokens.  The paper runs two pruning methods of this kind (Ada-KV, HeadKV: Related Work "KV Pruning", Sec. 4
+ * "Setup", Table 1) and says of them only that they retain different tokens per head; the rule here: within a
+ * batch entry the Hkv * (n_mean - w) prefix positions with the largest scores over all KV heads are marked
+ * (equal scores: lower head, then lower position); a head's share is its marked positions plus its w window
+ * tokens, rounded down to whole units of `unit` tokens, at least the smallest unit count above w, at most L
+ * rounded down to units; if raising small heads pushed the total above Hkv * n_mean, the largest heads (lowest
+ * first among equals) give back one unit at a time.
+ * scores fp32 [Bt,Hkv,P] (device, from qp_window_scores) -> n_keep_heads int32 [Bt,Hkv] (device).  The caller
+ * copies the counts to the host to size one cache per (batch, KV head) (descriptors with batch = 1,
+ * n_kv_heads = 1, n_q_heads = G) and then runs qp_select_topk / qp_gather_quantize(_ex) per head on that
+ * head's slice of scores, K and V, and qp_decode_attn_layers(_ex) over the heads' descriptors.  With
+ * unit = group the heads' caches satisfy the per-channel key grouping of the main path; the paper pairs
+ * these methods with the per-token arrangement (k_axis = 1).
+ * workspace: qp_head_budgets_workspace_bytes(...) bytes, 16-byte aligned.  unit >= 1, n_mean > w.
+ */
+size_t qp_head_budgets_workspace_bytes(int batch, int n_kv_heads, int L, int w, int n_mean);
+qp_status qp_head_budgets(const float* scores, int batch, int n_kv_heads, int L, int w, int n_mean, int unit,
+                          int32_t* n_keep_heads, void* workspace, size_t workspace_bytes, void* stream);
+
+/* qp_decode_attn_ex for n_layers caches of one shape, bits and group in one launch pair (n_keep may differ: e.g. the
+ * per-head caches of a head-level budget).  Side lists (filtering) are supported for n_layers = 1 only:
+ * QP_ERR_UNSUPPORTED otherwise.  workspace: the sum of qp_decode_workspace_bytes over the caches. */
+qp_status qp_decode_attn_layers_ex(int n_layers, const void* const* q, const qp_cache* caches /* host */,
+                                   const qp_strategy* strategy /* host */, void* const* out, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
+/*
  * Decode attention without any caller-supplied scratch.  (The paper has no counterpart to this
  * call; it exists for integration reasons only.)  Some hosts of this library cannot give it
  * scratch memory: a serving process that hands all device memory to its own arena at start-up,

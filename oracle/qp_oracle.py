@@ -302,3 +302,39 @@ def decode_state(q: np.ndarray, st: GenState, D: int) -> np.ndarray:
         kd = np.concatenate([kd, _bf16_to_f64(st.tail_k)], axis=2)
         vd = np.concatenate([vd, _bf16_to_f64(st.tail_v)], axis=2)
     return decode(q, kd, vd)
+
+
+# ------------------------------------------------------------------ head-level token budgets
+
+def head_budgets(pooled: np.ndarray, L: int, w: int, n_mean: int, unit: int = 32) -> np.ndarray:
+    """Tokens kept per KV head when the layer's budget is shared between its heads.
+
+    The paper runs two pruning methods of this kind (Ada-KV, HeadKV: Related Work "KV Pruning", Sec. 4
+    "Setup", Table 1) and only says of them that they retain different numbers of tokens per head.  The rule
+    taken here: within one batch entry the Hkv * (n_mean - w) prefix positions with the largest pooled scores
+    over ALL KV heads are marked (equal scores: lower head first, then lower position); a head's raw share is
+    its number of marked positions plus its w window tokens.  Shares are rounded down to whole units of
+    `unit` tokens, raised to the smallest whole unit count above w where they fall below it, capped at L
+    rounded down to units, and, should the raising have pushed the total above Hkv * n_mean, the largest heads
+    (lowest head first among equals) give back one unit at a time.  pooled [Bt,Hkv,P] -> n [Bt,Hkv] int32.
+    """
+    pooled = np.asarray(pooled, np.float64)
+    Bt, Hkv, P = pooled.shape
+    assert P == L - w and n_mean > w
+    k_total = min(Hkv * (n_mean - w), Hkv * P)
+    floor_u = lambda x: (x // unit) * unit
+    n_min = floor_u(w) + unit                          # smallest whole number of units above w
+    n_max = max(n_min, floor_u(L))
+    out = np.zeros((Bt, Hkv), np.int32)
+    for b in range(Bt):
+        items = [(-pooled[b, h, j], h, j) for h in range(Hkv) for j in range(P)]
+        items.sort()
+        raw = [w] * Hkv
+        for _, h, _j in items[:k_total]:
+            raw[h] += 1
+        n = [min(n_max, max(n_min, floor_u(r))) for r in raw]
+        while sum(n) > Hkv * n_mean and max(n) > n_min:
+            h = max(range(Hkv), key=lambda i: (n[i], -i))
+            n[h] -= unit
+        out[b] = n
+    return out

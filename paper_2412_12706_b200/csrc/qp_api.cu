@@ -468,28 +468,57 @@ qp_status qp_gather_quantize_ex(const void* K, const void* V, const int32_t* kep
              ? QP_OK : QP_ERR_CUDA;
 }
 
-qp_status qp_decode_attn_ex(const void* q, const qp_cache* cache, const qp_strategy* strategy, void* out,
-                            void* workspace, size_t workspace_bytes, void* stream) {
-  if (!q || !out || !workspace) return QP_ERR_INVALID_ARG;
-  qp_status s = check_cache(cache, true);
-  if (s != QP_OK) return s;
-  bool filter = false;
-  s = check_strategy(strategy, cache, &filter);
-  if (s != QP_OK) return s;
-  if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return QP_ERR_ALIGNMENT;
-  const qp_cache& c = *cache;
+size_t qp_head_budgets_workspace_bytes(int batch, int n_kv_heads, int L, int w, int n_mean) {
+  if (batch < 1 || n_kv_heads < 1 || w < 1 || w >= L || n_mean <= w) return 0;
+  const long long P = L - w;
+  const long long k_total = std::min<long long>((long long)n_kv_heads * (n_mean - w), (long long)n_kv_heads * P);
+  return (size_t)(((size_t)batch * (k_total + 1) * sizeof(int32_t) + 255) & ~(size_t)255);
+}
+
+qp_status qp_head_budgets(const float* scores, int batch, int n_kv_heads, int L, int w, int n_mean, int unit,
+                          int32_t* n_keep_heads, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!scores || !n_keep_heads || !workspace || batch < 1 || n_kv_heads < 1 || w < 1 || w >= L || unit < 1)
+    return QP_ERR_INVALID_ARG;
+  if (n_mean <= w) return QP_ERR_BUDGET;
+  if ((long long)n_kv_heads * (L - w) + 1 > 0x7fffffffLL || n_kv_heads > 8192) return QP_ERR_UNSUPPORTED;
+  if (!aligned16(workspace)) return QP_ERR_ALIGNMENT;
+  if (workspace_bytes < qp_head_budgets_workspace_bytes(batch, n_kv_heads, L, w, n_mean)) return QP_ERR_WORKSPACE;
+  return launch_head_budgets(scores, batch, n_kv_heads, L, w, n_mean, unit, n_keep_heads,
+                             static_cast<int32_t*>(workspace), static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_decode_attn_layers_ex(int n_layers, const void* const* q, const qp_cache* caches, const qp_strategy* strategy,
+                                   void* const* out, void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_layers < 1 || n_layers > QP_MAX_LAYERS || !q || !caches || !out || !workspace) return QP_ERR_INVALID_ARG;
+  if (!aligned16(workspace)) return QP_ERR_ALIGNMENT;
+  const qp_cache& c0 = caches[0];
   DecTable tab;
-  tab.n_layers = 1;
-  tab.l[0] = DecLayer{c.k_codes, c.v_codes, static_cast<const __half*>(c.k_scale), static_cast<const __half*>(c.k_zero),
-                      static_cast<const __half*>(c.v_scale), static_cast<const __half*>(c.v_zero), q, out, c.n_keep, 0, 0,
-                      cache_capacity(c)};
-  const DecDims d{c.batch, c.n_q_heads, c.n_kv_heads, c.head_dim, c.bits, c.group};
+  tab.n_layers = n_layers;
+  bool filter = false;
+  for (int l = 0; l < n_layers; ++l) {
+    const qp_cache& c = caches[l];
+    qp_status s = check_cache(&c, true);
+    if (s != QP_OK) return s;
+    s = check_strategy(strategy, &c, &filter);
+    if (s != QP_OK) return s;
+    if (c.batch != c0.batch || c.n_q_heads != c0.n_q_heads || c.n_kv_heads != c0.n_kv_heads ||
+        c.head_dim != c0.head_dim || c.bits != c0.bits || c.group != c0.group)
+      return QP_ERR_INVALID_ARG;
+    if (!q[l] || !out[l]) return QP_ERR_INVALID_ARG;
+    if (!aligned16(q[l]) || !aligned16(out[l])) return QP_ERR_ALIGNMENT;
+    tab.l[l] = DecLayer{c.k_codes, c.v_codes, static_cast<const __half*>(c.k_scale), static_cast<const __half*>(c.k_zero),
+                        static_cast<const __half*>(c.v_scale), static_cast<const __half*>(c.v_zero), q[l], out[l], c.n_keep,
+                        0, 0, cache_capacity(c)};
+  }
+  if (filter && n_layers > 1) return QP_ERR_UNSUPPORTED;
+  const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
   if (workspace_bytes < decode_plan_chunked(tab, d)) return QP_ERR_WORKSPACE;
   DecEx ex{};
   ex.k_axis = strategy->k_axis;
   ex.has_side = filter ? 1 : 0;
   if (filter) {
-    const int n_tiles = (c.n_keep + 31) / 32;
+    const int n_tiles = (c0.n_keep + 31) / 32;
     auto side = [&](const qp_side& x) {
       return SideList{x.idx, static_cast<const uint16_t*>(x.val), x.cnt, x.tile_ptr, x.cap, n_tiles};
     };
@@ -498,6 +527,14 @@ qp_status qp_decode_attn_ex(const void* q, const qp_cache* cache, const qp_strat
   }
   cache_written(static_cast<cudaStream_t>(stream));           // plain stream order here and for the next decode call
   return launch_decode_ex(tab, d, ex, workspace, static_cast<cudaStream_t>(stream)) == cudaSuccess ? QP_OK : QP_ERR_CUDA;
+}
+
+qp_status qp_decode_attn_ex(const void* q, const qp_cache* cache, const qp_strategy* strategy, void* out,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+  if (!cache) return QP_ERR_INVALID_ARG;
+  const void* qs[1] = {q};
+  void* os[1] = {out};
+  return qp_decode_attn_layers_ex(1, qs, cache, strategy, os, workspace, workspace_bytes, stream);
 }
 
 qp_status qp_decode_overlap(void* stream, int enable) {

@@ -94,6 +94,10 @@ cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_
 cudaError_t launch_select_topk_layers(int n_layers, const float* scores, int BH, int L, int w, const int* n_keep,
                                       int32_t* const* kept, cudaStream_t st);
 
+// per-head token counts under a shared layer budget; kept_flat: scratch int32 [Bt, min(Hkv*(n_mean-w), Hkv*P) + 1]
+cudaError_t launch_head_budgets(const float* scores, int Bt, int Hkv, int L, int w, int n_mean, int unit,
+                                int32_t* n_heads, int32_t* kept_flat, cudaStream_t st);
+
 cudaError_t launch_gather_quantize(const void* K, const void* V, const int32_t* kept, int L, const qp_cache& c,
                                    cudaStream_t st);
 // n_layers caches of one shape (n_keep may differ) in one launch; kept[l] int32 [BH, caches[l].n_keep]

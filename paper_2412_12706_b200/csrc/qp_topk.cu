@@ -458,4 +458,56 @@ cudaError_t launch_select_topk_layers(int n_layers, const float* scores, int BH,
   return launch_topk<QP_MAX_LAYERS>(scores, n_layers * BH, BH, L, w, o, st);
 }
 
+// ---- head-level budgets: how many tokens each KV head of a layer keeps when the heads share the layer's budget
+namespace {
+// kept_flat [Bt, k_total + 1]: ascending indices h*P + j of the k_total marked positions of a batch entry (the
+// last entry is the selection kernel's window slot and is ignored).  One block per batch entry: a thread per
+// head counts its marked positions by two binary searches, thread 0 then applies the rounding rule in order.
+__global__ void __launch_bounds__(64)
+head_budget_kernel(const int32_t* __restrict__ kept_flat, int k_total, int Hkv, int P, int L, int w, int n_mean,
+                   int unit, int32_t* __restrict__ n_heads) {
+  extern __shared__ int s_n[];
+  const int b = blockIdx.x;
+  const int32_t* kf = kept_flat + (size_t)b * (k_total + 1);
+  auto lower = [&](long long key) {                 // first position whose index is >= key
+    int lo = 0, hi = k_total;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if ((long long)kf[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+  };
+  const int n_min = (w / unit) * unit + unit, n_max = max(n_min, (L / unit) * unit);
+  for (int h = threadIdx.x; h < Hkv; h += blockDim.x) {
+    const int raw = lower((long long)(h + 1) * P) - lower((long long)h * P) + w;
+    s_n[h] = min(n_max, max(n_min, (raw / unit) * unit));
+  }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  long long total = 0;
+  for (int h = 0; h < Hkv; ++h) total += s_n[h];
+  while (total > (long long)Hkv * n_mean) {        // the largest head (lowest first among equals) gives back a unit
+    int best = 0;
+    for (int h = 1; h < Hkv; ++h)
+      if (s_n[h] > s_n[best]) best = h;
+    if (s_n[best] <= n_min) break;
+    s_n[best] -= unit;
+    total -= unit;
+  }
+  for (int h = 0; h < Hkv; ++h) n_heads[(size_t)b * Hkv + h] = s_n[h];
+}
+}  // namespace
+
+cudaError_t launch_head_budgets(const float* scores, int Bt, int Hkv, int L, int w, int n_mean, int unit,
+                                int32_t* n_heads, int32_t* kept_flat, cudaStream_t st) {
+  const int P = L - w;
+  const long long k_total = std::min<long long>((long long)Hkv * (n_mean - w), (long long)Hkv * P);
+  // the marked positions: top-k over the row of all heads' scores (ties to the lower flat index = lower head,
+  // then lower position); the selection kernel wants a window, so the row gets one extra position
+  const cudaError_t e = launch_select_topk(scores, Bt, Hkv * P + 1, 1, (int)k_total + 1, kept_flat, st);
+  if (e != cudaSuccess) return e;
+  head_budget_kernel<<<Bt, 64, Hkv * sizeof(int), st>>>(kept_flat, (int)k_total, Hkv, P, L, w, n_mean, unit, n_heads);
+  return cudaGetLastError();
+}
+
 }  // namespace qp

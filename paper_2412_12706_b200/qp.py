@@ -26,7 +26,7 @@ EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_work
            "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static",
            "qp_cache_layout_cap", "qp_append_kv", "qp_append_kv_layers", "qp_decode_attn_tail",
            "qp_decode_attn_tail_layers", "qp_compress_layers", "qp_decode_overlap", "qp_gather_quantize_ex",
-           "qp_decode_attn_ex"]
+           "qp_decode_attn_ex", "qp_decode_attn_layers_ex", "qp_head_budgets", "qp_head_budgets_workspace_bytes"]
 
 
 class QpError(RuntimeError):
@@ -117,6 +117,12 @@ def lib() -> ctypes.CDLL:
         L.qp_gather_quantize_ex.argtypes = [p, p, p, i, cp, sp, p]
         L.qp_decode_attn_ex.restype = i
         L.qp_decode_attn_ex.argtypes = [p, cp, sp, p, p, sz, p]
+        L.qp_decode_attn_layers_ex.restype = i
+        L.qp_decode_attn_layers_ex.argtypes = [i, ctypes.POINTER(p), cp, sp, ctypes.POINTER(p), p, sz, p]
+        L.qp_head_budgets_workspace_bytes.restype = sz
+        L.qp_head_budgets_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.qp_head_budgets.restype = i
+        L.qp_head_budgets.argtypes = [p, i, i, i, i, i, i, p, p, sz, p]
         L.qp_decode_overlap.restype = i
         L.qp_decode_overlap.argtypes = [p, i]
         _lib = L
@@ -489,6 +495,92 @@ def decode_attn_ex(q: torch.Tensor, cache: Cache, strategy: Strategy, out: torch
     return out
 
 
+def decode_attn_layers_ex(qs: list[torch.Tensor], caches: list[Cache], strategy: Strategy, outs: list[torch.Tensor],
+                          workspace: torch.Tensor | None = None) -> None:
+    n = len(caches)
+    assert 1 <= n <= QP_MAX_LAYERS and len(qs) == n and len(outs) == n
+    if workspace is None:
+        workspace = new_decode_workspace(sum(decode_workspace_bytes(c) for c in caches), qs[0].device)
+    arr = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+    _check(lib().qp_decode_attn_layers_ex(n, arr(qs), (qp_cache * n)(*[c.desc for c in caches]),
+                                          ctypes.byref(strategy.desc), arr(outs), _ptr(workspace), workspace.numel(),
+                                          _stream()), "qp_decode_attn_layers_ex")
+
+
+def head_budgets(scores: torch.Tensor, L: int, w: int, n_mean: int, unit: int = 32) -> torch.Tensor:
+    """qp_head_budgets: scores fp32 [Bt,Hkv,P] (device) -> tokens kept per KV head, int32 [Bt,Hkv] (device)."""
+    assert scores.is_cuda and scores.dtype == torch.float32 and scores.is_contiguous()
+    Bt, Hkv, P = scores.shape
+    assert P == L - w
+    out = torch.empty((Bt, Hkv), dtype=torch.int32, device=scores.device)
+    ws = torch.empty(max(16, int(lib().qp_head_budgets_workspace_bytes(Bt, Hkv, L, w, n_mean))), dtype=torch.uint8,
+                     device=scores.device)
+    _check(lib().qp_head_budgets(_ptr(scores), Bt, Hkv, L, w, n_mean, unit, _ptr(out), _ptr(ws), ws.numel(), _stream()),
+           "qp_head_budgets")
+    return out
+
+
+@dataclass
+class HeadCaches:
+    """One packed cache per (batch, KV head) of a layer pruned with head-level budgets (descriptors with
+    batch = 1, n_kv_heads = 1, n_q_heads = G), in (batch, head) order, and the strategy they were written with."""
+    caches: list
+    kept: list
+    n_heads: list            # tokens kept per (batch, KV head), host ints
+    strategy: "Strategy | None"
+    shape: tuple             # (Bt, Hq, Hkv, D)
+
+
+def compress_layer_heads(K: torch.Tensor, V: torch.Tensor, Q_win: torch.Tensor, n_mean: int, bits: int, group: int = 32,
+                         pool: int = 7, k_axis: int = 1, unit: int | None = None) -> HeadCaches:
+    """The prefill-side path with head-level budgets: qp_window_scores -> qp_head_budgets -> (one copy of the
+    Bt x Hkv counts to the host, to size the heads' caches) -> per head qp_select_topk and
+    qp_gather_quantize(_ex).  k_axis = 1: keys per token, the arrangement the paper pairs with these methods;
+    k_axis = 0: the main path's per-channel keys (unit must then be a multiple of the group)."""
+    _dev_bf16(K); _dev_bf16(V); _dev_bf16(Q_win)
+    Bt, Hq, Hkv, D, L, w = _dims(K, Q_win)
+    G = Hq // Hkv
+    unit = unit or group
+    scores = window_scores(Q_win, K, pool)
+    n_dev = head_budgets(scores, L, w, n_mean, unit)
+    n_host = n_dev.cpu().view(-1).tolist()             # the one host round trip of this path
+    caches, kepts = [], []
+    strategy = None
+    for i, n in enumerate(n_host):
+        b, h = divmod(i, Hkv)
+        c = alloc_cache(1, G, 1, D, bits, group, n, K.device)
+        kept = torch.empty((1, 1, n), dtype=torch.int32, device=K.device)
+        _check(lib().qp_select_topk(scores[b, h].data_ptr(), 1, 1, L, w, n, _ptr(kept), _stream()), "qp_select_topk")
+        if bits == 16 or k_axis == 0:
+            _check(lib().qp_gather_quantize(K[b, h].data_ptr(), V[b, h].data_ptr(), _ptr(kept), L, ctypes.byref(c.desc),
+                                            _stream()), "qp_gather_quantize")
+        else:
+            strategy = strategy or make_strategy(c, 1, None)
+            _check(lib().qp_gather_quantize_ex(K[b, h].data_ptr(), V[b, h].data_ptr(), _ptr(kept), L, ctypes.byref(c.desc),
+                                               ctypes.byref(strategy.desc), _stream()), "qp_gather_quantize_ex")
+        caches.append(c); kepts.append(kept)
+    return HeadCaches(caches, kepts, n_host, strategy, (Bt, Hq, Hkv, D))
+
+
+def decode_attn_heads(q: torch.Tensor, hc: HeadCaches, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Decode attention over the per-head caches of compress_layer_heads: q, out bf16 [Bt,Hq,D]; every head is one
+    entry of a multi-cache call (qp_decode_attn_layers, or qp_decode_attn_layers_ex for per-token keys)."""
+    _dev_bf16(q)
+    Bt, Hq, Hkv, D = hc.shape
+    G = Hq // Hkv
+    if out is None:
+        out = torch.empty_like(q)
+    qv, ov = q.view(Bt * Hkv, 1, G, D), out.view(Bt * Hkv, 1, G, D)
+    for lo in range(0, len(hc.caches), QP_MAX_LAYERS):
+        hi = min(len(hc.caches), lo + QP_MAX_LAYERS)
+        qs, outs = [qv[i] for i in range(lo, hi)], [ov[i] for i in range(lo, hi)]
+        if hc.strategy is None:
+            decode_attn_layers(LayerBatch(qs, hc.caches[lo:hi], outs))
+        else:
+            decode_attn_layers_ex(qs, hc.caches[lo:hi], hc.strategy, outs)
+    return out
+
+
 # the C entry points under their own names
 qp_status_string = status_string
 qp_n_keep = n_keep
@@ -506,6 +598,9 @@ qp_decode_attn_static = decode_attn_static
 qp_decode_overlap = decode_overlap
 qp_gather_quantize_ex = gather_quantize_ex
 qp_decode_attn_ex = decode_attn_ex
+qp_decode_attn_layers_ex = decode_attn_layers_ex
+qp_head_budgets = head_budgets
+qp_head_budgets_workspace_bytes = lambda *a: int(lib().qp_head_budgets_workspace_bytes(*a))
 qp_cache_layout_cap = cache_layout_cap
 qp_append_kv = append_kv
 qp_append_kv_layers = append_kv_layers

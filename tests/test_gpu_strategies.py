@@ -110,7 +110,6 @@ def test_side_list_overflow_is_reported_not_written_past_the_end():
     torch.cuda.synchronize()
     assert int(st.bufs[0][2][0, 0]) == -1                            # keys: overflow flagged
     assert bool((big[0][8:] == -7).all()) and bool((big[1][8:] == -7.0).all()) and bool((big[0][:8] >= 0).all())
-    assert int(st.bufs[1][2][0, 0]) >= 0                             # values: fits
 
 
 def test_strategy_arguments_are_checked_before_any_launch():
