@@ -103,7 +103,7 @@ __device__ __forceinline__ uint32_t sw128_off(int r, int c) {
 
 template <int PASS, int D, int NL>
 __global__ void __launch_bounds__(TC_THREADS, 2)
-score_sweep_tc_kernel(const __grid_constant__ ScorePtrs<NL> ptrs, int BH, int Hq, int Hkv, int L, int w,
+score_sweep_tc_kernel(const __grid_constant__ ScorePtrs<NL> ptrs, int bh0, int BH, int Hq, int Hkv, int L, int w,
                       int n_rb, int n_tiles, int tiles_per_block, float scale_log2,
                       float2* __restrict__ stat_partial, const float2* __restrict__ rowstat,
                       float* __restrict__ votes_partial, int* __restrict__ error_word) {
@@ -119,7 +119,7 @@ score_sweep_tc_kernel(const __grid_constant__ ScorePtrs<NL> ptrs, int BH, int Hq
   const int tid = threadIdx.x, warp = tid >> 5;
   const int rloc = tid & (TC_M - 1), half = tid >> 7, wq = warp & 3;   // row in the block, column half, TMEM lane quarter
   // bh counts (layer, batch, KV head): the scratch arrays are laid out over all of them, the inputs are per layer
-  const int split = blockIdx.x, rb = blockIdx.y, bh = blockIdx.z, layer = bh / BH, bhl = bh % BH;
+  const int split = blockIdx.x, rb = blockIdx.y, bh = bh0 + blockIdx.z, layer = bh / BH, bhl = bh % BH;
   const bf16* __restrict__ Qwin = ptrs.q[layer];
   const bf16* __restrict__ K = ptrs.k[layer];
   const int b = bhl / Hkv, hk = bhl % Hkv, G = Hq / Hkv, P = L - w, R = G * w;
@@ -293,24 +293,23 @@ bool score_tc_supported(int D) { return D == 128 || D == 64; }
 
 namespace {
 template <int PASS, int D, int NL>
-cudaError_t launch_tc(dim3 grid, cudaStream_t st, const ScorePtrs<NL>& ptrs, const ScoreDims& d, const ScoreWorkspace& s,
+cudaError_t launch_tc(dim3 grid, int bh0, cudaStream_t st, const ScorePtrs<NL>& ptrs, const ScoreDims& d, const ScoreWorkspace& s,
                       int per, float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
                       int* error_word) {
   constexpr size_t smem = 3 * (size_t)TC_M * D * 2 + 1024;   // Q + two K stages + alignment slack
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(score_sweep_tc_kernel<PASS, D, NL>, smem, done);
   if (e != cudaSuccess) return e;
-  score_sweep_tc_kernel<PASS, D, NL><<<grid, TC_THREADS, smem, st>>>(ptrs, d.Bt * d.Hkv, d.Hq, d.Hkv, d.L, d.w, s.n_rb,
+  score_sweep_tc_kernel<PASS, D, NL><<<grid, TC_THREADS, smem, st>>>(ptrs, bh0, d.Bt * d.Hkv, d.Hq, d.Hkv, d.L, d.w, s.n_rb,
                                                                     s.n_tiles, per, scale_log2, stat_partial, rowstat,
                                                                     votes_partial, error_word);
   return cudaGetLastError();
 }
 
 template <int NL>
-cudaError_t launch_sweep(int pass, const ScorePtrs<NL>& ptrs, int n_layers, const ScoreDims& d, const ScoreWorkspace& s,
+cudaError_t launch_sweep(int pass, const ScorePtrs<NL>& ptrs, int bh0, int BH, const ScoreDims& d, const ScoreWorkspace& s,
                          float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
                          int* error_word, cudaStream_t st) {
-  const int BH = d.Bt * d.Hkv * n_layers;
   const int tiles = pass == 1 ? s.n_tiles : s.n_vote_tiles;
   // enough blocks for two per SM over a few waves, at least two tiles per block
   long long per = ((long long)tiles * s.n_rb * BH + 591) / 592;
@@ -319,29 +318,30 @@ cudaError_t launch_sweep(int pass, const ScorePtrs<NL>& ptrs, int n_layers, cons
   const int splits = (int)((tiles + per - 1) / per);
   const dim3 grid(splits, s.n_rb, BH);
   if (d.D == 128)
-    return pass == 1 ? launch_tc<1, 128, NL>(grid, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
-                     : launch_tc<2, 128, NL>(grid, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
-  return pass == 1 ? launch_tc<1, 64, NL>(grid, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
-                   : launch_tc<2, 64, NL>(grid, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
+    return pass == 1 ? launch_tc<1, 128, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
+                     : launch_tc<2, 128, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
+  return pass == 1 ? launch_tc<1, 64, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
+                   : launch_tc<2, 64, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
 }
 }  // namespace
 
 // s: the scratch layout for batch * n_layers batch entries (the layers are stacked along the batch dimension)
+// bh0, bh_count: the (layer, batch, KV head) triples this launch covers
 cudaError_t launch_score_sweep_tc(int pass, int n_layers, const void* const* q, const void* const* k, const ScoreDims& d,
                                   const ScoreWorkspace& s, float scale_log2, float2* stat_partial, const float2* rowstat,
-                                  float* votes_partial, int* error_word, cudaStream_t st) {
+                                  float* votes_partial, int* error_word, cudaStream_t st, int bh0, int bh_count) {
   if (n_layers == 1) {
     ScorePtrs<1> p;
     p.q[0] = static_cast<const bf16*>(q[0]);
     p.k[0] = static_cast<const bf16*>(k[0]);
-    return launch_sweep<1>(pass, p, 1, d, s, scale_log2, stat_partial, rowstat, votes_partial, error_word, st);
+    return launch_sweep<1>(pass, p, bh0, bh_count, d, s, scale_log2, stat_partial, rowstat, votes_partial, error_word, st);
   }
   ScorePtrs<QP_MAX_LAYERS> p;
   for (int l = 0; l < n_layers; ++l) {
     p.q[l] = static_cast<const bf16*>(q[l]);
     p.k[l] = static_cast<const bf16*>(k[l]);
   }
-  return launch_sweep<QP_MAX_LAYERS>(pass, p, n_layers, d, s, scale_log2, stat_partial, rowstat, votes_partial,
+  return launch_sweep<QP_MAX_LAYERS>(pass, p, bh0, bh_count, d, s, scale_log2, stat_partial, rowstat, votes_partial,
                                      error_word, st);
 }
 
