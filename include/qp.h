@@ -343,6 +343,18 @@ qp_status qp_decode_attn_layers_ex(int n_layers, const void* const* q, const qp_
                                    size_t workspace_bytes, void* stream);
 
 /*
+ * Debug build only (libqp_checked.so, compiled with -DQP_CHECKED; no counterpart in the paper).  In that build
+ * every index a kernel reads from DEVICE memory and then uses as an address (the kept positions given to the
+ * gather / quantize kernels, the side lists' tile pointers and entries) is compared with its limit first; a
+ * violation never traps: the first one is recorded, all are counted, and the access goes to element 0 or is
+ * skipped.  This call synchronises the device, copies the record to words4 (host: 1 + site of the first
+ * violation or 0, the offending index, its limit, the number of violations) and clears it.  Indices that
+ * come from host fields (n_keep, n_cap, n_tail, shapes) are validated by every entry point before any launch in
+ * both builds.  The normal build returns QP_ERR_UNSUPPORTED and zeros.
+ */
+qp_status qp_debug_check(uint32_t* words4 /* host, out */);
+
+/*
  * Decode attention without any caller-supplied scratch.  (The paper has no counterpart to this
  * call; it exists for integration reasons only.)  Some hosts of this library cannot give it
  * scratch memory: a serving process that hands all device memory to its own arena at start-up,

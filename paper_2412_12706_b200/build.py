@@ -9,6 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqp.so")
+LIB_CHECKED = os.path.join(HERE, "libqp_checked.so")   # the same sources with -DQP_CHECKED (device-side range checks)
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--shared", "-Xptxas", "-v"]
@@ -19,9 +20,9 @@ def sources() -> list[str]:
 
 
 def needs_build() -> bool:
-    if not os.path.exists(LIB):
+    if not os.path.exists(LIB) or not os.path.exists(LIB_CHECKED):
         return True
-    t = os.path.getmtime(LIB)
+    t = min(os.path.getmtime(LIB), os.path.getmtime(LIB_CHECKED))
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + \
         [os.path.join(os.path.dirname(HERE), "include", "qp.h")]
     return any(os.path.getmtime(p) > t for p in deps)
@@ -31,12 +32,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + os.environ.get("QP_NVCC_EXTRA", "").split() + ["-o", LIB] + sources()
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed building libqp.so")
+    extra = os.environ.get("QP_NVCC_EXTRA", "").split()
+    cmds = [[nvcc] + NVCC_FLAGS + extra + ["-o", LIB] + sources(),
+            [nvcc] + NVCC_FLAGS + extra + ["-DQP_CHECKED", "-o", LIB_CHECKED] + sources()]
+    procs = [subprocess.Popen(c, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True) for c in cmds]
+    for p, target in zip(procs, (LIB, LIB_CHECKED)):
+        out, _ = p.communicate()
+        if verbose or p.returncode != 0:
+            sys.stderr.write(out)
+        if p.returncode != 0:
+            raise RuntimeError(f"nvcc failed building {os.path.basename(target)}")
     return LIB
 
 

@@ -6,6 +6,7 @@
 // form in the log2 domain, and each block leaves one partial (m, l, acc[D]) per query head.
 // A second kernel merges the partials of a (batch, query head) in a fixed order.
 // No block ever waits for another one.
+#include "qp_checked.cuh"
 #include "qp_common.cuh"
 
 namespace qp {
@@ -112,8 +113,10 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
         const int32_t* tp = ex.k.tile_ptr + (size_t)bh * (ex.k.n_tiles + 1) + (tile >> 5);
         const int32_t* sidx = ex.k.idx + (size_t)bh * ex.k.cap;
         const uint16_t* sval = ex.k.val + (size_t)bh * ex.k.cap;
-        for (int i = tp[0]; i < tp[1]; ++i) {
+        const bool ptr_ok = QP_IN_RANGE(tp[0], ex.k.cap + 1, QP_SITE_SIDE_PTR) && QP_IN_RANGE(tp[1], ex.k.cap + 1, QP_SITE_SIDE_PTR);
+        for (int i = ptr_ok ? tp[0] : 0; i < (ptr_ok ? tp[1] : 0); ++i) {
           const int fi = sidx[i], t2 = fi / D, d = fi % D;      // warp-uniform
+          if (!QP_IN_RANGE(fi, (long long)n * D, QP_SITE_SIDE_IDX)) continue;
           if (t2 == tok) {
             const size_t gi = ex.k_axis == 1 ? ((size_t)bh * ns + t2) * ngv + d / g
                                              : ((size_t)bh * (ns / g) + t2 / g) * D + d;
@@ -180,8 +183,10 @@ decode_generic_kernel(const __grid_constant__ DecTable tab, const DecDims dm, fl
         const int32_t* tp = ex.v.tile_ptr + (size_t)bh * (ex.v.n_tiles + 1) + (tile >> 5);
         const int32_t* sidx = ex.v.idx + (size_t)bh * ex.v.cap;
         const uint16_t* sval = ex.v.val + (size_t)bh * ex.v.cap;
-        for (int i = tp[0]; i < tp[1]; ++i) {
+        const bool ptr_ok = QP_IN_RANGE(tp[0], ex.v.cap + 1, QP_SITE_SIDE_PTR) && QP_IN_RANGE(tp[1], ex.v.cap + 1, QP_SITE_SIDE_PTR);
+        for (int i = ptr_ok ? tp[0] : 0; i < (ptr_ok ? tp[1] : 0); ++i) {
           const int fi = sidx[i], t2 = fi / D, d = fi % D;      // warp-uniform
+          if (!QP_IN_RANGE(fi, (long long)n * D, QP_SITE_SIDE_IDX) || t2 < tile || t2 >= tile + 32) continue;
           const size_t gi = ((size_t)bh * ns + t2) * ngv + d / g;
           const float delta = bf16_bits_to_f32(sval[i]) - __half2float(ly.vz[gi]);
 #pragma unroll
@@ -386,5 +391,9 @@ size_t decode_plan_chunked(DecTable& tab, const DecDims& d) {
   }
   return slots * record_bytes(d);
 }
+
+#ifdef QP_CHECKED
+cudaError_t decode_check_read(unsigned int (&out)[4]) { return checked::read_and_clear(out); }
+#endif
 
 }  // namespace qp

@@ -9,6 +9,7 @@
 // codes, scales and zeros are reproducible bit for bit.
 #include <algorithm>
 
+#include "qp_checked.cuh"
 #include "qp_common.cuh"
 
 namespace qp {
@@ -96,7 +97,10 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   const int ud = ql.u0 + u;                        // destination group
   const int wpg = g * BITS / 32;
 
-  for (int e = tid; e < g; e += nthr) sidx[e] = kept ? kept[(size_t)bh * n + (size_t)u * g + e] : u * g + e;
+  for (int e = tid; e < g; e += nthr) {
+    const int src = kept ? kept[(size_t)bh * n + (size_t)u * g + e] : u * g + e;
+    sidx[e] = QP_IN_RANGE(src, L, QP_SITE_GATHER_KEPT) ? src : 0;
+  }
   __syncthreads();
   const uint16_t* Kh = K + (size_t)bh * L * D;
   const uint16_t* Vh = V + (size_t)bh * L * D;
@@ -216,7 +220,8 @@ side_list_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ V,
     int t = 0, d0 = 0;
     if (c < total8) {
       t = (c * 8) / D; d0 = (c * 8) % D;
-      const uint4 q = *reinterpret_cast<const uint4*>(X + (size_t)(kp ? kp[t] : t) * D + d0);
+      const int pos = kp ? kp[t] : t;
+      const uint4 q = *reinterpret_cast<const uint4*>(X + (size_t)(QP_IN_RANGE(pos, L, QP_SITE_SIDE_KEPT) ? pos : 0) * D + d0);
       w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
     }
     unsigned mask = 0;
@@ -268,7 +273,8 @@ gather_rows_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ 
   const int rows_per_blk = blockDim.x / cpr;
   const int t = blockIdx.x * rows_per_blk + threadIdx.x / cpr, c = (threadIdx.x % cpr) * 8;
   if (t >= n || (int)threadIdx.x >= rows_per_blk * cpr) return;
-  const size_t src = ((size_t)bh * L + kept[(size_t)bh * n + t]) * D + c;
+  const int pos = kept[(size_t)bh * n + t];
+  const size_t src = ((size_t)bh * L + (QP_IN_RANGE(pos, L, QP_SITE_ROWS_KEPT) ? pos : 0)) * D + c;
   const size_t dst = ((size_t)bh * ns + t) * D + c;   // ns: tokens the destination has room for
   *reinterpret_cast<uint4*>(Ko + dst) = *reinterpret_cast<const uint4*>(K + src);
   *reinterpret_cast<uint4*>(Vo + dst) = *reinterpret_cast<const uint4*>(V + src);
@@ -433,5 +439,9 @@ cudaError_t launch_flush_tails(int n_layers, const int* which, const qp_cache* c
   for (int i = 0; i < n_layers; ++i) fill(tab.l[i], which[i]);
   return launch_quant_table<QP_MAX_LAYERS>(c0.bits, tab, dim3(2, BH, n_layers), D, g, st);
 }
+
+#ifdef QP_CHECKED
+cudaError_t quant_check_read(unsigned int (&out)[4]) { return checked::read_and_clear(out); }
+#endif
 
 }  // namespace qp

@@ -14,7 +14,8 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libqp.so")
+# QP_LIBRARY selects another build of the same library (the range-checked debug build libqp_checked.so)
+LIB_PATH = os.environ.get("QP_LIBRARY") or os.path.join(_HERE, "libqp.so")
 
 QP_OK = 0
 QP_MAX_LAYERS = 128
@@ -26,7 +27,7 @@ EXPORTS = ["qp_status_string", "qp_n_keep", "qp_cache_layout", "qp_compress_work
            "qp_compress_layer", "qp_decode_attn", "qp_decode_attn_layers", "qp_decode_attn_static",
            "qp_cache_layout_cap", "qp_append_kv", "qp_append_kv_layers", "qp_decode_attn_tail",
            "qp_decode_attn_tail_layers", "qp_compress_layers", "qp_decode_overlap", "qp_gather_quantize_ex",
-           "qp_decode_attn_ex", "qp_decode_attn_layers_ex", "qp_head_budgets", "qp_head_budgets_workspace_bytes"]
+           "qp_decode_attn_ex", "qp_decode_attn_layers_ex", "qp_head_budgets", "qp_head_budgets_workspace_bytes", "qp_debug_check"]
 
 
 class QpError(RuntimeError):
@@ -123,6 +124,8 @@ def lib() -> ctypes.CDLL:
         L.qp_head_budgets_workspace_bytes.argtypes = [i, i, i, i, i]
         L.qp_head_budgets.restype = i
         L.qp_head_budgets.argtypes = [p, i, i, i, i, i, i, p, p, sz, p]
+        L.qp_debug_check.restype = i
+        L.qp_debug_check.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         L.qp_decode_overlap.restype = i
         L.qp_decode_overlap.argtypes = [p, i]
         _lib = L
@@ -581,6 +584,14 @@ def decode_attn_heads(q: torch.Tensor, hc: HeadCaches, out: torch.Tensor | None 
     return out
 
 
+def debug_check() -> tuple[int, list[int]]:
+    """qp_debug_check: (status, [1 + site of the first violation or 0, index, limit, violations]); status is
+    QP_ERR_UNSUPPORTED (2) unless the loaded library is the range-checked build."""
+    w = (ctypes.c_uint32 * 4)()
+    st = lib().qp_debug_check(w)
+    return st, list(w)
+
+
 # the C entry points under their own names
 qp_status_string = status_string
 qp_n_keep = n_keep
@@ -598,6 +609,7 @@ qp_decode_attn_static = decode_attn_static
 qp_decode_overlap = decode_overlap
 qp_gather_quantize_ex = gather_quantize_ex
 qp_decode_attn_ex = decode_attn_ex
+qp_debug_check = debug_check
 qp_decode_attn_layers_ex = decode_attn_layers_ex
 qp_head_budgets = head_budgets
 qp_head_budgets_workspace_bytes = lambda *a: int(lib().qp_head_budgets_workspace_bytes(*a))

@@ -135,6 +135,35 @@ def test_decode_matches_oracle(bits, Hq, Hkv, D, group, n):
         assert err <= 3e-3 + 2.0 ** -7 * np.abs(ref).max(), err
 
 
+@pytest.mark.parametrize("bits", [2, 4, 8, 16])
+def test_decode_at_the_documented_magnitude_bounds(bits):
+    """max|q| * max|K| just inside 2^19 and max|V| just inside 4096 (the decode calls' stated input range): the
+    f16 products of the tensor-core path (query x key scale, softmax weight x value scale) stay finite and the
+    result stays within the decode tolerance."""
+    Hq, Hkv, D, n, group = 8, 2, 128, 1024, 32
+    wl = small(synth.TINY, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, L=n, batch=1, group=group)
+    k, v, _ = make_inputs(wl)
+    k, v = k.float(), v.float()
+    k[..., 7] *= 2000.0 / float(k[..., 7].abs().max())          # one key channel carries the large magnitudes
+    v *= 4000.0 / float(v.abs().max())
+    k, v = k.to(torch.bfloat16), v.to(torch.bfloat16)
+    kmax = float(k.float().abs().max())
+    q = synth.make_q_dec(wl, 0, 0).float()
+    q[..., 7] = torch.sign(q[..., 7]) * (0.97 * 2.0 ** 19 / kmax)
+    q = q.to(torch.bfloat16)
+    assert float(q.float().abs().max()) * kmax <= 2.0 ** 19 and float(v.float().abs().max()) <= 4096
+    kept = np.broadcast_to(np.arange(n, dtype=np.int32), (1, Hkv, n)).copy()
+    pk = orc.quantize(bits_u16(k), bits_u16(v), kept, bits, group)
+    cache = qp.alloc_cache(1, Hq, Hkv, D, bits, group, n, DEV)
+    qp.gather_quantize(k.to(DEV), v.to(DEV), torch.from_numpy(kept).to(DEV), cache)
+    assert_packed_equal(cache_to_packed(cache), pk)
+    kd, vd = orc.dequantize(pk, D)
+    ref = orc.decode(bits_u16(q), kd, vd)
+    out = qp.decode_attn(q.to(DEV), cache).float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(out).all()
+    assert np.abs(out - ref).max() <= decode_tolerance(ref), (np.abs(out - ref).max(), decode_tolerance(ref))
+
+
 def test_decode_16bit_ragged_length_and_zero_query_mean():
     wl = small(synth.TINY, L=1000, batch=1)
     k, v, _ = make_inputs(wl)
