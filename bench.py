@@ -279,7 +279,7 @@ def per_config_figures(args, qp, dev, peak, stream, rank):
             ws_d = qp.new_decode_workspace(sum(qp.decode_workspace_bytes(c) for c in seqs[0][b]), dev)
             batches = [qp.LayerBatch(q[(i + s) % 4], seqs[s][b], outs, ws_d) for i in range(2) for s in range(n_rot)]
             bytes_call = model_bytes(wl)
-            reps = int(max(32, min(2048, 0.04 / (bytes_call / 5e12))))
+            reps = int(max(32, min(4096, 0.08 / (bytes_call / 5e12))))     # about 0.1 s per figure: clocks settle under load
             ms_on = time_calls(qp, batches, reps, True, stream)
             ms_off = time_calls(qp, batches, reps, False, stream)
             ach = bytes_call / (ms_on * 1e-3) / 1e9
@@ -395,7 +395,7 @@ def run_gpu(args, wl):
     if not args.lean and world == 1:       # single-GPU side figures
         # ---- the same decode calls in plain stream order (the library's default)
         flat = [grp[t] for t in range(n_q) for grp in groups]
-        reps = int(max(16, min(1024, 0.05 / (dec_bytes_call / 5e12))))
+        reps = int(max(16, min(4096, 0.12 / (dec_bytes_call / 5e12))))     # a sustained loop, like the timed region's
         off_ms = time_calls(qp, flat, reps, False, stream)
         extras["decode_stream_order"] = {"note": "the same calls without qp_decode_overlap (the library's default)",
                                          "us_per_call": off_ms * 1e3, "GB/s": dec_bytes_call / (off_ms * 1e-3) / 1e9}

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "qp_common.cuh"
+#include "qp_mma.cuh"
 
 using namespace qp;
 
@@ -513,6 +514,15 @@ qp_status qp_decode_attn_layers_ex(int n_layers, const void* const* q, const qp_
   }
   if (filter && n_layers > 1) return QP_ERR_UNSUPPORTED;
   const DecDims d{c0.batch, c0.n_q_heads, c0.n_kv_heads, c0.head_dim, c0.bits, c0.group};
+  if (!filter && strategy->k_axis == 1 && decode_mma4t_supported(d)) {
+    // per-token keys at 4 bit without side lists: the tensor-core kernel and the flat-range merge, plain stream order
+    const size_t need_flat = decode_plan_flat(tab, d, decode_mma4t_workers_per_sm(), 4);
+    if (workspace_bytes < need_flat) return QP_ERR_WORKSPACE;
+    cache_written(static_cast<cudaStream_t>(stream));
+    float* partials = static_cast<float*>(workspace);
+    if (launch_decode_mma4t(tab, d, partials, static_cast<cudaStream_t>(stream)) != cudaSuccess) return QP_ERR_CUDA;
+    return launch_merge_flat(tab, d, partials, static_cast<cudaStream_t>(stream)) == cudaSuccess ? QP_OK : QP_ERR_CUDA;
+  }
   if (workspace_bytes < decode_plan_chunked(tab, d)) return QP_ERR_WORKSPACE;
   DecEx ex{};
   ex.k_axis = strategy->k_axis;

@@ -176,7 +176,9 @@ constexpr int kMaxDecodeWorkers = QP_MAX_DECODE_WORKERS;
 // paired: the stream lets consecutive calls overlap (two calls share the GPU most of the time), so a small launch
 // does better with fewer, longer-lived workers; alone on the GPU it wants as many as it can feed.
 size_t decode_plan(DecTable& tab, const DecDims& d, bool paired);
-size_t decode_plan_chunked(DecTable& tab, const DecDims& d);   // the chunked decomposition, whatever the shape
+size_t decode_plan_chunked(DecTable& tab, const DecDims& d);
+// the flat-range decomposition for a kernel with `workers_per_sm` resident workers; returns the bytes of ONE record area
+size_t decode_plan_flat(DecTable& tab, const DecDims& d, int workers_per_sm, int tiles_per_worker_min);   // the chunked decomposition, whatever the shape
 // Upper bound of decode_plan's result for one layer of n_keep tokens, whatever else is in the launch.
 size_t decode_workspace_bound(const DecDims& d, int n_keep);
 // Workspace of the tensor-core kernels: two areas of partial records, used by alternate calls (parity), so that

@@ -6,6 +6,8 @@
 // form in the log2 domain, and each block leaves one partial (m, l, acc[D]) per query head.
 // A second kernel merges the partials of a (batch, query head) in a fixed order.
 // No block ever waits for another one.
+#include <algorithm>
+
 #include "qp_checked.cuh"
 #include "qp_common.cuh"
 
@@ -375,6 +377,24 @@ cudaError_t launch_decode_ex(const DecTable& tab, const DecDims& d, const DecEx&
   if (e != cudaSuccess) return e;
   decode_merge_kernel<<<dim3(d.Bt * d.Hq, tab.n_layers), 128, 0, st>>>(tab, d, partials);
   return cudaGetLastError();
+}
+
+size_t decode_plan_flat(DecTable& tab, const DecDims& d, int workers_per_sm, int tiles_per_worker_min) {
+  const int BH = d.Bt * d.Hkv;
+  long long T = 0;
+  for (int l = 0; l < tab.n_layers; ++l) {
+    tab.l[l].tile_base = (int)T;
+    tab.l[l].part_base = 0;
+    T += (long long)BH * ((tab.l[l].n + 31) / 32);
+  }
+  long long W = std::min<long long>((long long)sm_count() * workers_per_sm, kMaxDecodeWorkers);
+  W = std::min(W, (T + tiles_per_worker_min - 1) / tiles_per_worker_min);
+  if (W < 1) W = 1;
+  while (W > 1 && T * W >= (1ll << 31)) W /= 2;
+  tab.total_tiles = (int)T;
+  tab.n_workers = (int)W;
+  tab.chunk = tab.wide = tab.paired = 0;
+  return decode_workspace_layout(tab, d).record_bytes;
 }
 
 size_t decode_plan_chunked(DecTable& tab, const DecDims& d) {

@@ -673,6 +673,10 @@ cudaError_t launch_decode_mma(const DecTable& tab, const DecDims& d, float* part
                                 : launch_decode_mma2(tab, d, partials, st, overlap_prev);
   if (e != cudaSuccess) return e;
   if (tails) return launch_merge_tail(tab, d, partials, *tails, st, true);
+  return launch_merge_flat(tab, d, partials, st);
+}
+
+cudaError_t launch_merge_flat(const DecTable& tab, const DecDims& d, const float* partials, cudaStream_t st) {
   const int items = d.Bt * d.Hq * tab.n_layers;
   cudaLaunchConfig_t cfg = {};
   const int row_blocks = (items + MG_WARPS - 1) / MG_WARPS;

@@ -111,6 +111,12 @@ cudaError_t launch_decode_mma8(const DecTable& tab, const DecDims& d, float* par
 int decode_mma8_blocks_per_sm();
 int decode_mma8_warps();
 cudaError_t launch_decode_mma16(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st, bool overlap_prev);
+// 4-bit caches whose keys are quantized token by token (qp_strategy.k_axis = 1): attention kernel only
+bool decode_mma4t_supported(const DecDims& d);
+int decode_mma4t_workers_per_sm();
+cudaError_t launch_decode_mma4t(const DecTable& tab, const DecDims& d, float* partials, cudaStream_t st);
+// the merge kernels of the flat-range decomposition (records of every attention kernel above)
+cudaError_t launch_merge_flat(const DecTable& tab, const DecDims& d, const float* partials, cudaStream_t st);
 int decode_mma16_blocks_per_sm();
 
 // opt in to more than 48 KB of dynamic shared memory, once per device and kernel

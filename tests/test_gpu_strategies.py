@@ -31,6 +31,7 @@ def _side_np(bufs):
 
 @pytest.mark.parametrize("bits,group,D,G,k_axis,thr", [
     (4, 32, 128, 4, 1, None), (4, 64, 128, 4, 1, None), (2, 32, 128, 4, 1, None), (8, 32, 64, 2, 1, None),
+    (4, 32, 64, 8, 1, None), (4, 128, 128, 2, 1, None), (4, 64, 64, 3, 1, None), (4, 32, 128, 8, 1, None),
     (4, 32, 128, 4, 0, 6.0), (4, 64, 128, 4, 1, 6.0), (2, 32, 64, 8, 1, 6.0), (8, 128, 128, 1, 0, 6.0),
     (2, 32, 128, 3, 0, 6.0)])
 def test_quantize_and_decode_under_a_strategy(bits, group, D, G, k_axis, thr):
