@@ -299,6 +299,75 @@ def per_config_figures(args, qp, dev, peak, stream, rank):
     return out
 
 
+def strategy_figures(qp, dev, peak, stream, rank):
+    """Decode figures of the rows beyond the main path, on the Llama-3-8B 8k shapes at 4 bit: the FlexGen arrangement
+    (keys per token, g = 64, the paper's setting for it), outlier filtering (|x| > 6 kept in 16 bit) and head-level
+    budgets.  One sequence per call where the entry point takes several caches."""
+    wl = synth.LLAMA8B_8K
+    Bt, Hq, Hkv, D, L, w = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.L, wl.w
+    n, n_seq = wl.n_keep(0), 4
+    ws_c = torch.empty(qp.compress_workspace_bytes(Bt, Hq, Hkv, D, L, w), dtype=torch.uint8, device=dev)
+    flex, filt, heads = [], [], []
+    st_flex = st_filt = None
+    filt_cnt = 0
+    for s in range(n_seq):
+        wls = synth.dataclasses.replace(wl, seed=shard.sequence_seed(wl.seed, rank, 64, 32 + s))
+        fl = []
+        for l in range(wl.n_layers):
+            k, v = synth.make_kv(wls, l, device=dev)
+            qw = synth.make_q_win(wls, l, device=dev)
+            _, kept = qp.compress_layer(k, v, qw, wl.budget_bits, 4, 32, wl.pool, workspace=ws_c)
+            c = qp.alloc_cache(Bt, Hq, Hkv, D, 4, 64, n, dev)
+            st_flex = st_flex or qp.make_strategy(c, 1, None)
+            qp.gather_quantize_ex(k, v, kept, c, st_flex)
+            fl.append(c)
+            if s == 0 and l < 8:
+                c2 = qp.alloc_cache(Bt, Hq, Hkv, D, 4, 32, n, dev)
+                st2 = qp.make_strategy(c2, 0, 6.0)
+                qp.gather_quantize_ex(k, v, kept, c2, st2)
+                filt.append((c2, st2))
+                heads.append(qp.compress_layer_heads(k, v, qw, n, 4, 32, wl.pool, k_axis=1))
+        flex.append(fl)
+    torch.cuda.synchronize()
+    filt_cnt = sum(int(st.bufs[0][2].sum()) + int(st.bufs[1][2].sum()) for _, st in filt) / max(1, len(filt))
+    qs = [synth.make_q_dec(wl, l, 0, device=dev) for l in range(wl.n_layers)]
+    outs = [torch.empty_like(q) for q in qs]
+    ws = qp.new_decode_workspace(sum(qp.decode_workspace_bytes(c) for c in flex[0]), dev)
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn(0)
+        a, z = ev(), ev()
+        a.record(stream)
+        for r in range(reps):
+            fn(r)
+        z.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / reps
+
+    flex_bytes = Bt * Hkv * n * D * 2 * (4 + 32 // 64) // 8 * wl.n_layers
+    ms = timed(lambda r: qp.decode_attn_layers_ex(qs, flex[r % n_seq], st_flex, outs, ws), 512)
+    layer_bytes = Bt * Hkv * n * D * 2 * (4 + 1) // 8
+    ms_f = timed(lambda r: qp.decode_attn_ex(qs[0], filt[r % len(filt)][0], filt[r % len(filt)][1], outs[0], ws), 64)
+    ms_h = timed(lambda r: qp.decode_attn_heads(qs[0], heads[r % len(heads)], outs[0]), 64)
+    head_tokens = sum(sum(h.n_heads) for h in heads) / len(heads)
+    return {
+        "workload": wl.name + ", 4 bit",
+        "flexgen_g64": {"note": "keys and values per token, group 64; qp_decode_attn_layers_ex, 32 layers per call, plain "
+                                "stream order, rotating over 4 sequences", "bytes_per_call": flex_bytes,
+                        "us_per_call": ms * 1e3, "achieved": flex_bytes / (ms * 1e-3) / 1e9,
+                        "frac": flex_bytes / (ms * 1e-3) / 1e9 / peak},
+        "kivi_outliers": {"note": "per-channel keys, |x| > 6 kept in 16 bit (side lists); qp_decode_attn_ex, one layer per "
+                                  "call (the chunked kernel)", "outliers_per_layer": filt_cnt,
+                          "us_per_layer_call": ms_f * 1e3, "GB/s": layer_bytes / (ms_f * 1e-3) / 1e9},
+        "head_budgets": {"note": "per-head token counts under a shared layer budget, keys per token; one layer per call "
+                                 "(8 per-head caches in one qp_decode_attn_layers_ex call)",
+                         "tokens_per_head_min_max": [min(min(h.n_heads) for h in heads), max(max(h.n_heads) for h in heads)],
+                         "us_per_layer_call": ms_h * 1e3,
+                         "GB/s": head_tokens * D * 2 * (4 + 1) / 8 / (ms_h * 1e-3) / 1e9},
+    }
+
+
 def run_gpu(args, wl):
     from paper_2412_12706_b200 import qp
     dist, rank, world, local = shard.init_ranks("nccl")
@@ -516,12 +585,13 @@ def run_gpu(args, wl):
     e2e = None if args.no_e2e else run_e2e(args, wl, qp, seqs, groups, ws_c, dev, stream, per_call)
 
     # ---- the other configurations (decode, one sequence per call); the main workload's inputs are released first
-    per_config = None
+    per_config = strategies = None
     if not args.no_per_config and world == 1:
         for sq in seqs:
             sq["K"].clear(); sq["V"].clear(); sq["Qw"].clear()
         torch.cuda.empty_cache()
         per_config = per_config_figures(args, qp, dev, peak, stream, rank)
+        strategies = strategy_figures(qp, dev, peak, stream, rank)
     barrier()
 
     def allmax(x: float) -> float:
@@ -571,6 +641,7 @@ def run_gpu(args, wl):
         "gpu_launches": steps * (n_seq * n_layers * KERNELS_PER_COMPRESS + n_calls_step * KERNELS_PER_DECODE_CALL),
         "clocks": clocks,
         "per_config": per_config,
+        "strategies": strategies,
     }
     line.update(extras)
     if cpu is not None:

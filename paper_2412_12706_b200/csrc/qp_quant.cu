@@ -36,23 +36,42 @@ __device__ __forceinline__ QParams group_params(float mn, float mx, int qmax) {
 // (x - z) * (1/s), which is within 2^-22 relative (< 1e-4 absolute for codes up to 255) of it, so the
 // rounded integer can only differ when the estimate lies that close to a half-integer; only then is
 // the IEEE division done.  The result is the same integer in every case.
-// Rounding and the conversion to an integer use the 1.5 * 2^23 trick (adding that constant rounds a float
-// below 2^22 to the nearest integer, ties to even, and leaves the integer in the low mantissa bits): plain
-// additions instead of the conversion instructions, which issue at a quarter of the rate.
-__device__ __forceinline__ uint32_t quant_code(float x, const QParams& p, int qmax) {
+// Rounding uses the 1.5 * 2^23 trick (adding that constant rounds a float below 2^22 to the nearest integer, ties
+// to even): plain additions instead of the conversion instructions, which issue at a quarter of the rate.
+// One packed word = 32/BITS codes.  The common case costs seven floating-point instructions per element: the codes
+// are rounded with the 1.5 * 2^23 trick and packed by exact multiply-adds with powers of two (two half words of at most
+// 16 bits each, so every partial sum is an exact small integer), and the test "could the estimate have rounded
+// differently from the true quotient" is one running maximum per word instead of a branch per element.  Only a
+// word that fails the test is redone with the IEEE division.
+template <int BITS, bool FILTER>
+__device__ __forceinline__ uint32_t quant_word(const float (&x)[32 / BITS], const QParams& p, float thr) {
+  constexpr int PER = 32 / BITS, HALF = PER / 2, QMAX = (1 << BITS) - 1;
   if (p.sf == 0.f) return 0u;
   constexpr float kMagic = 12582912.f;                 // 1.5 * 2^23
-  const float d = __fsub_rn(x, p.zf);
-  const float q = __fmul_rn(d, p.inv);                 // 0 <= q <= qmax (1 + 2^-22)
-  float m = __fadd_rn(q, kMagic);
-  const float r = __fsub_rn(m, kMagic);                // rint(q)
-  if (fabsf(__fsub_rn(q, r)) > 0.4995f) m = __fadd_rn(rintf(__fdiv_rn(d, p.sf)), kMagic);
-  // 0 <= code <= qmax already: x >= min >= z, and the scale was rounded up so (max - z)/s <= qmax (1 + 2^-23)
-  return min(__float_as_uint(m) & 0x3ffu, (uint32_t)qmax);
-}
-
-__device__ __forceinline__ uint32_t code_or_zero(float x, const QParams& p, int qmax, float thr) {
-  return fabsf(x) > thr ? 0u : quant_code(x, p, qmax);
+  float lo = 0.f, hi = 0.f, worst = 0.f;
+#pragma unroll
+  for (int c = 0; c < PER; ++c) {
+    const float d = __fsub_rn(x[c], p.zf);
+    const float q = __fmul_rn(d, p.inv);               // 0 <= q <= qmax (1 + 2^-22) for an inlier
+    float r = __fsub_rn(__fadd_rn(q, kMagic), kMagic); // rint(q)
+    const bool outlier = FILTER && fabsf(x[c]) > thr;
+    if (outlier) r = 0.f;
+    else worst = fmaxf(worst, fabsf(__fsub_rn(q, r)));
+    const float wgt = (float)(1u << ((c % HALF) * BITS));
+    if (c < HALF) lo = __fmaf_rn(r, wgt, lo);
+    else hi = __fmaf_rn(r, wgt, hi);
+  }
+  if (worst > 0.4995f) {                               // rare: some estimate sits next to a half-integer
+    uint32_t w = 0;
+#pragma unroll
+    for (int c = 0; c < PER; ++c) {
+      const bool outlier = FILTER && fabsf(x[c]) > thr;
+      const float r = fminf(fmaxf(rintf(__fdiv_rn(__fsub_rn(x[c], p.zf), p.sf)), 0.f), (float)QMAX);
+      w |= (outlier ? 0u : (uint32_t)r) << (c * BITS);
+    }
+    return w;
+  }
+  return (uint32_t)lo | ((uint32_t)hi << 16);
 }
 
 // One layer's arguments.  Sources: K, V rows [BH, L, D]; kept [BH, n_idx] positions of the rows to take
@@ -72,9 +91,13 @@ struct QuantTable {
   QuantLayer l[NL];
 };
 
-template <int BITS, int NL>
+// FILTER: outlier filtering compiled in (the threshold test costs two instructions per element otherwise spent for nothing)
+// D is a compile-time constant and the loops over a group run in fully unrolled chunks of 32 elements: with
+// run-time extents the address arithmetic and loop control cost more instructions than the quantization itself
+// (25 instructions per element under ncu against about 13 of arithmetic).
+template <int BITS, int NL, int D, bool FILTER = false>
 __global__ void __launch_bounds__(128)
-gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
+gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int g) {
   extern __shared__ __align__(16) uint16_t sK[];   // [g][D] gathered key rows
   __shared__ int sidx[128];
   constexpr int QMAX = (1 << BITS) - 1, PER = 32 / BITS;
@@ -88,7 +111,7 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   __half* __restrict__ Ks = ql.Ks; __half* __restrict__ Kz = ql.Kz;
   __half* __restrict__ Vs = ql.Vs; __half* __restrict__ Vz = ql.Vz;
   const int L = ql.L, n = ql.n_idx, ns = ql.ns;
-  const float thr = ql.thr;
+  const float thr = FILTER ? ql.thr : INFINITY;
   const bool k_rows = ql.k_axis == 1;              // keys token by token: the value loop below, run on K
   // two blocks per run of g kept tokens: an even block quantizes its key group, the odd one its value rows (each has
   // a shorter chain of dependent memory round trips than one block doing both)
@@ -114,11 +137,14 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
   // keys: channel d, tokens e = 0..g-1
   for (int d = tid; key_part && !k_rows && d < D; d += nthr) {
     float mn = INFINITY, mx = -INFINITY;
-    for (int e = 0; e < g; ++e) {
-      const float x = bf16_bits_to_f32(sK[e * D + d]);
-      if (fabsf(x) > thr) continue;
-      mn = fminf(mn, x);
-      mx = fmaxf(mx, x);
+    for (int e0 = 0; e0 < g; e0 += 32) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float x = bf16_bits_to_f32(sK[(e0 + j) * D + d]);
+        if (FILTER && fabsf(x) > thr) continue;
+        mn = fminf(mn, x);
+        mx = fmaxf(mx, x);
+      }
     }
     if (mn > mx) mn = mx = 0.f;                     // outliers only
     const QParams p = group_params(mn, mx, QMAX);
@@ -127,10 +153,12 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
     for (int wd = 0; wd < wpg; wd += 4) {       // wpg is 2 (B=2,g=32) or a multiple of 4
       uint32_t wv[4] = {0u, 0u, 0u, 0u};
       const int nw = min(4, wpg - wd);
-      for (int i = 0; i < nw; ++i)
+      for (int i = 0; i < nw; ++i) {
+        float x[PER];
 #pragma unroll
-        for (int c = 0; c < PER; ++c)
-          wv[i] |= code_or_zero(bf16_bits_to_f32(sK[((wd + i) * PER + c) * D + d]), p, QMAX, thr) << (c * BITS);
+        for (int c = 0; c < PER; ++c) x[c] = bf16_bits_to_f32(sK[((wd + i) * PER + c) * D + d]);
+        wv[i] = quant_word<BITS, FILTER>(x, p, thr);
+      }
       if (nw == 4) *reinterpret_cast<uint4*>(dst + wd) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
       else *reinterpret_cast<uint2*>(dst + wd) = make_uint2(wv[0], wv[1]);
     }
@@ -148,46 +176,39 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int D, int g) {
     const int e = it / ngv, v = it % ngv;
     const uint16_t* src = Rh + (size_t)sidx[e] * D + (size_t)v * g;
     float mn = INFINITY, mx = -INFINITY;
-    for (int c8 = 0; c8 < g; c8 += 8) {
-      const uint4 q = *reinterpret_cast<const uint4*>(src + c8);
-      const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+    for (int c32 = 0; c32 < g; c32 += 32) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float x0 = bf16lo(ww[i]), x1 = bf16hi(ww[i]);
-        if (!(fabsf(x0) > thr)) { mn = fminf(mn, x0); mx = fmaxf(mx, x0); }
-        if (!(fabsf(x1) > thr)) { mn = fminf(mn, x1); mx = fmaxf(mx, x1); }
+      for (int c8 = 0; c8 < 32; c8 += 8) {
+        const uint4 q = *reinterpret_cast<const uint4*>(src + c32 + c8);
+        const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float x0 = bf16lo(ww[i]), x1 = bf16hi(ww[i]);
+          if (!FILTER || !(fabsf(x0) > thr)) { mn = fminf(mn, x0); mx = fmaxf(mx, x0); }
+          if (!FILTER || !(fabsf(x1) > thr)) { mn = fminf(mn, x1); mx = fmaxf(mx, x1); }
+        }
       }
     }
     if (mn > mx) mn = mx = 0.f;                     // outliers only
     const QParams p = group_params(mn, mx, QMAX);
     const size_t gi = ((size_t)bh * ns + (size_t)ud * g + e) * ngv + v;
     uint32_t* dst = Rc + gi * wpg;
-    // second sweep over the group in 16-byte pieces (8 channels); a piece fills 8/PER words
-    constexpr int WPP = PER >= 8 ? 1 : 8 / PER;                 // words completed per piece (PER 16: half a word)
-    uint32_t word = 0;
-    for (int c8 = 0; c8 < g; c8 += 8) {
-      const uint4 q = *reinterpret_cast<const uint4*>(src + c8);
-      const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
-      uint32_t codes[8];
+    // second sweep over the group, one packed word (32/BITS channels) at a time
+    for (int wd = 0; wd < wpg; ++wd) {
+      float x[PER];
+      const uint16_t* wsrc = src + wd * PER;
+      if constexpr (PER >= 8) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        codes[2 * i] = code_or_zero(bf16lo(ww[i]), p, QMAX, thr);
-        codes[2 * i + 1] = code_or_zero(bf16hi(ww[i]), p, QMAX, thr);
-      }
-      if constexpr (PER == 16) {                                // 2-bit: two pieces per word
-        const int sh = (c8 & 8) ? 16 : 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) word |= codes[i] << (sh + i * BITS);
-        if (c8 & 8) { dst[c8 / 16] = word; word = 0; }
-      } else {
-#pragma unroll
-        for (int wq = 0; wq < WPP; ++wq) {
-          uint32_t wv = 0;
-#pragma unroll
-          for (int i = 0; i < PER; ++i) wv |= codes[wq * PER + i] << (i * BITS);
-          dst[(c8 / 8) * WPP + wq] = wv;
+        for (int h8 = 0; h8 < PER / 8; ++h8) {
+          const uint4 q = *reinterpret_cast<const uint4*>(wsrc + 8 * h8);
+          x[8 * h8 + 0] = bf16lo(q.x); x[8 * h8 + 1] = bf16hi(q.x); x[8 * h8 + 2] = bf16lo(q.y); x[8 * h8 + 3] = bf16hi(q.y);
+          x[8 * h8 + 4] = bf16lo(q.z); x[8 * h8 + 5] = bf16hi(q.z); x[8 * h8 + 6] = bf16lo(q.w); x[8 * h8 + 7] = bf16hi(q.w);
         }
+      } else {                                                  // 8 bit: four channels = 8 bytes
+        const uint2 q = *reinterpret_cast<const uint2*>(wsrc);
+        x[0] = bf16lo(q.x); x[1] = bf16hi(q.x); x[2] = bf16lo(q.y); x[3] = bf16hi(q.y);
       }
+      dst[wd] = quant_word<BITS, FILTER>(x, p, thr);
     }
     Rs[gi] = p.s16;
     Rz[gi] = p.z16;
@@ -280,16 +301,28 @@ gather_rows_kernel(const uint16_t* __restrict__ K, const uint16_t* __restrict__ 
   *reinterpret_cast<uint4*>(Vo + dst) = *reinterpret_cast<const uint4*>(V + src);
 }
 
-template <int NL>
-cudaError_t launch_quant_table(int bits, const QuantTable<NL>& tab, dim3 grid, int D, int g, cudaStream_t st) {
+template <int BITS, int NL, int D>
+cudaError_t launch_quant_bits(const QuantTable<NL>& tab, dim3 grid, int g, cudaStream_t st, bool filter) {
   const size_t smem = (size_t)g * D * sizeof(uint16_t);
+  if constexpr (NL == 1) {
+    if (filter) {
+      gather_quant_kernel<BITS, NL, D, true><<<grid, 128, smem, st>>>(tab, g);
+      return cudaGetLastError();
+    }
+  }
+  gather_quant_kernel<BITS, NL, D, false><<<grid, 128, smem, st>>>(tab, g);
+  return cudaGetLastError();
+}
+template <int NL>
+cudaError_t launch_quant_table(int bits, const QuantTable<NL>& tab, dim3 grid, int D, int g, cudaStream_t st,
+                               bool filter = false) {
+  if (D != 64 && D != 128) return cudaErrorInvalidValue;
   switch (bits) {
-    case 2: gather_quant_kernel<2, NL><<<grid, 128, smem, st>>>(tab, D, g); break;
-    case 4: gather_quant_kernel<4, NL><<<grid, 128, smem, st>>>(tab, D, g); break;
-    case 8: gather_quant_kernel<8, NL><<<grid, 128, smem, st>>>(tab, D, g); break;
+    case 2: return D == 128 ? launch_quant_bits<2, NL, 128>(tab, grid, g, st, filter) : launch_quant_bits<2, NL, 64>(tab, grid, g, st, filter);
+    case 4: return D == 128 ? launch_quant_bits<4, NL, 128>(tab, grid, g, st, filter) : launch_quant_bits<4, NL, 64>(tab, grid, g, st, filter);
+    case 8: return D == 128 ? launch_quant_bits<8, NL, 128>(tab, grid, g, st, filter) : launch_quant_bits<8, NL, 64>(tab, grid, g, st, filter);
     default: return cudaErrorInvalidValue;
   }
-  return cudaGetLastError();
 }
 
 // rows of the new token into the tails (or, at 16 bit, into the caches): 16 bytes per thread
@@ -348,7 +381,7 @@ cudaError_t launch_gather_quantize_ex(const void* K, const void* V, const int32_
                         static_cast<__half*>(c.k_scale), static_cast<__half*>(c.k_zero),
                         static_cast<__half*>(c.v_scale), static_cast<__half*>(c.v_zero), L, n, ns, 0,
                         s.k_axis, filter ? s.outlier_threshold : INFINITY};
-  cudaError_t e = launch_quant_table<1>(c.bits, tab, dim3(2 * (n / g), BH, 1), D, g, st);
+  cudaError_t e = launch_quant_table<1>(c.bits, tab, dim3(2 * (n / g), BH, 1), D, g, st, filter);
   if (e != cudaSuccess || !filter) return e;
   const int n_tiles = (n + 31) / 32;
   auto side = [&](const qp_side& q) {
