@@ -226,9 +226,12 @@ def build_caches(qp, wl, seed, dev, ws_c, bits_list=None, keep_inputs=False):
         qw = synth.make_q_win(wls, l, device=dev)
         for b in bits_list:
             wb = synth.dataclasses.replace(wls, bits=b)
+            n = wb.n_keep(l)                        # buffers are allocated outside the timed call (an allocation can synchronise)
+            c = qp.alloc_cache(wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, b, wl.group, n, dev)
+            kept = torch.empty((wl.batch, wl.n_kv_heads, n), dtype=torch.int32, device=dev)
             a, z = ev(), ev()
             a.record(stream)
-            c, _ = qp.compress_layer(k, v, qw, wb.layer_budget_bits(l), b, wl.group, wl.pool, workspace=ws_c)
+            qp.compress_layer(k, v, qw, wb.layer_budget_bits(l), b, wl.group, wl.pool, c, kept, ws_c)
             z.record(stream)
             torch.cuda.synchronize()
             comp_ms[b] += a.elapsed_time(z)
@@ -349,7 +352,10 @@ def strategy_figures(qp, dev, peak, stream, rank):
     ms = timed(lambda r: qp.decode_attn_layers_ex(qs, flex[r % n_seq], st_flex, outs, ws), 512)
     layer_bytes = Bt * Hkv * n * D * 2 * (4 + 1) // 8
     ms_f = timed(lambda r: qp.decode_attn_ex(qs[0], filt[r % len(filt)][0], filt[r % len(filt)][1], outs[0], ws), 64)
-    ms_h = timed(lambda r: qp.decode_attn_heads(qs[0], heads[r % len(heads)], outs[0]), 64)
+    G = Hq // Hkv
+    hq = [qs[0].view(Bt * Hkv, 1, G, D)[i] for i in range(Bt * Hkv)]          # per-head views, built once
+    ho = [outs[0].view(Bt * Hkv, 1, G, D)[i] for i in range(Bt * Hkv)]
+    ms_h = timed(lambda r: qp.decode_attn_layers_ex(hq, heads[r % len(heads)].caches, heads[r % len(heads)].strategy, ho, ws), 64)
     head_tokens = sum(sum(h.n_heads) for h in heads) / len(heads)
     return {
         "workload": wl.name + ", 4 bit",

@@ -119,6 +119,14 @@ def test_llama70b_pyramid_first_and_last_layer():
     assert swaps <= 4
 
 
+def test_llama70b_pyramid_with_the_papers_window_of_8():
+    """The same 70B-shape pyramid layers with the observation window the paper uses for PyramidKV (the last 8
+    tokens, Appendix B "KV eviction methods") instead of 32, at full size."""
+    wl = dataclasses.replace(synth.LLAMA70B_32K_B4, w=8)
+    swaps = run_fullsize(wl, layers=[0, 79], samples=[(1, 3), (2, 7)], decode_steps=1)
+    assert swaps <= 4
+
+
 def test_llama8b_generation_loop_in_the_bench_configuration():
     """Append + decode over packed tokens and tail at the benchmark's launch shape: 128 layer descriptors
     (32 layers of 4 sequences) per qp_append_kv_layers / qp_decode_attn_tail_layers call, tails cycling
