@@ -607,16 +607,16 @@ int decode_mma_workers_per_sm(const DecDims& d) {
          : d.bits == 16 ? decode_mma16_blocks_per_sm() : decode_mma2_workers_per_sm();
 }
 // Launches that do not fill every worker slot with a long range use fewer workers, not emptier ones: a worker's
-// ramp and its partial record (which the merge step has to read) are costs per worker.  Measured for the 4-bit
-// kernel on caches of 64 tiles per head: per-layer calls (512 tiles) from a CUDA graph take 9.8 / 6.4 / 4.0 / 3.6 /
-// 3.3 / 3.8 us with at least 1 / 2 / 4 / 8 / 16 / 32 tiles per worker, 84 MB calls (16384 tiles) 20.4 us with the
-// 1776 workers of a full grid, 19.5 us with 16 tiles per worker and 17.5 us with 32 (512 workers, two per head,
-// ranges aligned with the heads), 26.6 us with 64.  So: 32 tiles where that still leaves 256 workers, else 16.
-// The 8-bit kernel behaves alike (151 MB calls of 16384 tiles: 4.22 / 4.02 / 5.08 / 2.76 TB/s with 4 / 16 / 32 / 64);
-// the 2-bit and 16-bit kernels showed no gain (4.96 / 4.78 / 4.87 / 4.65 and 5.60 / 5.61 / 5.60 / 4.81 TB/s) and keep
-// four tiles per worker.
+// ramp and its partial record (which the merge step has to read) are costs per worker.  On a stream whose calls
+// overlap, two calls share the GPU most of the time, so a call wants about half of the resident worker slots:
+// measured for the 4- and 8-bit kernels with at least 12 / 16 / 20 / 24 / 32 tiles per worker (us per call, calls
+// overlapping): 84 MB 4-bit 28.2 / 20.2 / 22.1 / 23.5 / 22.3, 168 MB 4-bit 35.9 / 35.8 / 40.8 / 38.1 / 34.2, 151 MB 8-bit
+// 34.9 / 33.0 / 35.1 / 38.7 / 36.6, 75 MB 8-bit 23.1 / 22.3 / 25.0 / 26.4 / 24.0, 42 MB 4-bit 16.9 / 16.3 / 16.6 / 17.4 / 18.6.
+// A call that runs alone (plain stream order) takes as many workers as it can give four tiles each: per-layer calls
+// replayed from a CUDA graph 10.2 / 8.4 / 8.4 / 10.2 us with at least 1 / 2 / 4 / 8 tiles per worker.  The 2-bit and
+// 16-bit kernels showed no gain from fewer workers and always use four tiles.
 #ifndef QP_TMIN_BIG
-#define QP_TMIN_BIG 32
+#define QP_TMIN_BIG 16
 #endif
 #ifndef QP_TMIN_SMALL
 #define QP_TMIN_SMALL 16
