@@ -152,3 +152,40 @@ def test_bad_arguments_are_rejected_before_any_launch(lib):
     assert lib.qp_gather_quantize(A, A, None, 1024, ref, None) == 1
     assert lib.qp_select_topk(A, 1, 2, 1024, 32, 32, A, None) == 3
     assert lib.qp_window_scores(A, A, 1, 8, 2, 64, 1024, 32, 7, A, A, 16, None) == 4
+
+
+def test_strategy_head_budget_and_overlap_arguments_are_checked_before_any_launch(lib):
+    A = 0x10000
+    assert ctypes.sizeof(qp.qp_side) == 2 * 4 + 4 * 8
+    assert ctypes.sizeof(qp.qp_strategy) == 2 * 4 + 2 * ctypes.sizeof(qp.qp_side)
+    c16 = qp.cache_layout(1, 4, 1, 128, 16, 32, 64)
+    c16.k_codes = c16.v_codes = A
+    s = qp.qp_strategy()
+    assert lib.qp_decode_attn_ex(A, ctypes.byref(c16), ctypes.byref(s), A, A, 1 << 20, None) == 2   # nothing to quantize
+    c = qp.cache_layout(1, 4, 1, 128, 4, 32, 64)
+    c.k_codes = c.v_codes = c.k_scale = c.k_zero = c.v_scale = c.v_zero = A
+    cr = ctypes.byref(c)
+    assert lib.qp_decode_attn_ex(A, cr, None, A, A, 1 << 20, None) == 1
+    s.k_axis = 2
+    assert lib.qp_decode_attn_ex(A, cr, ctypes.byref(s), A, A, 1 << 20, None) == 1
+    s.k_axis, s.outlier_threshold = 1, 6.0                        # filtering on, side lists missing
+    assert lib.qp_gather_quantize_ex(A, A, A, 100, cr, ctypes.byref(s), None) == 1
+    s.outlier_threshold = 0.0
+    assert lib.qp_decode_attn_ex(A, cr, ctypes.byref(s), A, A, 16, None) == 4
+    assert lib.qp_decode_attn_ex(A + 2, cr, ctypes.byref(s), A, A, 1 << 20, None) == 5
+
+    hb = lib.qp_head_budgets
+    need = lib.qp_head_budgets_workspace_bytes(2, 8, 4096, 32, 512)
+    assert need >= 2 * (8 * (512 - 32) + 1) * 4 and need % 256 == 0
+    assert lib.qp_head_budgets_workspace_bytes(2, 8, 4096, 32, 32) == 0
+    assert hb(None, 2, 8, 4096, 32, 512, 32, A, A, need, None) == 1
+    assert hb(A, 2, 8, 4096, 4096, 512, 32, A, A, need, None) == 1          # no prefix
+    assert hb(A, 2, 8, 4096, 32, 512, 0, A, A, need, None) == 1
+    assert hb(A, 2, 8, 4096, 32, 32, 32, A, A, need, None) == 3             # mean budget inside the window
+    assert hb(A, 2, 8, 4096, 32, 512, 32, A, A + 4, need, None) == 5
+    assert hb(A, 2, 8, 4096, 32, 512, 32, A, A, need - 1, None) == 4
+    assert hb(A, 1, 8200, 4096, 32, 512, 32, A, A, 1 << 40, None) == 2
+
+    words = (ctypes.c_uint32 * 4)(9, 9, 9, 9)
+    assert lib.qp_debug_check(None) == 1
+    assert lib.qp_debug_check(words) == 2 and list(words) == [0, 0, 0, 0]     # the release build carries no checks
