@@ -3,7 +3,7 @@
 // For one (batch, KV head) the R = G*w window-query rows form a [R x D] matrix and the keys a [L x D]
 // matrix; the logits are their product (a dense contraction: qp_score_tc.cu runs it on tcgen05).  The row
 // softmax needs every visible key of a row before any column can be normalised, hence two sweeps over K:
-//   sweep 1  per (key tile, row) running (max, sum of exp)        -> stat partials
+//   sweep 1  per (run of key tiles, row) running (max, sum of exp) -> stat partials
 //   merge    per row: global max M and 1/Z
 //   sweep 2  recompute the tile's logits, p = exp2(t - M)/Z, sum the tile's columns over the
 //            rows of the block                                     -> vote partials
@@ -23,7 +23,7 @@ constexpr int SC_RB = 128;       // window-query rows per thread block (8 warps 
 __host__ __device__ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // per row: M = max over tiles, Z = sum_i s_i * 2^(m_i - M); stores (M, 1/Z); rows beyond R get 1/Z = 0.
-// One block per (batch, KV head, row block, group of RM_ROWS rows): thread (row, slice) folds tiles slice,
+// One block per (batch, KV head, row block, group of RM_ROWS rows): thread (row, slice) folds partials slice,
 // slice + RM_SLICES, ... into a running (max, sum) pair with coalesced reads across rows; the slices are then
 // combined in a fixed order.
 constexpr int RM_SLICES = 32, RM_ROWS = 32, RM_PARTS = SC_RB / RM_ROWS;
@@ -93,8 +93,8 @@ ScoreWorkspace score_workspace(int Bt, int Hq, int Hkv, int L, int w) {
   s.n_tiles = (L + SC_TILE - 1) / SC_TILE;
   s.n_vote_tiles = (P + SC_TILE - 1) / SC_TILE;
   size_t off = 0;
-  // (max, sum) per row and key tile; the tensor-memory sweep keeps one per 64-column half tile
-  s.stat_partial = off;  off += align256((size_t)BH * s.n_rb * s.n_tiles * 2 * SC_RB * sizeof(float2));
+  // (max, sum) per row and sweep-1 block: at most one block per two key tiles
+  s.stat_partial = off;  off += align256((size_t)BH * s.n_rb * ((s.n_tiles + 1) / 2) * SC_RB * sizeof(float2));
   s.rowstat = off;       off += align256((size_t)BH * s.n_rb * SC_RB * sizeof(float2));
   s.votes_partial = off; off += align256((size_t)BH * s.n_rb * P * sizeof(float));
   s.pooled = off;        off += align256((size_t)BH * P * sizeof(float));
@@ -119,9 +119,9 @@ cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, c
   if (e != cudaSuccess) return e;
   // The two sweeps of a (batch, KV head) read the same keys, so the keys cross the HBM interface twice.  Taking the
   // heads in groups whose keys fit in the L2 cache (sweep 1 -> merge -> sweep 2 per group) lets the second sweep find
-  // them there, but the sweeps are bound by their exponentials, not by HBM, and the smaller launches lose more at
-  // their ends than the cache hits save: measured per layer with groups of 0 (off) / 48 / 100 MB: 0.54 / 0.77 / 0.67 ms
-  // at 32k x batch 8, 0.33 / 0.55 / 0.40 ms at 128k, 0.41 / 0.52 / 0.44 ms for the 70B shapes.  Off by default.
+  // them there, but the smaller launches fill the SMs worse and lose more at their ends than the cache hits save:
+  // measured for the whole score stage with groups of 0 (off) / 64 / 100 MB: 250 / 396 / 361 us at 32k x batch 8,
+  // 128 / 210 / 188 us at 128k, 222 / 259 / 244 us for the 70B shapes.  Off by default.
 #ifndef QP_SCORE_GROUP_MB
 #define QP_SCORE_GROUP_MB 0
 #endif
@@ -130,11 +130,14 @@ cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, c
   if ((long long)per_group * s.n_tiles * s.n_rb < 2 * 296) per_group = BH;     // small problems: one group
   for (int bh0 = 0; bh0 < BH; bh0 += per_group) {
     const int cnt = std::min(per_group, BH - bh0);
-    e = launch_score_sweep_tc(1, n_layers, Qwin, K, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st, bh0, cnt);
+    int n_splits = 0;
+    e = launch_score_sweep_tc(1, n_layers, Qwin, K, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st, bh0, cnt,
+                              &n_splits);
     if (e != cudaSuccess) return e;
     rowstat_merge_kernel<<<cnt * s.n_rb * RM_PARTS, RM_ROWS * RM_SLICES, 0, st>>>(stat_partial, bh0 * s.n_rb, s.n_rb,
-                                                                                 2 * s.n_tiles, R, rowstat);
-    e = launch_score_sweep_tc(2, n_layers, Qwin, K, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st, bh0, cnt);
+                                                                                 n_splits, R, rowstat);
+    e = launch_score_sweep_tc(2, n_layers, Qwin, K, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st, bh0, cnt,
+                              nullptr);
     if (e != cudaSuccess) return e;
   }
   pool_kernel<<<dim3((P + 255) / 256, BH), 256, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);

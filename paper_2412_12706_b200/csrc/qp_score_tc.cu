@@ -1,27 +1,41 @@
-// S1 on the 5th-generation tensor cores: the window-score sweeps with tcgen05.mma and TMEM.
+// S1 on the 5th-generation tensor cores: the window-score sweeps with TMA, tcgen05.mma and TMEM.
 //
 // One thread block owns 128 window-query rows (M) of one (batch, KV head) and walks over a run of
-// 128-key tiles (N).  Per tile a single thread issues D/16 tcgen05.mma (bf16 x bf16 -> f32, both
-// operands K-major in shared memory with the 128-byte swizzle), the [128 x 128] logit tile lands in
-// tensor memory, and the four warps read it back with tcgen05.ld: TMEM lane = query row, so every
-// thread owns one row (two warpgroups split the columns) and the softmax statistics of sweep 1 need
-// no shuffles at all.  Sweep 2 swaps the operands (TMEM lane = key, column = query row), so the vote
-// of a key is again a thread-local sum.
-// Two TMEM buffers and two shared-memory stages let the MMA of tile i+1 and the copy of tile i+2
-// run under the epilogue of tile i.
+// 128-key tiles (N).  The block is specialised by warp and its parts talk through mbarriers only:
+//   warp 8     one lane asks the TMA unit for the next key tile ([128 keys x D] bf16 into one of two
+//              shared-memory stages, 128-byte swizzle) as soon as the MMAs that read the stage have retired;
+//   warp 9     one lane issues the D/16 tcgen05.mma of a tile (bf16 x bf16 -> f32, both operands K-major
+//              in shared memory) into one of two [128 x 128] tensor-memory buffers once the tile has landed
+//              and the buffer's previous reader is done;
+//   warps 0-7  two groups of four warps read the buffers back with tcgen05.ld: group 0 takes the even
+//              tiles (buffer 0), group 1 the odd ones, so a thread owns one TMEM lane of a whole tile: a
+//              query row in sweep 1 (running max and sum, no shuffles), a key in sweep 2 (the operands are
+//              swapped, so the vote of a key is again a thread-local sum).  The next chunk of 32 columns
+//              is in flight while a chunk is folded, and the buffer is handed back before the last chunk's
+//              arithmetic.
+// With two blocks per SM four such groups keep the exponential unit busy while the others wait.
 //
-// Every wait on an mbarrier is bounded: if it runs out, the block records an error word, frees its
-// tensor memory and returns.  Outputs and their layout are the ones of score_sweep_kernel.
+// Every wait on an mbarrier is bounded: if it runs out, the block records an error word, waits (bounded)
+// for the copies it still has in flight, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include <algorithm>
+#include <cstring>
+
 #include "qp_mma.cuh"
 
 namespace qp {
 
 namespace {
 
-constexpr int TC_THREADS = 256;                     // two warpgroups: each reads half of the tile's columns
 constexpr int TC_M = 128, TC_N = 128;
+constexpr int TC_EPI_WARPS = 8;                       // two groups of four: one TMEM buffer each
+constexpr int TC_THREADS = (TC_EPI_WARPS + 2) * 32;   // + the copy warp and the MMA warp
 constexpr uint32_t TC_TMEM_COLS = 256;                // two accumulator buffers of 128 columns
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 22;
+
+// mbarriers of one block
+enum : int { BAR_K_FULL = 0, BAR_K_EMPTY = 2, BAR_T_FULL = 4, BAR_T_EMPTY = 6, BAR_COUNT = 8 };
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
@@ -37,11 +51,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// bounded wait; false = gave up
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < TC_SPIN_LIMIT; ++i)
+// bounded wait; false = gave up (or another part of the block already has)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* give_up) {
+  for (uint32_t i = 0; i < TC_SPIN_LIMIT; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *give_up) return false;
+  }
   return false;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+// one box of a 2-D tensor map into shared memory; completion is counted in bytes on `bar`
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
 }
 
 // shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 B apart
@@ -69,8 +98,8 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 32 columns of this warp's 32 TMEM lanes; the registers hold nothing until tmem_wait has returned them
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -79,10 +108,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+      : "r"(taddr)
+      : "memory");
+}
+// waits for every tcgen05.ld of this thread; the registers pass through it, so no use of them can be scheduled earlier
+__device__ __forceinline__ void tmem_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 // 2^x by the hardware approximation (about 2 ulp; results below 2^-126 flush to 0)
 __device__ __forceinline__ float ex2a(float x) {
@@ -96,32 +133,77 @@ __device__ __forceinline__ void cp_async16_zfill(uint32_t saddr, const void* gpt
 }
 
 // byte offset of 16-byte chunk c (8 bf16) of row r inside a [128 rows x D] operand: D/64 blocks of
-// [128 rows x 128 B], each made of 8-row groups of 1024 B with the chunk index XORed by the row
+// [128 rows x 128 B], each made of 8-row groups of 1024 B with the chunk index XORed by the row (the
+// layout the TMA unit writes for a [128 x 64] box with the 128-byte swizzle at a 1024-byte aligned address)
 __device__ __forceinline__ uint32_t sw128_off(int r, int c) {
   return (uint32_t)((c >> 3) * (TC_M * 128) + (r >> 3) * 1024 + (r & 7) * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
+// per-layer inputs of a sweep: the keys as a tensor map over [batch * KV heads * L, D], the window queries as a pointer
+template <int NL>
+struct ScoreMaps {
+  CUtensorMap k[NL];
+  const bf16* q[NL];
+};
+
+// sweep 1: folds 32 logits of a row into its running (max, sum)
+__device__ __forceinline__ void fold_row(const uint32_t (&r)[32], bool all_visible, int col0, int lim, float scale_log2,
+                                         float& m, float& s) {
+  if (all_visible) {
+    float cm = __uint_as_float(r[0]);
+#pragma unroll
+    for (int i = 1; i < 32; ++i) cm = fmaxf(cm, __uint_as_float(r[i]));
+    const float mn = fmaxf(m, cm * scale_log2);               // scale > 0: max commutes with it
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc += ex2a(fmaf(__uint_as_float(r[i]), scale_log2, -mn));
+    s = fmaf(s, ex2a(m - mn), acc);
+    m = mn;
+  } else {
+    float v[32], cm = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      v[i] = col0 + i <= lim ? __uint_as_float(r[i]) * scale_log2 : -INFINITY;
+      cm = fmaxf(cm, v[i]);
+    }
+    if (cm != -INFINITY) {
+      const float mn = fmaxf(m, cm);
+      float acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) acc += ex2a(v[i] - mn);
+      s = fmaf(s, ex2a(m - mn), acc);
+      m = mn;
+    }
+  }
+}
+// sweep 2: adds the probabilities of 32 query rows (columns c0 .. c0+31 of the swapped tile) to a key's vote
+__device__ __forceinline__ void fold_vote(const uint32_t (&r)[32], const float2* sRow, int c0, float scale_log2, float& vote) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    const float4 ms = *reinterpret_cast<const float4*>(&sRow[c0 + i]);   // (M, 1/Z) x 2 rows
+    vote = fmaf(ex2a(fmaf(__uint_as_float(r[i]), scale_log2, -ms.x)), ms.y, vote);
+    vote = fmaf(ex2a(fmaf(__uint_as_float(r[i + 1]), scale_log2, -ms.z)), ms.w, vote);
+  }
+}
+
 template <int PASS, int D, int NL>
 __global__ void __launch_bounds__(TC_THREADS, 2)
-score_sweep_tc_kernel(const __grid_constant__ ScorePtrs<NL> ptrs, int bh0, int BH, int Hq, int Hkv, int L, int w,
-                      int n_rb, int n_tiles, int tiles_per_block, float scale_log2,
+score_sweep_tc_kernel(const __grid_constant__ ScoreMaps<NL> maps, int bh0, int BH, int Hq, int Hkv, int L, int w,
+                      int n_rb, int n_tiles, int tiles_per_block, int n_splits, float scale_log2,
                       float2* __restrict__ stat_partial, const float2* __restrict__ rowstat,
                       float* __restrict__ votes_partial, int* __restrict__ error_word) {
   constexpr int CPR = D / 8;                           // 16-byte chunks per row
   constexpr uint32_t OPER_BYTES = TC_M * D * 2;        // one operand tile: D/64 swizzled blocks of 16 KB
   extern __shared__ unsigned char smem_raw[];
-  __shared__ uint64_t bars[2];
+  __shared__ uint64_t bars[BAR_COUNT];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int give_up;
-  __shared__ float sVote[PASS == 2 ? 2 : 1][TC_N];
-  __shared__ __align__(16) float2 sRow[PASS == 2 ? TC_M : 1];      // sweep 2: (M, 1/Z) of the block's rows
+  __shared__ __align__(16) float2 sRow[TC_M];          // sweep 2: (M, 1/Z) of the block's rows; sweep 1: group 1's result
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int rloc = tid & (TC_M - 1), half = tid >> 7, wq = warp & 3;   // row in the block, column half, TMEM lane quarter
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
   // bh counts (layer, batch, KV head): the scratch arrays are laid out over all of them, the inputs are per layer
   const int split = blockIdx.x, rb = blockIdx.y, bh = bh0 + blockIdx.z, layer = bh / BH, bhl = bh % BH;
-  const bf16* __restrict__ Qwin = ptrs.q[layer];
-  const bf16* __restrict__ K = ptrs.k[layer];
   const int b = bhl / Hkv, hk = bhl % Hkv, G = Hq / Hkv, P = L - w, R = G * w;
   const int tile_lo = split * tiles_per_block;
   const int n_vis = PASS == 1 ? n_tiles : (P + TC_N - 1) / TC_N;    // sweep 2 only needs prefix columns
@@ -132,157 +214,160 @@ score_sweep_tc_kernel(const __grid_constant__ ScorePtrs<NL> ptrs, int bh0, int B
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;     // operands need 1024-byte alignment
   const uint32_t sQ = sbase, sK0 = sbase + OPER_BYTES;              // then two K stages
   const uint32_t bar0 = smem_u32(&bars[0]);
+  auto bar = [&](int which, int i) { return bar0 + (uint32_t)(which + i) * 8u; };
+  const volatile int* gu = &give_up;
 
   if (tid == 0) {
-    mbar_init(bar0, 1);
-    mbar_init(bar0 + 8, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_K_FULL, i), 1);                // the copy lane's expect_tx; the bytes complete it
+      mbar_init(bar(BAR_K_EMPTY, i), 1);               // a tcgen05.commit
+      mbar_init(bar(BAR_T_FULL, i), 1);                // a tcgen05.commit
+      mbar_init(bar(BAR_T_EMPTY, i), 4 * 32);          // every thread of the reading group
+    }
     give_up = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  if (warp == 0) {
+  if (warp == TC_EPI_WARPS + 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&tmem_base_slot)),
                  "r"(TC_TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
 
-  // stage a [128 x D] bf16 operand (rows beyond `rows_valid` are zero)
-  auto stage_rows = [&](uint32_t dst, const bf16* src, int rows_valid) {
-#pragma unroll
-    for (int i = 0; i < TC_M * CPR / TC_THREADS; ++i) {
-      const int idx = tid + TC_THREADS * i, r = idx / CPR, c = idx % CPR;
+  // the block's [128 x D] window-query rows (rows beyond R are zero), by every thread
+  {
+    const bf16* Qh = maps.q[layer] + ((size_t)(b * Hq + hk * G) * w + (size_t)rb * TC_M) * D;
+    const int rows_valid = min(TC_M, R - rb * TC_M);
+    for (int idx = tid; idx < TC_M * CPR; idx += TC_THREADS) {
+      const int r = idx / CPR, c = idx % CPR;
       const bool ok = r < rows_valid;
-      cp_async16_zfill(dst + sw128_off(r, c), src + (ok ? (size_t)r * D + c * 8 : 0), ok);
-    }
-  };
-  const bf16* Qh = Qwin + ((size_t)(b * Hq + hk * G) * w + (size_t)rb * TC_M) * D;
-  const bf16* Kh = K + (size_t)bhl * L * D;
-  stage_rows(sQ, Qh, min(TC_M, R - rb * TC_M));
-  stage_rows(sK0, Kh + (size_t)tile_lo * TC_N * D, min(TC_N, L - tile_lo * TC_N));
-  cp_async_commit();
-  if (n_loc > 1) stage_rows(sK0 + OPER_BYTES, Kh + (size_t)(tile_lo + 1) * TC_N * D, min(TC_N, L - (tile_lo + 1) * TC_N));
-  cp_async_commit();
-
-  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-  const uint32_t tmem_base = tmem_base_slot;
-  constexpr uint32_t IDESC = instr_desc(TC_M, TC_N);
-
-  // issue the D/16 MMAs of local tile j (shared-memory stage j & 1 -> TMEM buffer j & 1)
-  auto issue_mma = [&](int j) {
-    const uint32_t sK = sK0 + (j & 1) * OPER_BYTES, tm = tmem_base + (j & 1) * TC_N;
-#pragma unroll
-    for (int kb = 0; kb < D / 64; ++kb)
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (PASS == 1)      // rows = queries, columns = keys
-          umma_bf16(tm, smem_desc(sQ + kb * (TC_M * 128) + k * 32), smem_desc(sK + kb * (TC_N * 128) + k * 32), IDESC,
-                    (kb | k) ? 1u : 0u);
-        else                // rows = keys, columns = queries
-          umma_bf16(tm, smem_desc(sK + kb * (TC_N * 128) + k * 32), smem_desc(sQ + kb * (TC_M * 128) + k * 32), IDESC,
-                    (kb | k) ? 1u : 0u);
-    umma_commit(bar0 + (j & 1) * 8);
-  };
-
-  // this thread's query row and its statistics
-  const int row = rb * TC_M + rloc;
-  const int lim = min(P + (row % w), L - 1);            // last key this row may see
-  if (PASS == 2 && tid < TC_M) sRow[tid] = rowstat[(size_t)(bh * n_rb + rb) * TC_M + tid];   // visible after the next barrier
-
-  cp_async_wait<1>();                                   // Q and the first K tile have landed
-  asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-  __syncthreads();
-  if (tid == 0) issue_mma(0);
-
-  for (int j = 0; j < n_loc; ++j) {
-    if (j + 1 < n_loc) {                                // next tile's operands -> MMA under this tile's epilogue
-      cp_async_wait<0>();
-      asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-      __syncthreads();
-      if (tid == 0) issue_mma(j + 1);
-    }
-    const bool ok = mbar_wait(bar0 + (j & 1) * 8, (j >> 1) & 1);
-    if (!ok) give_up = 1;
-    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-    __syncthreads();                                    // everyone sees the outcome; stage j & 1 is free again
-    if (give_up) break;
-    if (j + 2 < n_loc) {
-      const int tl = tile_lo + j + 2;
-      stage_rows(sK0 + (j & 1) * OPER_BYTES, Kh + (size_t)tl * TC_N * D, min(TC_N, L - tl * TC_N));
+      cp_async16_zfill(sQ + sw128_off(r, c), Qh + (ok ? (size_t)r * D + c * 8 : 0), ok);
     }
     cp_async_commit();
+  }
+  if (PASS == 2 && tid < TC_M) sRow[tid] = rowstat[(size_t)(bh * n_rb + rb) * TC_M + tid];
+  cp_async_wait<0>();
+  asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();                                     // barriers, TMEM base, Q and sRow are visible
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
 
-    const int tile = tile_lo + j, key0 = tile * TC_N;
-    const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + (j & 1) * TC_N + half * (TC_N / 2);
-    const int col0 = key0 + half * (TC_N / 2);
-    if constexpr (PASS == 1) {
-      // TMEM lane = query row: this thread folds its row's 64 columns into a running (max, sum)
-      float m = -INFINITY, s = 0.f;
-      const bool all_visible = key0 + TC_N - 1 <= P;            // every row sees every key up to P
-#pragma unroll 1
-      for (int c0 = 0; c0 < TC_N / 2; c0 += 32) {
-        float v[32];
-        tmem_ld32(taddr + c0, v);
-        if (all_visible) {
-          float cm = v[0];
+  float m_run = -INFINITY, s_run = 0.f;                // sweep 1: this thread's row over the group's tiles
+
+  if (warp == TC_EPI_WARPS) {
+    // ---- copy warp: tile j -> stage j & 1 once the MMAs of tile j - 2 have retired
+    const CUtensorMap* map = &maps.k[layer];
+    int issued = 0;
+    bool ok = true;
+    for (int j = 0; j < n_loc && ok; ++j) {
+      const int st = j & 1;
+      if (j >= 2) ok = mbar_wait(bar(BAR_K_EMPTY, st), (uint32_t)(((j >> 1) - 1) & 1), gu);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_expect_tx(bar(BAR_K_FULL, st), OPER_BYTES);
+        const int y = bhl * L + (tile_lo + j) * TC_N;
 #pragma unroll
-          for (int i = 1; i < 32; ++i) cm = fmaxf(cm, v[i]);
-          const float mn = fmaxf(m, cm * scale_log2);           // scale > 0: max commutes with it
-          float acc = 0.f;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) acc += ex2a(fmaf(v[i], scale_log2, -mn));
-          s = fmaf(s, ex2a(m - mn), acc);
-          m = mn;
-        } else {
-          float cm = -INFINITY;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            v[i] = col0 + c0 + i <= lim ? v[i] * scale_log2 : -INFINITY;
-            cm = fmaxf(cm, v[i]);
-          }
-          if (cm != -INFINITY) {
-            const float mn = fmaxf(m, cm);
-            float acc = 0.f;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc += ex2a(v[i] - mn);
-            s = fmaf(s, ex2a(m - mn), acc);
-            m = mn;
-          }
-        }
+        for (int kb = 0; kb < D / 64; ++kb)
+          tma_load_2d(sK0 + st * OPER_BYTES + kb * (TC_N * 128), map, kb * 64, y, bar(BAR_K_FULL, st));
       }
-      // one (max, sum) per row and 64-column half tile
-      stat_partial[(((size_t)(bh * n_rb + rb) * n_tiles + tile) * 2 + half) * TC_M + rloc] = make_float2(m, s);
-    } else {
-      // operands swapped: TMEM lane = key, column = query row, so a key's vote is a thread-local sum over
-      // the rows.  Only prefix keys (< P) are written and every row sees all of them: no mask needed;
-      // rows beyond R carry 1/Z = 0.
-      float vote = 0.f;
-#pragma unroll 1
-      for (int c0 = 0; c0 < TC_N / 2; c0 += 32) {
-        float v[32];
-        tmem_ld32(taddr + c0, v);
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float4 ms = *reinterpret_cast<const float4*>(&sRow[half * (TC_N / 2) + c0 + i]);   // (M, 1/Z) x 2 rows
-          vote = fmaf(ex2a(fmaf(v[i], scale_log2, -ms.x)), ms.y, vote);
-          vote = fmaf(ex2a(fmaf(v[i + 1], scale_log2, -ms.z)), ms.w, vote);
-        }
-      }
-      sVote[half][rloc] = vote;
-      __syncthreads();
-      if (tid < TC_N && key0 + tid < P)
-        votes_partial[(size_t)(bh * n_rb + rb) * P + key0 + tid] = sVote[0][tid] + sVote[1][tid];
+      issued = j + 1;
+      __syncwarp();
     }
-    asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-    __syncthreads();                                    // TMEM buffer j & 1 and sVote may be overwritten
+    if (!ok) {
+      give_up = 1;
+      // the copies still on their way land in this block's shared memory: wait for them before it is given up
+      for (int j = max(0, issued - 2); j < issued; ++j) {
+        bool landed = false;
+        for (uint32_t i = 0; i < TC_SPIN_LIMIT && !landed; ++i) landed = mbar_try_wait(bar(BAR_K_FULL, j & 1), (uint32_t)((j >> 1) & 1));
+      }
+    }
+  } else if (warp == TC_EPI_WARPS + 1) {
+    // ---- MMA warp: tile j from stage j & 1 into TMEM buffer j & 1
+    constexpr uint32_t IDESC = instr_desc(TC_M, TC_N);
+    bool ok = true;
+    for (int j = 0; j < n_loc && ok; ++j) {
+      const int st = j & 1;
+      ok = mbar_wait(bar(BAR_K_FULL, st), (uint32_t)((j >> 1) & 1), gu);
+      if (ok && j >= 2) ok = mbar_wait(bar(BAR_T_EMPTY, st), (uint32_t)(((j >> 1) - 1) & 1), gu);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      if (lane == 0) {
+        const uint32_t sK = sK0 + st * OPER_BYTES, tm = tmem_base + st * TC_N;
+#pragma unroll
+        for (int kb = 0; kb < D / 64; ++kb)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (PASS == 1)      // rows = queries, columns = keys
+              umma_bf16(tm, smem_desc(sQ + kb * (TC_M * 128) + k * 32), smem_desc(sK + kb * (TC_N * 128) + k * 32), IDESC,
+                        (kb | k) ? 1u : 0u);
+            else                // rows = keys, columns = queries
+              umma_bf16(tm, smem_desc(sK + kb * (TC_N * 128) + k * 32), smem_desc(sQ + kb * (TC_M * 128) + k * 32), IDESC,
+                        (kb | k) ? 1u : 0u);
+        umma_commit(bar(BAR_K_EMPTY, st));              // the stage may be refilled ...
+        umma_commit(bar(BAR_T_FULL, st));               // ... and the tile read, once these MMAs have retired
+      }
+      __syncwarp();
+    }
+    if (!ok) give_up = 1;
+  } else {
+    // ---- reading groups: group gq takes the tiles j = gq, gq + 2, ... from TMEM buffer gq
+    const int gq = warp >> 2, wq = warp & 3, rloc = wq * 32 + lane;
+    const int row = rb * TC_M + rloc;
+    const int lim = min(P + (row % w), L - 1);          // sweep 1: last key this row may see
+    const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + gq * TC_N;
+    bool ok = true;
+    for (int j = gq; j < n_loc; j += 2) {
+      ok = mbar_wait(bar(BAR_T_FULL, gq), (uint32_t)((j >> 1) & 1), gu);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      const int key0 = (tile_lo + j) * TC_N;
+      uint32_t va[32], vb[32];
+      float vote = 0.f;
+      const bool all_visible = key0 + TC_N - 1 <= P;    // every row sees every key up to P
+      auto fold = [&](const uint32_t (&r)[32], int c0) {
+        if constexpr (PASS == 1) fold_row(r, all_visible, key0 + c0, lim, scale_log2, m_run, s_run);
+        else fold_vote(r, sRow, c0, scale_log2, vote);
+      };
+      tmem_ld32_issue(taddr, va);
+      tmem_wait(va);
+      tmem_ld32_issue(taddr + 32, vb);
+      fold(va, 0);
+      tmem_wait(vb);
+      tmem_ld32_issue(taddr + 64, va);
+      fold(vb, 32);
+      tmem_wait(va);
+      tmem_ld32_issue(taddr + 96, vb);
+      fold(va, 64);
+      tmem_wait(vb);
+      asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+      mbar_arrive(bar(BAR_T_EMPTY, gq));                // the buffer is free for tile j + 2
+      fold(vb, 96);
+      if constexpr (PASS == 2) {
+        // only prefix keys (< P) are written and every row sees all of them: no mask needed; rows beyond R
+        // carry 1/Z = 0
+        if (key0 + rloc < P) votes_partial[(size_t)(bh * n_rb + rb) * P + key0 + rloc] = vote;
+      }
+    }
+    if (!ok) give_up = 1;
+    if (PASS == 1 && gq == 1) sRow[rloc] = make_float2(m_run, s_run);
   }
 
-  cp_async_wait<0>();
-  if (give_up && tid == 0) atomicExch(error_word, 1);
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
-  __syncthreads();
-  if (warp == 0) {
+  __syncthreads();                                      // every part is done with shared and tensor memory
+  if (PASS == 1 && warp < 4) {
+    // one (max, sum) per row and block: the even tiles' pair, then the odd tiles'
+    const int rloc = warp * 32 + lane;
+    const float2 o = sRow[rloc];
+    const float mn = fmaxf(m_run, o.x);
+    float s = 0.f;
+    if (m_run != -INFINITY) s = s_run * ex2a(m_run - mn);
+    if (o.x != -INFINITY) s = fmaf(o.y, ex2a(o.x - mn), s);
+    stat_partial[((size_t)(bh * n_rb + rb) * n_splits + split) * TC_M + rloc] = make_float2(mn, s);
+  }
+  if (give_up && tid == 0) atomicExch(error_word, 1);
+  if (warp == TC_EPI_WARPS + 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
   }
 }
@@ -292,57 +377,103 @@ score_sweep_tc_kernel(const __grid_constant__ ScorePtrs<NL> ptrs, int bh0, int B
 bool score_tc_supported(int D) { return D == 128 || D == 64; }
 
 namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+// the driver's tensor-map encoder, looked up through the runtime (the library does not link against the driver)
+EncodeTiledFn encode_tiled() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+// keys of one layer as a [rows x D] bf16 matrix, fetched in boxes of [128 rows x 64 columns] with the 128-byte swizzle;
+// boxes that reach past the last row are filled with zeros
+cudaError_t key_map(CUtensorMap* map, const void* k, long long rows, int D) {
+  EncodeTiledFn enc = encode_tiled();
+  if (!enc) return cudaErrorNotSupported;
+  const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)TC_N};
+  const cuuint32_t elem[2] = {1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(k), dims, strides, box, elem,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int PASS, int D, int NL>
-cudaError_t launch_tc(dim3 grid, int bh0, cudaStream_t st, const ScorePtrs<NL>& ptrs, const ScoreDims& d, const ScoreWorkspace& s,
-                      int per, float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
-                      int* error_word) {
+cudaError_t launch_tc(dim3 grid, int bh0, int BH, cudaStream_t st, const ScoreMaps<NL>& maps, const ScoreDims& d,
+                      const ScoreWorkspace& s, int per, float scale_log2, float2* stat_partial, const float2* rowstat,
+                      float* votes_partial, int* error_word) {
   constexpr size_t smem = 3 * (size_t)TC_M * D * 2 + 1024;   // Q + two K stages + alignment slack
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(score_sweep_tc_kernel<PASS, D, NL>, smem, done);
   if (e != cudaSuccess) return e;
-  score_sweep_tc_kernel<PASS, D, NL><<<grid, TC_THREADS, smem, st>>>(ptrs, bh0, d.Bt * d.Hkv, d.Hq, d.Hkv, d.L, d.w, s.n_rb,
-                                                                    s.n_tiles, per, scale_log2, stat_partial, rowstat,
+  score_sweep_tc_kernel<PASS, D, NL><<<grid, TC_THREADS, smem, st>>>(maps, bh0, BH, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles,
+                                                                    per, (int)grid.x, scale_log2, stat_partial, rowstat,
                                                                     votes_partial, error_word);
   return cudaGetLastError();
 }
 
 template <int NL>
-cudaError_t launch_sweep(int pass, const ScorePtrs<NL>& ptrs, int bh0, int BH, const ScoreDims& d, const ScoreWorkspace& s,
-                         float scale_log2, float2* stat_partial, const float2* rowstat, float* votes_partial,
-                         int* error_word, cudaStream_t st) {
+cudaError_t launch_sweep(int pass, int n_layers, const void* const* q, const void* const* k, int bh0, int bh_count,
+                         const ScoreDims& d, const ScoreWorkspace& s, float scale_log2, float2* stat_partial,
+                         const float2* rowstat, float* votes_partial, int* error_word, cudaStream_t st, int* n_splits) {
+  const int BH = d.Bt * d.Hkv;                          // (batch, KV head) pairs of one layer
+  if ((long long)BH * d.L > 0x7fffffffLL - TC_N) return cudaErrorInvalidValue;   // row coordinates are 32-bit
+  ScoreMaps<NL> maps;
+  memset(&maps, 0, sizeof(maps));
+  for (int l = 0; l < n_layers; ++l) {
+    maps.q[l] = static_cast<const bf16*>(q[l]);
+    const cudaError_t e = key_map(&maps.k[l], k[l], (long long)BH * d.L, d.D);
+    if (e != cudaSuccess) return e;
+  }
   const int tiles = pass == 1 ? s.n_tiles : s.n_vote_tiles;
-  // enough blocks for two per SM over a few waves, at least two tiles per block
-  long long per = ((long long)tiles * s.n_rb * BH + 591) / 592;
-  if (per < 2) per = 2;
-  if (per > 32) per = 32;
+  // Blocks along the keys.  All blocks of a launch take the same time per tile and two fit on an SM, so the launch
+  // lasts about ceil(blocks / 2 SMs) rounds of (tiles per block + a fixed cost of about three tiles for the block's
+  // set-up and first copy): take the split with the shortest such schedule, at least two tiles per block.
+  const int slots = 2 * sm_count();
+  long long per = 2;
+  double best = 1e300;
+  for (int cand = 1; cand <= std::max(1, tiles / 2); ++cand) {
+    const long long p = std::max<long long>(2, (tiles + cand - 1) / cand);
+    const long long blocks = ((tiles + p - 1) / p) * s.n_rb * bh_count;
+    const double cost = (double)((blocks + slots - 1) / slots) * (double)(p + 3);
+    if (cost < best) { best = cost; per = p; }
+  }
   const int splits = (int)((tiles + per - 1) / per);
-  const dim3 grid(splits, s.n_rb, BH);
+  if (n_splits) *n_splits = splits;
+  const dim3 grid(splits, s.n_rb, bh_count);
   if (d.D == 128)
-    return pass == 1 ? launch_tc<1, 128, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
-                     : launch_tc<2, 128, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
-  return pass == 1 ? launch_tc<1, 64, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
-                   : launch_tc<2, 64, NL>(grid, bh0, st, ptrs, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
+    return pass == 1 ? launch_tc<1, 128, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
+                     : launch_tc<2, 128, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
+  return pass == 1 ? launch_tc<1, 64, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
+                   : launch_tc<2, 64, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
 }
 }  // namespace
 
 // s: the scratch layout for batch * n_layers batch entries (the layers are stacked along the batch dimension)
-// bh0, bh_count: the (layer, batch, KV head) triples this launch covers
+// bh0, bh_count: the (layer, batch, KV head) triples this launch covers; *n_splits: blocks along the keys, i.e. the
+// (max, sum) pairs sweep 1 leaves per row in stat_partial [triple, row block, split, 128 rows]
 cudaError_t launch_score_sweep_tc(int pass, int n_layers, const void* const* q, const void* const* k, const ScoreDims& d,
                                   const ScoreWorkspace& s, float scale_log2, float2* stat_partial, const float2* rowstat,
-                                  float* votes_partial, int* error_word, cudaStream_t st, int bh0, int bh_count) {
-  if (n_layers == 1) {
-    ScorePtrs<1> p;
-    p.q[0] = static_cast<const bf16*>(q[0]);
-    p.k[0] = static_cast<const bf16*>(k[0]);
-    return launch_sweep<1>(pass, p, bh0, bh_count, d, s, scale_log2, stat_partial, rowstat, votes_partial, error_word, st);
-  }
-  ScorePtrs<QP_MAX_LAYERS> p;
-  for (int l = 0; l < n_layers; ++l) {
-    p.q[l] = static_cast<const bf16*>(q[l]);
-    p.k[l] = static_cast<const bf16*>(k[l]);
-  }
-  return launch_sweep<QP_MAX_LAYERS>(pass, p, bh0, bh_count, d, s, scale_log2, stat_partial, rowstat, votes_partial,
-                                     error_word, st);
+                                  float* votes_partial, int* error_word, cudaStream_t st, int bh0, int bh_count,
+                                  int* n_splits) {
+#define QP_SWEEP(NL) \
+  return launch_sweep<NL>(pass, n_layers, q, k, bh0, bh_count, d, s, scale_log2, stat_partial, rowstat, votes_partial, \
+                          error_word, st, n_splits)
+  if (n_layers == 1) QP_SWEEP(1);
+  if (n_layers <= 8) QP_SWEEP(8);
+  if (n_layers <= 32) QP_SWEEP(32);
+  QP_SWEEP(QP_MAX_LAYERS);
+#undef QP_SWEEP
 }
 
 }  // namespace qp
