@@ -15,6 +15,7 @@ namespace {
 
 constexpr int TK_THREADS = 1024;
 constexpr int TK_UNROLL = 8;
+constexpr int TKR_BINS = 4096;     // histogram bins of the register kernel's 12-bit digits
 
 // Outputs of the layers of one launch: block (layer, bh) reads scores[(layer * BH + bh) * P ..] and writes
 // kept[layer][bh * n_keep[layer] ..].
@@ -148,8 +149,8 @@ topk_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid
 }
 
 // The same selection for P <= ITEMS * 1024 with the keys held in registers: the scores are read from memory once
-// (all loads in flight together) instead of five times, the four digit passes and the compaction run from
-// registers, and the ordered compaction needs one block-wide prefix over (chunk, warp) counts instead of one
+// (all loads in flight together) instead of five times, the digit passes (three here, over wider digits) and the
+// compaction run from registers, and the ordered compaction needs one block-wide prefix over (chunk, warp) counts instead of one
 // per chunk.  Element j = q * 1024 + tid is item q of thread tid, so ascending position = (q, warp, lane) order.
 template <int ITEMS, int NL>
 __global__ void __launch_bounds__(TK_THREADS)
@@ -166,7 +167,8 @@ topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __
     return;
   }
 
-  __shared__ unsigned hist[256];
+  __shared__ unsigned hist[TKR_BINS];
+  __shared__ unsigned warp_tot[32];
   __shared__ unsigned sh_prefix, sh_need;
   __shared__ unsigned cnt_g[ITEMS][32], cnt_e[ITEMS][32];        // per (chunk, warp): counts, then exclusive prefixes
   __shared__ unsigned row_g[ITEMS], row_e[ITEMS];                // per chunk: totals, then exclusive prefixes
@@ -178,50 +180,63 @@ topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __
     key[q] = order_key(j < P ? s[j] : 0.f);
   }
 
+  // Three digit passes of 12, 12 and 8 bits over a 4096-bin histogram.  The leading 12 bits (sign, exponent, three
+  // mantissa bits) of real scores take dozens of values, so the lanes of a warp mostly hit different bins and plain
+  // shared-memory atomics do; only a warp whose 32 candidates all carry one digit (constant scores) adds once.
   unsigned prefix = 0, mask = 0, need = (unsigned)k;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 20 : pass == 1 ? 8 : 0;
+    const unsigned dmask = pass == 2 ? 255u : (unsigned)(TKR_BINS - 1);
+#pragma unroll
+    for (int i = 0; i < TKR_BINS / TK_THREADS; ++i) hist[tid + i * TK_THREADS] = 0;
     __syncthreads();
 #pragma unroll
     for (int q = 0; q < ITEMS; ++q) {
       if (q * TK_THREADS >= P) break;
       const bool cand = q * TK_THREADS + tid < P && (key[q] & mask) == prefix;
-      const unsigned digit = (key[q] >> shift) & 255u;
-      if (shift >= 16) {                                         // crowded digits: one atomic per distinct digit and warp
-        const unsigned peers = __match_any_sync(0xffffffffu, cand ? digit : 256u + lane);
-        if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+      const unsigned digit = (key[q] >> shift) & dmask;
+      if (pass == 0) {
+        const unsigned d0 = __shfl_sync(0xffffffffu, digit, 0);
+        if (__all_sync(0xffffffffu, cand && digit == d0)) {
+          if (lane == 0) atomicAdd(&hist[d0], 32u);
+        } else if (cand) {
+          atomicAdd(&hist[digit], 1u);
+        }
       } else if (cand) {
         atomicAdd(&hist[digit], 1u);
       }
     }
     __syncthreads();
-    if (warp == 0) {
-      // lane l owns bins 8l .. 8l+7; find the bin where the count from the top reaches `need`
-      unsigned c[8], tot = 0;
+    // thread t owns bins 4t .. 4t+3; find the bin where the count from the top reaches `need`
+    unsigned c[TKR_BINS / TK_THREADS], tot = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { c[i] = hist[8 * lane + i]; tot += c[i]; }
-      unsigned suf = tot;
+    for (int i = 0; i < TKR_BINS / TK_THREADS; ++i) { c[i] = hist[(TKR_BINS / TK_THREADS) * tid + i]; tot += c[i]; }
+    unsigned suf = tot;                                          // this thread and the higher lanes of its warp
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned v = __shfl_down_sync(0xffffffffu, suf, o);
-        if (lane + o < 32) suf += v;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned v = __shfl_down_sync(0xffffffffu, suf, o);
+      if (lane + o < 32) suf += v;
+    }
+    if (lane == 0) warp_tot[warp] = suf;
+    __syncthreads();
+    unsigned higher = 0;                                         // the warps above this one
+    for (int wv = warp + 1; wv < 32; ++wv) higher += warp_tot[wv];
+    const unsigned incl = suf + higher, above = incl - tot;
+    if (above < need && incl >= need) {                          // exactly one thread
+      unsigned cum = above;
+      int bsel = TKR_BINS / TK_THREADS - 1;
+      for (; bsel > 0; --bsel) {
+        if (cum + c[bsel] >= need) break;
+        cum += c[bsel];
       }
-      const unsigned above = suf - tot;
-      if (above < need && suf >= need) {                         // exactly one lane
-        unsigned cum = above;
-        int bsel = 7;
-        for (; bsel > 0; --bsel) {
-          if (cum + c[bsel] >= need) break;
-          cum += c[bsel];
-        }
-        sh_need = need - cum;
-        sh_prefix = prefix | ((unsigned)(8 * lane + bsel) << shift);
-      }
+      sh_need = need - cum;
+      sh_prefix = prefix | ((unsigned)((TKR_BINS / TK_THREADS) * tid + bsel) << shift);
     }
     __syncthreads();
     prefix = sh_prefix;
     need = sh_need;
-    mask |= 0xffu << shift;
+    mask |= dmask << shift;
   }
   const uint32_t T = prefix;   // image of the k-th largest score; `need` elements equal to it are kept
 
@@ -427,11 +442,10 @@ namespace {
 template <int NL>
 cudaError_t launch_topk(const float* scores, int blocks, int BH, int L, int w, const TopkOut<NL>& o, cudaStream_t st) {
   const int P = L - w;
-  // a cluster per head also pays for shorter prefixes (above 2048 positions) when the heads alone would leave most
-  // SMs idle: eight CTAs with one or two keys per thread beat one CTA with eight
+  // a cluster per head also pays for prefixes of 8k to 32k positions when the heads alone would leave most SMs
+  // idle (measured at 32k positions: 19.5 us against 24.8 us for 8 heads)
   const bool few_heads = blocks * TKC_CTAS <= sm_count();
-  if (P <= 8 * TK_THREADS && !(few_heads && P > 2 * TK_THREADS))
-    topk_reg_kernel<8, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
+  if (P <= 8 * TK_THREADS) topk_reg_kernel<8, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
   else if (P <= 32 * TK_THREADS && !few_heads) topk_reg_kernel<32, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
   else if (P <= TKC_CTAS * TKC_ITEMS * TK_THREADS)
     topk_cluster_kernel<NL><<<blocks * TKC_CTAS, TK_THREADS, 0, st>>>(scores, L, w, BH, o);

@@ -68,6 +68,31 @@ def test_select_topk_bit_exact_with_ties(P, w, n):
     assert np.array_equal(got.cpu().numpy(), ref)
 
 
+@pytest.mark.parametrize("P,w,n", [(5000, 32, 32 + 1000), (8192, 16, 16 + 4096), (20000, 32, 32 + 2048),
+                                   (32736, 32, 8192), (12345, 8, 8 + 12000), (9000, 32, 32 + 1)])
+def test_select_topk_one_block_per_head_with_many_heads(P, w, n):
+    """With more heads than an eighth of the SMs every head is selected by one block from registers (12-bit digits):
+    ties, constant rows, sorted rows, rows whose scores share their leading bits, denormals and zeros."""
+    L = P + w
+    rng = np.random.default_rng(P * 7 + n)
+    Bt, Hkv = 4, 6
+    s = rng.random((Bt, Hkv, P)).astype(np.float32)
+    s[0, 0] = np.round(s[0, 0] * 16) / 16
+    s[0, 1] = 0.5
+    s[1, 0, ::3] = 0.0
+    s[1, 1] = np.sort(s[1, 1])
+    s[1, 2] = np.sort(s[1, 2])[::-1]
+    s[2, 0] = 1.0 + rng.random(P).astype(np.float32) * 1e-4        # one leading digit, spread only in the low bits
+    s[2, 1] = (rng.random(P) * 1e-40).astype(np.float32)           # denormals
+    s[2, 2] = np.exp(rng.standard_normal(P) * 6).astype(np.float32)  # many binades
+    s[3, 0, : P // 2] = s[3, 0, P // 2: 2 * (P // 2)]              # every value twice
+    s[3, 1] = np.float32(1e-3) * (rng.integers(0, 3, P)).astype(np.float32)   # three values only
+    ref = orc.select(s.astype(np.float64), L, w, n)
+    got = qp.select_topk(torch.from_numpy(s).to(DEV), L, w, n)
+    torch.cuda.synchronize()
+    assert np.array_equal(got.cpu().numpy(), ref)
+
+
 # ------------------------------------------------------------------ S1: window scores
 
 @pytest.mark.parametrize("Hq,Hkv,D,L,w,pool", [(8, 2, 64, 1024, 32, 7), (4, 4, 128, 333, 8, 7),
