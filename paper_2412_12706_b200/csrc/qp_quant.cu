@@ -32,46 +32,36 @@ __device__ __forceinline__ QParams group_params(float mn, float mx, int qmax) {
   return p;
 }
 
-// code = clamp(rint((x - z) / s)) with the true quotient.  The quotient is first estimated as
-// (x - z) * (1/s), which is within 2^-22 relative (< 1e-4 absolute for codes up to 255) of it, so the
-// rounded integer can only differ when the estimate lies that close to a half-integer; only then is
-// the IEEE division done.  The result is the same integer in every case.
-// Rounding uses the 1.5 * 2^23 trick (adding that constant rounds a float below 2^22 to the nearest integer, ties
-// to even): plain additions instead of the conversion instructions, which issue at a quarter of the rate.
-// One packed word = 32/BITS codes.  The common case costs seven floating-point instructions per element: the codes
-// are rounded with the 1.5 * 2^23 trick and packed by exact multiply-adds with powers of two (two half words of at most
-// 16 bits each, so every partial sum is an exact small integer), and the test "could the estimate have rounded
-// differently from the true quotient" is one running maximum per word instead of a branch per element.  Only a
-// word that fails the test is redone with the IEEE division.
+// code = rint((x - z) / s) with the correctly rounded quotient Q = RN(d / s), d = RN(x - z) >= 0, without a division
+// per element: with y = RN(1/s) (once per group), q = RN(d * y) is within an ulp of the quotient, the remainder
+// d - q * s comes exactly rounded out of one FMA, and q' = RN(q + rem * y) is the correctly rounded quotient (the
+// classical FMA division step; s is an fp16 value, so its significand is never all ones, the one excluded case).
+// Exact ties (q' = k + 1/2) are frequent with bf16 inputs and fp16 scales, and they round to even exactly as in the
+// division.  Rounding adds 1.5 * 2^23 (a float below 2^22 becomes that constant plus its nearest integer, ties to
+// even, in the low mantissa bits), and the codes are packed with integer shift-adds of those bit patterns, the
+// constant's contribution taken off once per word.  Six instructions per element, no branch.
+// (An earlier form estimated d * y, tested a margin around the half-integers and redid a word with the IEEE division
+// when a lane failed the test: with exact ties in about one group in eight that redo ran for a tenth of the warps'
+// words and doubled the instruction count, 13 per element under ncu.)
 template <int BITS, bool FILTER>
 __device__ __forceinline__ uint32_t quant_word(const float (&x)[32 / BITS], const QParams& p, float thr) {
-  constexpr int PER = 32 / BITS, HALF = PER / 2, QMAX = (1 << BITS) - 1;
-  if (p.sf == 0.f) return 0u;
+  constexpr int PER = 32 / BITS;
+  if (p.inv == 0.f) return 0u;                         // scale 0 (a constant group) or infinite: every code is 0
   constexpr float kMagic = 12582912.f;                 // 1.5 * 2^23
-  float lo = 0.f, hi = 0.f, worst = 0.f;
+  constexpr uint32_t kMagicBits = 0x4B400000u;
+  uint32_t acc = 0, bias = 0;
 #pragma unroll
   for (int c = 0; c < PER; ++c) {
     const float d = __fsub_rn(x[c], p.zf);
-    const float q = __fmul_rn(d, p.inv);               // 0 <= q <= qmax (1 + 2^-22) for an inlier
-    float r = __fsub_rn(__fadd_rn(q, kMagic), kMagic); // rint(q)
-    const bool outlier = FILTER && fabsf(x[c]) > thr;
-    if (outlier) r = 0.f;
-    else worst = fmaxf(worst, fabsf(__fsub_rn(q, r)));
-    const float wgt = (float)(1u << ((c % HALF) * BITS));
-    if (c < HALF) lo = __fmaf_rn(r, wgt, lo);
-    else hi = __fmaf_rn(r, wgt, hi);
+    const float q = __fmul_rn(d, p.inv);
+    const float rem = __fmaf_rn(-q, p.sf, d);
+    const float q1 = __fmaf_rn(rem, p.inv, q);         // RN(d / s): 0 <= q1 <= qmax for an inlier
+    uint32_t bits = __float_as_uint(__fadd_rn(q1, kMagic));
+    if (FILTER && fabsf(x[c]) > thr) bits = kMagicBits;   // an outlier's code is 0
+    acc += bits << (c * BITS);
+    bias += kMagicBits << (c * BITS);                  // folded at compile time
   }
-  if (worst > 0.4995f) {                               // rare: some estimate sits next to a half-integer
-    uint32_t w = 0;
-#pragma unroll
-    for (int c = 0; c < PER; ++c) {
-      const bool outlier = FILTER && fabsf(x[c]) > thr;
-      const float r = fminf(fmaxf(rintf(__fdiv_rn(__fsub_rn(x[c], p.zf), p.sf)), 0.f), (float)QMAX);
-      w |= (outlier ? 0u : (uint32_t)r) << (c * BITS);
-    }
-    return w;
-  }
-  return (uint32_t)lo | ((uint32_t)hi << 16);
+  return acc - bias;
 }
 
 // One layer's arguments.  Sources: K, V rows [BH, L, D]; kept [BH, n_idx] positions of the rows to take
@@ -95,9 +85,12 @@ struct QuantTable {
 // D is a compile-time constant and the loops over a group run in fully unrolled chunks of 32 elements: with
 // run-time extents the address arithmetic and loop control cost more instructions than the quantization itself
 // (25 instructions per element under ncu against about 13 of arithmetic).
-template <int BITS, int NL, int D, bool FILTER = false>
+// GROUP = 32 (the usual group) is compiled with the group's 32 elements held in registers between the min/max sweep
+// and the packing, and with vector stores of a group's words; GROUP = 0 takes the group size at run time.
+template <int BITS, int NL, int D, int GROUP, bool FILTER = false>
 __global__ void __launch_bounds__(128)
-gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int g) {
+gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int g_rt) {
+  const int g = GROUP > 0 ? GROUP : g_rt;
   extern __shared__ __align__(16) uint16_t sK[];   // [g][D] gathered key rows
   __shared__ int sidx[128];
   constexpr int QMAX = (1 << BITS) - 1, PER = 32 / BITS;
@@ -134,8 +127,46 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int g) {
   }
   __syncthreads();
 
+  // one group of 32 elements held in registers: range, parameters, BITS packed words
+  auto quant_group32 = [&](const float (&x)[32], uint32_t* dst, __half* s_out, __half* z_out) {
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      if (FILTER && fabsf(x[j]) > thr) continue;
+      mn = fminf(mn, x[j]);
+      mx = fmaxf(mx, x[j]);
+    }
+    if (mn > mx) mn = mx = 0.f;                     // outliers only
+    const QParams p = group_params(mn, mx, QMAX);
+    uint32_t wv[BITS];                              // 32 * BITS / 32 words
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) {
+      float xs[PER];
+#pragma unroll
+      for (int c = 0; c < PER; ++c) xs[c] = x[i * PER + c];
+      wv[i] = quant_word<BITS, FILTER>(xs, p, thr);
+    }
+    if constexpr (BITS == 2) {
+      *reinterpret_cast<uint2*>(dst) = make_uint2(wv[0], wv[1]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < BITS; i += 4) *reinterpret_cast<uint4*>(dst + i) = make_uint4(wv[i], wv[i + 1], wv[i + 2], wv[i + 3]);
+    }
+    *s_out = p.s16;
+    *z_out = p.z16;
+  };
+
   // keys: channel d, tokens e = 0..g-1
-  for (int d = tid; key_part && !k_rows && d < D; d += nthr) {
+  if constexpr (GROUP == 32) {
+    for (int d = tid; key_part && !k_rows && d < D; d += nthr) {
+      float x[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) x[j] = bf16_bits_to_f32(sK[j * D + d]);
+      const size_t gi = ((size_t)bh * (ns / 32) + ud) * D + d;
+      quant_group32(x, Kc + gi * BITS, Ks + gi, Kz + gi);
+    }
+  }
+  for (int d = tid; GROUP != 32 && key_part && !k_rows && d < D; d += nthr) {
     float mn = INFINITY, mx = -INFINITY;
     for (int e0 = 0; e0 < g; e0 += 32) {
 #pragma unroll
@@ -172,7 +203,22 @@ gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int g) {
   uint32_t* __restrict__ Rc = key_part ? Kc : Vc;
   __half* __restrict__ Rs = key_part ? Ks : Vs;
   __half* __restrict__ Rz = key_part ? Kz : Vz;
-  for (int it = tid; (!key_part || k_rows) && it < g * ngv; it += nthr) {
+  if constexpr (GROUP == 32) {
+    for (int it = tid; (!key_part || k_rows) && it < 32 * (D / 32); it += nthr) {
+      const int e = it / (D / 32), v = it % (D / 32);
+      const uint4* src = reinterpret_cast<const uint4*>(Rh + (size_t)sidx[e] * D + (size_t)v * 32);
+      float x[32];
+#pragma unroll
+      for (int c8 = 0; c8 < 4; ++c8) {
+        const uint4 q = src[c8];
+        x[8 * c8 + 0] = bf16lo(q.x); x[8 * c8 + 1] = bf16hi(q.x); x[8 * c8 + 2] = bf16lo(q.y); x[8 * c8 + 3] = bf16hi(q.y);
+        x[8 * c8 + 4] = bf16lo(q.z); x[8 * c8 + 5] = bf16hi(q.z); x[8 * c8 + 6] = bf16lo(q.w); x[8 * c8 + 7] = bf16hi(q.w);
+      }
+      const size_t gi = ((size_t)bh * ns + (size_t)ud * 32 + e) * (D / 32) + v;
+      quant_group32(x, Rc + gi * BITS, Rs + gi, Rz + gi);
+    }
+  }
+  for (int it = tid; GROUP != 32 && (!key_part || k_rows) && it < g * ngv; it += nthr) {
     const int e = it / ngv, v = it % ngv;
     const uint16_t* src = Rh + (size_t)sidx[e] * D + (size_t)v * g;
     float mn = INFINITY, mx = -INFINITY;
@@ -306,11 +352,13 @@ cudaError_t launch_quant_bits(const QuantTable<NL>& tab, dim3 grid, int g, cudaS
   const size_t smem = (size_t)g * D * sizeof(uint16_t);
   if constexpr (NL == 1) {
     if (filter) {
-      gather_quant_kernel<BITS, NL, D, true><<<grid, 128, smem, st>>>(tab, g);
+      if (g == 32) gather_quant_kernel<BITS, NL, D, 32, true><<<grid, 128, smem, st>>>(tab, g);
+      else gather_quant_kernel<BITS, NL, D, 0, true><<<grid, 128, smem, st>>>(tab, g);
       return cudaGetLastError();
     }
   }
-  gather_quant_kernel<BITS, NL, D, false><<<grid, 128, smem, st>>>(tab, g);
+  if (g == 32) gather_quant_kernel<BITS, NL, D, 32, false><<<grid, 128, smem, st>>>(tab, g);
+  else gather_quant_kernel<BITS, NL, D, 0, false><<<grid, 128, smem, st>>>(tab, g);
   return cudaGetLastError();
 }
 template <int NL>
