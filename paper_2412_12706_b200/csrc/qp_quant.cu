@@ -26,7 +26,12 @@ __device__ __forceinline__ QParams group_params(float mn, float mx, int qmax) {
   p.z16 = __float2half_rd(mn);                      // zero: largest fp16 <= min
   p.zf = __half2float(p.z16);
   const float range = __fsub_rn(mx, p.zf);
-  p.s16 = __float2half_ru(__fdiv_rn(range, (float)qmax));   // scale: rounded up, so max never clips
+  // RN(range / qmax) by the FMA division step with the constant's reciprocal (see quant_word); exact wherever the
+  // quotient is a normal fp32 number, and below that every positive quotient rounds up to the same smallest fp16
+  const float qm = (float)qmax, y = 1.0f / qm;
+  const float q0 = __fmul_rn(range, y);
+  const float quot = __fmaf_rn(__fmaf_rn(-q0, qm, range), y, q0);
+  p.s16 = __float2half_ru(quot);                    // scale: rounded up, so max never clips
   p.sf = __half2float(p.s16);
   p.inv = p.sf != 0.f ? __frcp_rn(p.sf) : 0.f;
   return p;
