@@ -59,29 +59,30 @@ rowstat_merge_kernel(const float2* __restrict__ stat_partial, int blk0, int n_rb
 }
 
 // scores[j] = (sum over |t| <= r of vote[j + t], zero outside [0, P)) / pool with vote = the sum of the row blocks'
-// partial votes.  A block stages the votes of its 256 outputs and their halo in shared memory.
-constexpr int PK_THREADS = 256, PK_MAX_HALO = 32;
+// partial votes.  A block stages the votes of its PK_OUT outputs and their halo in shared memory (zeros outside the
+// prefix, so the window sum needs no bounds test) and every thread then forms PK_OUT / PK_THREADS outputs.
+constexpr int PK_THREADS = 256, PK_PER = 4, PK_OUT = PK_THREADS * PK_PER, PK_MAX_HALO = 32;
 __global__ void __launch_bounds__(PK_THREADS)
 pool_kernel(const float* __restrict__ votes_partial, int n_rb, int P, int pool, float* __restrict__ scores) {
-  __shared__ float sv[PK_THREADS + 2 * PK_MAX_HALO];
-  const int bh = blockIdx.y, j0 = blockIdx.x * PK_THREADS, r = (pool - 1) / 2;
-  for (int i = threadIdx.x; i < PK_THREADS + 2 * r; i += PK_THREADS) {
+  __shared__ float sv[PK_OUT + 2 * PK_MAX_HALO];
+  const int bh = blockIdx.y, j0 = blockIdx.x * PK_OUT, r = (pool - 1) / 2;
+  const float* vp = votes_partial + (size_t)bh * n_rb * P;
+  for (int i = threadIdx.x; i < PK_OUT + 2 * r; i += PK_THREADS) {
     const int jj = j0 - r + i;
     float v = 0.f;
     if (jj >= 0 && jj < P)
-      for (int rb = 0; rb < n_rb; ++rb) v += votes_partial[(size_t)(bh * n_rb + rb) * P + jj];
+      for (int rb = 0; rb < n_rb; ++rb) v += vp[(size_t)rb * P + jj];
     sv[i] = v;
   }
   __syncthreads();
-  const int j = j0 + threadIdx.x;
-  if (j >= P) return;
-  float acc = 0.f;
-  for (int dlt = 0; dlt <= 2 * r; ++dlt) {
-    const int jj = j - r + dlt;
-    if (jj < 0 || jj >= P) continue;
-    acc += sv[threadIdx.x + dlt];
+#pragma unroll
+  for (int k = 0; k < PK_PER; ++k) {
+    const int t = threadIdx.x + k * PK_THREADS, j = j0 + t;
+    if (j >= P) break;
+    float acc = 0.f;
+    for (int dlt = 0; dlt <= 2 * r; ++dlt) acc += sv[t + dlt];
+    scores[(size_t)bh * P + j] = __fdiv_rn(acc, (float)pool);
   }
-  scores[(size_t)bh * P + j] = __fdiv_rn(acc, (float)pool);
 }
 
 }  // namespace
@@ -140,7 +141,7 @@ cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, c
                               nullptr);
     if (e != cudaSuccess) return e;
   }
-  pool_kernel<<<dim3((P + 255) / 256, BH), 256, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);
+  pool_kernel<<<dim3((P + PK_OUT - 1) / PK_OUT, BH), PK_THREADS, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);
   return cudaGetLastError();
 }
 

@@ -428,12 +428,31 @@ cudaError_t launch_sweep(int pass, int n_layers, const void* const* q, const voi
                          const float2* rowstat, float* votes_partial, int* error_word, cudaStream_t st, int* n_splits) {
   const int BH = d.Bt * d.Hkv;                          // (batch, KV head) pairs of one layer
   if ((long long)BH * d.L > 0x7fffffffLL - TC_N) return cudaErrorInvalidValue;   // row coordinates are 32-bit
+  // the two sweeps of a call (and repeated calls on the same buffers) ask for the same maps: keep the last set
+  struct Last {
+    int n = 0, D = 0;
+    long long rows = 0;
+    const void* k[QP_MAX_LAYERS];
+    CUtensorMap map[QP_MAX_LAYERS];
+  };
+  static thread_local Last last;
+  const long long rows = (long long)BH * d.L;
+  bool same = last.n == n_layers && last.D == d.D && last.rows == rows;
+  for (int l = 0; same && l < n_layers; ++l) same = last.k[l] == k[l];
+  if (!same) {
+    last.n = 0;
+    for (int l = 0; l < n_layers; ++l) {
+      const cudaError_t e = key_map(&last.map[l], k[l], rows, d.D);
+      if (e != cudaSuccess) return e;
+      last.k[l] = k[l];
+    }
+    last.n = n_layers; last.D = d.D; last.rows = rows;
+  }
   ScoreMaps<NL> maps;
   memset(&maps, 0, sizeof(maps));
   for (int l = 0; l < n_layers; ++l) {
     maps.q[l] = static_cast<const bf16*>(q[l]);
-    const cudaError_t e = key_map(&maps.k[l], k[l], (long long)BH * d.L, d.D);
-    if (e != cudaSuccess) return e;
+    maps.k[l] = last.map[l];
   }
   const int tiles = pass == 1 ? s.n_tiles : s.n_vote_tiles;
   // Blocks along the keys.  All blocks of a launch take the same time per tile and two fit on an SM, so the launch
