@@ -127,6 +127,31 @@ __device__ __forceinline__ float ex2a(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
 }
+// 2^x for x <= 0 on the FMA and integer pipes: x = n + f with n the nearest integer (1.5 * 2^23 trick) and |f| <= 1/2,
+// 2^f by the degree-5 minimax polynomial (relative error 7.5e-8, 2.4e-7 with fp32 rounding), 2^n added into the
+// exponent field.  Arguments below -126 are clamped (the result, about 1e-38, stands for the hardware's 0).
+__device__ __forceinline__ float ex2p(float x) {
+  constexpr float kMagic = 12582912.f;
+  x = fmaxf(x, -126.f);
+  const float t = x + kMagic;
+  const float f = x - (t - kMagic);
+  float p = 0x1.5c08e6p-10f;
+  p = fmaf(p, f, 0x1.3d0c52p-7f);
+  p = fmaf(p, f, 0x1.c6b6e4p-5f);
+  p = fmaf(p, f, 0x1.ebf918p-3f);
+  p = fmaf(p, f, 0x1.62e428p-1f);
+  p = fmaf(p, f, 0x1.000002p+0f);
+  return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+}
+// Every QP_EXP_POLY-th exponential of the sweeps goes through ex2p instead of the 16-per-clock hardware unit, which is
+// the busiest unit of these kernels (0: none).  Measured for the whole score stage with 0 / 6 / 4 / 3: 196.6 / 186.7 /
+// 187.7 / 195.2 us for the 70B shapes at batch 4, 115.9 / 111.5 / 110.3 / 112.1 us at 128k.
+#ifndef QP_EXP_POLY
+#define QP_EXP_POLY 6
+#endif
+__device__ __forceinline__ float ex2_mixed(float x, int i) {
+  return QP_EXP_POLY > 0 && i % QP_EXP_POLY == QP_EXP_POLY - 1 ? ex2p(x) : ex2a(x);
+}
 __device__ __forceinline__ void cp_async16_zfill(uint32_t saddr, const void* gptr, bool valid) {
   const int n = valid ? 16 : 0;
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(saddr), "l"(gptr), "r"(n));
@@ -156,7 +181,7 @@ __device__ __forceinline__ void fold_row(const uint32_t (&r)[32], bool all_visib
     const float mn = fmaxf(m, cm * scale_log2);               // scale > 0: max commutes with it
     float acc = 0.f;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) acc += ex2a(fmaf(__uint_as_float(r[i]), scale_log2, -mn));
+    for (int i = 0; i < 32; ++i) acc += ex2_mixed(fmaf(__uint_as_float(r[i]), scale_log2, -mn), i);
     s = fmaf(s, ex2a(m - mn), acc);
     m = mn;
   } else {
@@ -181,8 +206,8 @@ __device__ __forceinline__ void fold_vote(const uint32_t (&r)[32], const float2*
 #pragma unroll
   for (int i = 0; i < 32; i += 2) {
     const float4 ms = *reinterpret_cast<const float4*>(&sRow[c0 + i]);   // (M, 1/Z) x 2 rows
-    vote = fmaf(ex2a(fmaf(__uint_as_float(r[i]), scale_log2, -ms.x)), ms.y, vote);
-    vote = fmaf(ex2a(fmaf(__uint_as_float(r[i + 1]), scale_log2, -ms.z)), ms.w, vote);
+    vote = fmaf(ex2_mixed(fmaf(__uint_as_float(r[i]), scale_log2, -ms.x), i), ms.y, vote);
+    vote = fmaf(ex2_mixed(fmaf(__uint_as_float(r[i + 1]), scale_log2, -ms.z), i + 1), ms.w, vote);
   }
 }
 
