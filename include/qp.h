@@ -43,7 +43,8 @@ extern "C" {
 typedef enum {
   QP_OK = 0,
   QP_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, Hq % Hkv != 0, w >= L, even pool ... */
-  QP_ERR_UNSUPPORTED = 2, /* bits not in {2,4,8,16}, group not in {32,64,128}, D not in {64,128}, G > 8, w > 64, pool > 65 */
+  QP_ERR_UNSUPPORTED = 2, /* bits not in {2,4,8,16}, group not in {32,64,128}, D not in {64,128}, G > 8, w > 64, pool > 65,
+                             batch * n_kv_heads * L >= 2^31 - 128 in the score stage */
   QP_ERR_BUDGET = 3,      /* budget gives n <= w, n is not a whole number of groups, or no room to append */
   QP_ERR_WORKSPACE = 4,   /* workspace too small */
   QP_ERR_ALIGNMENT = 5,   /* a base pointer is not 16-byte aligned */

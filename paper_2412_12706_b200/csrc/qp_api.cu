@@ -213,6 +213,8 @@ static qp_status check_score_args(const void* Q_win, const void* K, int batch, i
   if (s != QP_OK) return s;
   if (w < 1 || w >= L || pool < 1 || pool % 2 == 0) return QP_ERR_INVALID_ARG;
   if (w > 64 || pool > 65) return QP_ERR_UNSUPPORTED;
+  // the score sweeps address a layer's keys as one matrix of batch * n_kv_heads * L rows with 32-bit row coordinates
+  if ((long long)batch * Hkv * L > 0x7fffffffLL - 128) return QP_ERR_UNSUPPORTED;
   if (!aligned16(Q_win) || !aligned16(K)) return QP_ERR_ALIGNMENT;
   return QP_OK;
 }

@@ -152,6 +152,7 @@ def test_bad_arguments_are_rejected_before_any_launch(lib):
     assert lib.qp_gather_quantize(A, A, None, 1024, ref, None) == 1
     assert lib.qp_select_topk(A, 1, 2, 1024, 32, 32, A, None) == 3
     assert lib.qp_window_scores(A, A, 1, 8, 2, 64, 1024, 32, 7, A, A, 16, None) == 4
+    assert lib.qp_window_scores(A, A, 64, 64, 8, 64, 1 << 23, 32, 7, A, A, 1 << 62, None) == 2   # 2^32 key rows
 
 
 def test_strategy_head_budget_and_overlap_arguments_are_checked_before_any_launch(lib):

@@ -306,6 +306,26 @@ def test_compress_layers_is_bit_identical_to_per_layer_calls(bits, D, L, w):
         assert_packed_equal(cache_to_packed(caches[l]), cache_to_packed(ref_c))
 
 
+@pytest.mark.parametrize("nl", [9, 40])
+def test_compress_layers_with_many_layers_per_launch(nl):
+    """The score sweeps take the layers' key tensor maps as kernel parameters in tables of 8, 32 or 128 entries: 9 and
+    40 layers use the larger two.  Same comparison as above, on small layers."""
+    bits, group, w = 4, 32, 16
+    wl = small(synth.TINY, head_dim=64, n_q_heads=4, n_kv_heads=2, L=390, w=w, batch=1, bits=bits, group=group)
+    Ks, Vs, Qs = [], [], []
+    for l in range(nl):
+        k, v, qw = make_inputs(wl, l)
+        Ks.append(k.to(DEV)); Vs.append(v.to(DEV)); Qs.append(qw.to(DEV))
+    budgets = [bits * (32 + 32 * (1 + l % 5)) for l in range(nl)]
+    caches, kepts = qp.compress_layers(Ks, Vs, Qs, budgets, bits, group, wl.pool)
+    torch.cuda.synchronize()
+    for l in range(0, nl, 4):
+        ref_c, ref_k = qp.compress_layer(Ks[l], Vs[l], Qs[l], budgets[l], bits, group, wl.pool)
+        torch.cuda.synchronize()
+        assert torch.equal(kepts[l], ref_k), l
+        assert_packed_equal(cache_to_packed(caches[l]), cache_to_packed(ref_c))
+
+
 # ------------------------------------------------------------------ per-layer token / precision mixes in one decode call
 
 def test_decode_layers_with_mixed_precision_equals_separate_calls():
