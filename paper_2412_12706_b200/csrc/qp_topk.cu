@@ -288,8 +288,7 @@ topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __
 // The same selection for long prefixes (up to TKC_CTAS * TKC_ITEMS * 1024 positions) by a thread-block cluster per
 // (layer, batch, KV head): CTA c of the cluster holds the contiguous segment [c * S, (c + 1) * S) of the prefix in
 // registers, builds its own digit histogram in shared memory, and every CTA then sums the cluster's histograms
-// through distributed shared memory, so all of them take the same decision without any global traffic.  One
-// hardware cluster barrier per digit pass (the histograms are double-buffered) and two around the compaction.
+// through distributed shared memory, so all of them take the same decision without any global traffic.
 constexpr int TKC_CTAS = 8;
 constexpr int TKC_ITEMS = 16;
 
@@ -312,9 +311,10 @@ topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, cons
     return;
   }
 
-  __shared__ unsigned hist[2][256];                              // this CTA's histogram, alternating per pass
-  __shared__ unsigned ghist[256];                                // the cluster's histogram
-  __shared__ unsigned sh_prefix, sh_need;
+  __shared__ unsigned h12[TKR_BINS];                             // this CTA's histogram of a 12-bit digit
+  __shared__ unsigned xch[4][256];                               // exchanged counts, one buffer per step in rotation
+  __shared__ unsigned ghist[256];                                // the cluster's counts of the step
+  __shared__ unsigned sh_sel, sh_need;
   __shared__ unsigned cnt_g[TKC_ITEMS][32], cnt_e[TKC_ITEMS][32];
   __shared__ unsigned row_g[TKC_ITEMS], row_e[TKC_ITEMS];
   __shared__ unsigned tot_ge[2];                                 // this CTA's kept / equal totals
@@ -328,30 +328,24 @@ topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, cons
     key[q] = order_key(i < seg_n ? s[seg0 + i] : 0.f);
   }
 
+  // Three scans of the keys (digits of 12, 12 and 8 bits, plain shared-memory atomics as in the register kernel).  A
+  // 12-bit histogram stays in this CTA: what the cluster exchanges through distributed shared memory is its fold to
+  // 256 coarse bins (the digit's upper 8 bits) and then the 16 fine bins inside the chosen coarse bin, 272 counts per
+  // CTA instead of 4096, with one hardware cluster barrier per exchange (five in all).
   unsigned prefix = 0, mask = 0, need = (unsigned)k;
-  int pass = 0;
-  for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
-    unsigned* h = hist[pass & 1];
-    if (tid < 256) h[tid] = 0;
-    __syncthreads();
-#pragma unroll
-    for (int q = 0; q < TKC_ITEMS; ++q) {
-      if (q * TK_THREADS >= seg_n) break;
-      const bool cand = q * TK_THREADS + tid < seg_n && (key[q] & mask) == prefix;
-      const unsigned digit = (key[q] >> shift) & 255u;
-      if (shift >= 16) {
-        const unsigned peers = __match_any_sync(0xffffffffu, cand ? digit : 256u + lane);
-        if (cand && lane == __ffs(peers) - 1) atomicAdd(&h[digit], (unsigned)__popc(peers));
-      } else if (cand) {
-        atomicAdd(&h[digit], 1u);
-      }
-    }
-    cluster.sync();                                              // every CTA's histogram of this pass is complete
-    if (tid < 256) {
+  int step = 0;                                                  // exchange steps so far: buffer xch[step & 3]
+  // sums the CTAs' `n_bins` counts of buffer `buf`, finds the bin where the count from the top reaches `need`;
+  // every CTA takes the same decision
+  auto exchange_select = [&](int n_bins) -> unsigned {
+    unsigned* mine = xch[step & 3];
+    cluster.sync();                                              // every CTA's counts of this step are in place
+    if (tid < n_bins) {
       unsigned sum = 0;
 #pragma unroll
-      for (int c = 0; c < TKC_CTAS; ++c) sum += cluster.map_shared_rank(h, c)[tid];
+      for (int c = 0; c < TKC_CTAS; ++c) sum += cluster.map_shared_rank(mine, c)[tid];
       ghist[tid] = sum;
+    } else if (tid < 256) {
+      ghist[tid] = 0;
     }
     __syncthreads();
     if (warp == 0) {
@@ -373,13 +367,56 @@ topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, cons
           cum += c[bsel];
         }
         sh_need = need - cum;
-        sh_prefix = prefix | ((unsigned)(8 * lane + bsel) << shift);
+        sh_sel = (unsigned)(8 * lane + bsel);
       }
     }
     __syncthreads();
-    prefix = sh_prefix;
     need = sh_need;
-    mask |= 0xffu << shift;
+    ++step;
+    return sh_sel;
+  };
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 20 : pass == 1 ? 8 : 0;
+    const unsigned dmask = pass == 2 ? 255u : (unsigned)(TKR_BINS - 1);
+#pragma unroll
+    for (int i = 0; i < TKR_BINS / TK_THREADS; ++i) h12[tid + i * TK_THREADS] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < TKC_ITEMS; ++q) {
+      if (q * TK_THREADS >= seg_n) break;
+      const bool cand = q * TK_THREADS + tid < seg_n && (key[q] & mask) == prefix;
+      const unsigned digit = (key[q] >> shift) & dmask;
+      if (pass == 0) {
+        const unsigned d0 = __shfl_sync(0xffffffffu, digit, 0);
+        if (__all_sync(0xffffffffu, cand && digit == d0)) {
+          if (lane == 0) atomicAdd(&h12[d0], 32u);
+        } else if (cand) {
+          atomicAdd(&h12[digit], 1u);
+        }
+      } else if (cand) {
+        atomicAdd(&h12[digit], 1u);
+      }
+    }
+    __syncthreads();
+    if (pass == 2) {                                             // 8-bit digit: the histogram itself is exchanged
+      if (tid < 256) xch[step & 3][tid] = h12[tid];
+      const unsigned sel = exchange_select(256);
+      prefix |= sel;
+      mask |= 255u;
+    } else {
+      if (tid < 256) {                                           // fold to the digit's upper 8 bits
+        unsigned sum = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sum += h12[16 * tid + i];
+        xch[step & 3][tid] = sum;
+      }
+      const unsigned coarse = exchange_select(256);
+      if (tid < 16) xch[step & 3][tid] = h12[16 * coarse + tid];  // the 16 fine bins inside it
+      const unsigned fine = exchange_select(16);
+      prefix |= (16u * coarse + fine) << shift;
+      mask |= dmask << shift;
+    }
   }
   const uint32_t T = prefix;
 
