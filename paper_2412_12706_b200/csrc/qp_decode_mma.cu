@@ -419,7 +419,8 @@ constexpr int MG_WARPS = 4;
 // kernel fills the SMs as this call's drains, and this kernel runs in that kernel's shadow.  A large launch
 // would take too long that way; it uses a warp per output row and overlaps the next call's ramp only.
 // The same merge with plain loads (two records in flight per warp).
-__global__ void __launch_bounds__(MG_WARPS * 32, 16)
+template <int RUN, int MINB>
+__global__ void __launch_bounds__(MG_WARPS * 32, MINB)
 decode_merge_direct_kernel(const __grid_constant__ DecTable tab, const DecDims dm, const float* __restrict__ partials) {
   const int D = dm.D, G = dm.Hq / dm.Hkv, BH = dm.Bt * dm.Hkv, n_bq = dm.Bt * dm.Hq;
   const int lane = threadIdx.x & 31, n_items = n_bq * tab.n_layers;
@@ -443,16 +444,23 @@ decode_merge_direct_kernel(const __grid_constant__ DecTable tab, const DecDims d
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     if (4 * lane >= D) continue;
     float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
-#pragma unroll 2
-    for (int w = w_lo; w <= w_hi; ++w) {
-      const float* r = base + w * stride;
-      const float2 ml = *reinterpret_cast<const float2*>(r);
-      const float2 a01 = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
-      const float2 a23 = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
-      const float f = ex2(ml.x - M);
-      Ls = fmaf(ml.y, f, Ls);
-      A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
-      A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
+    // RUN records' loads are in flight together (past the row's end the last record again, with weight 0)
+    for (int w0 = w_lo; w0 <= w_hi; w0 += RUN) {
+      float2 ml[RUN], a01[RUN], a23[RUN];
+#pragma unroll
+      for (int i = 0; i < RUN; ++i) {
+        const float* r = base + min(w0 + i, w_hi) * stride;
+        ml[i] = *reinterpret_cast<const float2*>(r);
+        a01[i] = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
+        a23[i] = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
+      }
+#pragma unroll
+      for (int i = 0; i < RUN; ++i) {
+        const float f = w0 + i <= w_hi ? ex2(ml[i].x - M) : 0.f;
+        Ls = fmaf(ml[i].y, f, Ls);
+        A0 = fmaf(a01[i].x, f, A0); A1 = fmaf(a01[i].y, f, A1);
+        A2 = fmaf(a23[i].x, f, A2); A3 = fmaf(a23[i].y, f, A3);
+      }
     }
     const float inv = __fdiv_rn(1.0f, Ls);
     __nv_bfloat162 o01 = __floats2bfloat162_rn(A0 * inv, A1 * inv), o23 = __floats2bfloat162_rn(A2 * inv, A3 * inv);
@@ -534,7 +542,8 @@ decode_merge_sk_kernel(const __grid_constant__ DecTable tab, const DecDims dm, c
 // warps share the head's records (warp q takes records q, q + 4, ...), so a row's chain of dependent reads is a
 // quarter as long; the four partial sums are combined through shared memory in a fixed order.  Same launch
 // protocol as decode_merge_sk_kernel.
-__global__ void __launch_bounds__(MG_WARPS * 32, 16)
+constexpr int MR_RUN = 8;
+__global__ void __launch_bounds__(MG_WARPS * 32, 8)
 decode_merge_rows_kernel(const __grid_constant__ DecTable tab, const DecDims dm, const float* __restrict__ partials) {
   __shared__ float s_max[MG_WARPS];
   __shared__ float s_part[MG_WARPS][5 * 32];                      // per warp: lane's (A0..A3, Ls)
@@ -560,16 +569,26 @@ decode_merge_rows_kernel(const __grid_constant__ DecTable tab, const DecDims dm,
   __syncthreads();
   M = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
   float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
+  // a warp takes runs of MR_RUN consecutive records and has all of a run's loads in flight before it folds them: a long
+  // row (a single layer with thousands of kept tokens leaves a hundred records per row) is a chain of dependent
+  // round trips otherwise (measured for 128 records per row: 20 us with one record at a time)
   if (4 * lane < D)
-    for (int w = w_lo + wq; w <= w_hi; w += MG_WARPS) {
-      const float* r = base + w * stride;
-      const float2 ml = *reinterpret_cast<const float2*>(r);
-      const float2 a01 = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
-      const float2 a23 = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
-      const float f = ex2(ml.x - M);
-      Ls = fmaf(ml.y, f, Ls);
-      A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
-      A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
+    for (int w0 = w_lo + wq * MR_RUN; w0 <= w_hi; w0 += MG_WARPS * MR_RUN) {
+      float2 ml[MR_RUN], a01[MR_RUN], a23[MR_RUN];
+#pragma unroll
+      for (int i = 0; i < MR_RUN; ++i) {
+        const float* r = base + min(w0 + i, w_hi) * stride;     // past the end: the last record again, weight 0 below
+        ml[i] = *reinterpret_cast<const float2*>(r);
+        a01[i] = *reinterpret_cast<const float2*>(r + 2 + 4 * lane);
+        a23[i] = *reinterpret_cast<const float2*>(r + 4 + 4 * lane);
+      }
+#pragma unroll
+      for (int i = 0; i < MR_RUN; ++i) {
+        const float f = w0 + i <= w_hi ? ex2(ml[i].x - M) : 0.f;
+        Ls = fmaf(ml[i].y, f, Ls);
+        A0 = fmaf(a01[i].x, f, A0); A1 = fmaf(a01[i].y, f, A1);
+        A2 = fmaf(a23[i].x, f, A2); A3 = fmaf(a23[i].y, f, A3);
+      }
     }
   float* mine = s_part[wq] + 5 * lane;
   mine[0] = A0; mine[1] = A1; mine[2] = A2; mine[3] = A3; mine[4] = Ls;
@@ -613,8 +632,11 @@ int decode_mma_workers_per_sm(const DecDims& d) {
 // overlapping): 84 MB 4-bit 28.2 / 20.2 / 22.1 / 23.5 / 22.3, 168 MB 4-bit 35.9 / 35.8 / 40.8 / 38.1 / 34.2, 151 MB 8-bit
 // 34.9 / 33.0 / 35.1 / 38.7 / 36.6, 75 MB 8-bit 23.1 / 22.3 / 25.0 / 26.4 / 24.0, 42 MB 4-bit 16.9 / 16.3 / 16.6 / 17.4 / 18.6.
 // A call that runs alone (plain stream order) takes as many workers as it can give four tiles each: per-layer calls
-// replayed from a CUDA graph 10.2 / 8.4 / 8.4 / 10.2 us with at least 1 / 2 / 4 / 8 tiles per worker.  The 2-bit and
-// 16-bit kernels showed no gain from fewer workers and always use four tiles.
+// replayed from a CUDA graph 10.2 / 8.4 / 8.4 / 10.2 us with at least 1 / 2 / 4 / 8 tiles per worker.  Beyond 2048 tiles
+// (a layer of a whole batch, or one long sequence) eight tiles each pay, because the merge reads fewer records: from a
+// graph with at least 4 / 8 / 16 tiles, one layer of 8 heads x 16384 tokens 12.8 / 11.8 / 15.6 us, one layer of the 70B
+// shapes at batch 4 (42 MB) 20.8 / 17.7 / 17.8 us, 8 heads x 2048 tokens 7.7 / 10.1 / 15.1 us.  The 2-bit and 16-bit
+// kernels showed no gain from fewer workers on overlapping streams and use four tiles there.
 #ifndef QP_TMIN_BIG
 #define QP_TMIN_BIG 16
 #endif
@@ -625,7 +647,7 @@ int decode_mma_workers_per_sm(const DecDims& d) {
 #define QP_TMIN_SOLO 4
 #endif
 int decode_mma_tiles_per_worker_min(const DecDims& d, long long total_tiles, bool paired) {
-  if (!paired) return QP_TMIN_SOLO;
+  if (!paired) return total_tiles > 2048 ? 2 * QP_TMIN_SOLO : QP_TMIN_SOLO;
   if (d.bits != 4 && d.bits != 8) return 4;
   return total_tiles / QP_TMIN_BIG >= 256 ? QP_TMIN_BIG : QP_TMIN_SMALL;
 }
@@ -697,8 +719,14 @@ cudaError_t launch_merge_flat(const DecTable& tab, const DecDims& d, const float
   // form is the faster one beside the next call's attention blocks (overlapping calls; 168 MB 4-bit calls 52 -> 34 us
   // per call), while alone on the GPU the plain loads are (60 -> 45 us); on GB-sized launches, whose rows have one
   // or two records each, the plain loads win in both modes (2.1 GB calls: 422 -> 362 us).
-  if (!tab.paired || row_blocks > 2 * sm_count())
-    return cudaLaunchKernelEx(&cfg, decode_merge_direct_kernel, tab, d, (const float*)partials);
+  if (!tab.paired || row_blocks > 2 * sm_count()) {
+    // rows with a few records: two loads in flight and 32 registers, so the grid fits beside attention blocks; longer
+    // rows (one layer of a batch leaves dozens of records per row): eight in flight
+    const long long heads = (long long)tab.n_layers * d.Bt * d.Hkv;
+    if (tab.n_workers / heads + 1 <= 4)
+      return cudaLaunchKernelEx(&cfg, decode_merge_direct_kernel<2, 16>, tab, d, (const float*)partials);
+    return cudaLaunchKernelEx(&cfg, decode_merge_direct_kernel<8, 8>, tab, d, (const float*)partials);
+  }
   return cudaLaunchKernelEx(&cfg, decode_merge_sk_kernel, tab, d, (const float*)partials);
 }
 

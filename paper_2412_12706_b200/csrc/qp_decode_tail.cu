@@ -101,15 +101,22 @@ decode_merge_tail_kernel(const __grid_constant__ DecTable tab, const __grid_cons
   // ---- records, then tail tokens, in a fixed order
   float Ls = 0.f, A0 = 0.f, A1 = 0.f, A2 = 0.f, A3 = 0.f;
   if (chan)
-    for (int r = 0; r < count; ++r) {
-      const float* rec = base + r * stride;
-      const float2 ml = *reinterpret_cast<const float2*>(rec);
-      const float2 a01 = *reinterpret_cast<const float2*>(rec + 2 + 4 * lane);
-      const float2 a23 = *reinterpret_cast<const float2*>(rec + 4 + 4 * lane);
-      const float f = exp2f(ml.x - M);
-      Ls = fmaf(ml.y, f, Ls);
-      A0 = fmaf(a01.x, f, A0); A1 = fmaf(a01.y, f, A1);
-      A2 = fmaf(a23.x, f, A2); A3 = fmaf(a23.y, f, A3);
+    for (int r0 = 0; r0 < count; r0 += 4) {                      // four records' loads in flight together
+      float2 ml[4], a01[4], a23[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float* rec = base + min(r0 + i, count - 1) * stride;   // past the end: the last record again, weight 0
+        ml[i] = *reinterpret_cast<const float2*>(rec);
+        a01[i] = *reinterpret_cast<const float2*>(rec + 2 + 4 * lane);
+        a23[i] = *reinterpret_cast<const float2*>(rec + 4 + 4 * lane);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float f = r0 + i < count ? exp2f(ml[i].x - M) : 0.f;
+        Ls = fmaf(ml[i].y, f, Ls);
+        A0 = fmaf(a01[i].x, f, A0); A1 = fmaf(a01[i].y, f, A1);
+        A2 = fmaf(a23[i].x, f, A2); A3 = fmaf(a23[i].y, f, A3);
+      }
     }
   // value rows four at a time (row index clamped; the weight past the end is 0)
 #pragma unroll
