@@ -52,11 +52,11 @@ DTYPE = "f16-mma/f32-acc"      # bf16 inputs and outputs, f16 tensor-core operan
 # (sha256 of DECODE_KERNEL_SOURCES).  Captured on a few layers of the named workload; the traffic is proportional
 # to the tiles streamed, so a full launch's traffic is ratio x its algorithmic bytes.
 NCU_TRAFFIC: dict = {
-    "sha256": "10a770e58fb07914221ac9b395877cada41585638a5d052d3233118645aed1ec",
+    "sha256": "19c2c85de55d4ea6dd33aa50deecb688866ebceb1d17aca306556886ff7297c1",
     # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the attention kernel's launch, mean of two
-    # launches each: 16 layers x batch 1 of the 70B shapes (104.92 MB read + 3.53 MB written for 104.86 MB),
-    # 3 layers of the 32k x batch-8 2-bit workload (151.28 + 3.74 for 150.99 MB), the 8k workload (84.18 + 3.18 for 83.89 MB)
-    "ratio": {"llama3-70b-32k-b4-4bit-pyramid": 1.034, "llama3-8b-32k-b8-2bit": 1.027, "llama3-8b-8k-b1-4bit": 1.041},
+    # launches each: 16 layers x batch 1 of the 70B shapes (104.92 MB read + 5.05 MB written for 104.86 MB),
+    # 3 layers of the 32k x batch-8 2-bit workload (151.29 + 3.62 for 150.99 MB), the 8k workload (84.18 + 2.74 for 83.89 MB)
+    "ratio": {"llama3-70b-32k-b4-4bit-pyramid": 1.049, "llama3-8b-32k-b8-2bit": 1.026, "llama3-8b-8k-b1-4bit": 1.036},
 }
 
 KERNELS_PER_COMPRESS = 6      # sweep 1, row-stat merge, sweep 2, pool, top-k, gather+quantize (+ one 4-byte memset)
