@@ -421,3 +421,33 @@ def test_calls_of_different_sizes_may_share_one_workspace(overlap):
     for rep in range(5):
         for i in range(len(shapes)):
             assert torch.equal(outs[rep][i], refs[i]), (rep, i, shapes[i])
+
+
+# ------------------------------------------------------------------ random configurations, end to end
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_configurations_end_to_end(seed):
+    """Twelve seeded random shapes per seed (bits, head dimension, heads per group, group size, window, ragged context
+    lengths, pooling width, batch, budget) through compress and decode against the oracle, stage by stage."""
+    import random
+    rng = random.Random(seed)
+    done = 0
+    while done < 12:
+        bits = rng.choice([2, 4, 8, 16])
+        D = rng.choice([64, 128])
+        G = rng.choice([1, 2, 3, 4] if bits == 2 else [1, 2, 4, 8])
+        Hkv = rng.choice([1, 2, 3])
+        group = 32 if bits == 2 else rng.choice([32, 64] + ([128] if D == 128 else []))
+        w = rng.choice([1, 5, 8, 16, 32, 64])
+        L = rng.choice([rng.randint(300, 900), rng.randint(1000, 5000), rng.randint(5000, 9000)])
+        pool = rng.choice([1, 3, 7, 13])
+        batch = rng.choice([1, 2])
+        unit = max(group, 32)
+        n_lo, n_hi = w // unit + 1, (L - 1) // unit
+        if n_hi <= n_lo:
+            continue
+        n = rng.randint(n_lo, min(n_hi, n_lo + 40)) * unit
+        wl = small(synth.TINY, bits=bits, head_dim=D, n_q_heads=Hkv * G, n_kv_heads=Hkv, group=group, w=w, L=L,
+                   pool=pool, batch=batch, tokens16=n * bits // 16, seed=synth.BASE_SEED + 7000 + 100 * seed + done)
+        run_end_to_end(wl, decode_steps=2)
+        done += 1
