@@ -451,3 +451,44 @@ def test_random_configurations_end_to_end(seed):
                    pool=pool, batch=batch, tokens16=n * bits // 16, seed=synth.BASE_SEED + 7000 + 100 * seed + done)
         run_end_to_end(wl, decode_steps=2)
         done += 1
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_multi_layer_decode_calls(seed):
+    """Eight seeded random qp_decode_attn_layers calls per seed (1 to 9 layers with their own token counts, every bit
+    width, group size and heads-per-group count) against the oracle, in plain stream order and with overlapping calls:
+    the flat-range split, the three merge forms and the choice between them see shapes the fixed cases do not."""
+    import random
+    rng = random.Random(seed)
+    for case in range(8):
+        bits = rng.choice([2, 4, 8, 16]); D = rng.choice([64, 128])
+        G = rng.choice([1, 2, 3, 4] if bits == 2 else [1, 2, 4, 8]); Hkv = rng.choice([1, 2, 4, 8]); batch = rng.choice([1, 2, 4])
+        group = 32 if bits == 2 else rng.choice([32, 64] + ([128] if D == 128 else []))
+        unit = max(group, 32)
+        nl = rng.choice([1, 1, 2, 3, 5, 9])
+        ns = [rng.randint(1, 100 if rng.random() < 0.3 else 24) * unit for _ in range(nl)]
+        wl = small(synth.TINY, n_q_heads=Hkv * G, n_kv_heads=Hkv, head_dim=D, L=max(ns), batch=batch, group=group,
+                   seed=synth.BASE_SEED + 9500 + 50 * seed + case)
+        caches, qs, refs = [], [], []
+        for l, n in enumerate(ns):
+            k, v = synth.make_kv(wl, l)
+            kept = np.broadcast_to(np.arange(n, dtype=np.int32), (batch, Hkv, n)).copy()
+            pk = orc.quantize(bits_u16(k), bits_u16(v), kept, bits, group)
+            c = qp.alloc_cache(batch, Hkv * G, Hkv, D, bits, group, n, DEV)
+            qp.gather_quantize(k.to(DEV), v.to(DEV), torch.from_numpy(kept).to(DEV), c)
+            q = synth.make_q_dec(wl, l, 0)
+            kd, vd = orc.dequantize(pk, D)
+            refs.append(orc.decode(bits_u16(q), kd, vd)); caches.append(c); qs.append(q.to(DEV))
+        for overlap in (False, True):
+            outs = [torch.empty_like(x) for x in qs]
+            lb = qp.LayerBatch(qs, caches, outs)
+            qp.decode_overlap(overlap)
+            try:
+                for _ in range(3):
+                    qp.decode_attn_layers(lb)
+                torch.cuda.synchronize()
+            finally:
+                qp.decode_overlap(False)
+            for l in range(nl):
+                err = np.abs(outs[l].float().cpu().numpy().astype(np.float64) - refs[l]).max()
+                assert err <= 3e-3 + 2.0 ** -7 * np.abs(refs[l]).max(), (case, l, ns[l], overlap, err)
