@@ -135,3 +135,29 @@ def test_layers_calls_with_layers_in_different_states(bits):
             assert err <= decode_tolerance(ref), (s, l, err)
     for l in range(nl):
         assert_packed_equal(cache_to_packed(caches[l], gb.cache_arr[l]), states[l].packed)
+
+
+@pytest.mark.parametrize("bits,n", [(4, 4096), (8, 2080), (2, 3104)])
+def test_generation_steps_on_a_long_cache_with_many_records_per_row(bits, n):
+    """One layer with thousands of kept tokens leaves dozens of partial records per output row; the merge that also
+    folds the tail takes them four at a time (the last batch is ragged for these sizes)."""
+    group, D, G = 32, 128, 4
+    wl = workload(bits, group, D, G, L=n + 1500, tokens16=n * bits // 16, batch=1)
+    cache = compress(wl, 2 * group)
+    tail = qp.alloc_tail(cache)
+    st = orc.gen_state(cache_to_packed(cache), D)
+    ws = qp.new_decode_workspace(qp.decode_workspace_bytes(cache), DEV)
+    for s in range(group + 3):
+        kn, vn = synth.make_kv_new(wl, 0, s)
+        qp.append_kv(kn.to(DEV), vn.to(DEV), cache, tail)
+        st = orc.append(st, bits_u16(kn), bits_u16(vn))
+        if s % 7 and s < group:
+            continue
+        q = synth.make_q_dec(wl, 0, s)
+        out = qp.decode_attn_tail(q.to(DEV), cache, tail, workspace=ws)
+        torch.cuda.synchronize()
+        ref = orc.decode_state(bits_u16(q), st, D)
+        err = float(np.abs(out.float().cpu().numpy() - ref).max())
+        assert err <= decode_tolerance(ref), (s, err)
+        assert err <= 3e-3 + 2.0 ** -7 * float(np.abs(ref).max()), (s, err)
+    assert_packed_equal(cache_to_packed(cache), st.packed)
