@@ -346,7 +346,8 @@ qp_status qp_decode_attn_layers_ex(int n_layers, const void* const* q, const qp_
 /*
  * Debug build only (libqp_checked.so, compiled with -DQP_CHECKED; no counterpart in the paper).  In that build
  * every index a kernel reads from DEVICE memory and then uses as an address (the kept positions given to the
- * gather / quantize kernels, the side lists' tile pointers and entries) is compared with its limit first; a
+ * gather / quantize kernels, the side lists' tile pointers and entries), and every output position the top-k kernels
+ * compute from their counts, is compared with its limit first; a
  * violation never traps: the first one is recorded, all are counted, and the access goes to element 0 or is
  * skipped.  This call synchronises the device, copies the record to words4 (host: 1 + site of the first
  * violation or 0, the offending index, its limit, the number of violations) and clears it.  Indices that

@@ -554,17 +554,20 @@ qp_status qp_decode_attn_ex(const void* q, const qp_cache* cache, const qp_strat
 namespace qp {
 cudaError_t quant_check_read(unsigned int (&out)[4]);
 cudaError_t decode_check_read(unsigned int (&out)[4]);
+cudaError_t topk_check_read(unsigned int (&out)[4]);
 }
 extern "C" {
 #endif
 qp_status qp_debug_check(uint32_t* words4) {
   if (!words4) return QP_ERR_INVALID_ARG;
 #ifdef QP_CHECKED
-  unsigned int a[4], b[4];
-  if (qp::quant_check_read(a) != cudaSuccess || qp::decode_check_read(b) != cudaSuccess) return QP_ERR_CUDA;
-  const unsigned int* first = a[0] ? a : b;
+  unsigned int a[4], b[4], c[4];
+  if (qp::quant_check_read(a) != cudaSuccess || qp::decode_check_read(b) != cudaSuccess ||
+      qp::topk_check_read(c) != cudaSuccess)
+    return QP_ERR_CUDA;
+  const unsigned int* first = a[0] ? a : b[0] ? b : c;
   words4[0] = first[0]; words4[1] = first[1]; words4[2] = first[2];
-  words4[3] = a[3] + b[3];
+  words4[3] = a[3] + b[3] + c[3];
   return QP_OK;
 #else
   words4[0] = words4[1] = words4[2] = words4[3] = 0u;

@@ -1,6 +1,6 @@
 // Debug build with device-side range checks (compile with -DQP_CHECKED; the build script makes it as
 // libqp_checked.so).  Every index that a kernel takes from DEVICE memory before using it as an address (the kept
-// positions, the side lists' entries and tile pointers) is compared with its limit first.  A violation never traps:
+// positions, the side lists' entries and tile pointers; also the output positions the top-k kernels compute from their counts) is compared with its limit first.  A violation never traps:
 // the first one is recorded (site, index, limit), all are counted, and the access is redirected to element 0 or
 // skipped.  The host reads the record with qp_debug_check().  The normal build compiles the checks away.
 #pragma once
@@ -43,3 +43,4 @@ inline cudaError_t read_and_clear(unsigned int (&out)[4]) {
 #define QP_SITE_SIDE_KEPT 3u        // side-list build: a kept position >= L
 #define QP_SITE_SIDE_PTR 4u         // decode: a side list's tile pointer outside [0, cap]
 #define QP_SITE_SIDE_IDX 5u         // decode: a side-list entry outside the cache
+#define QP_SITE_TOPK_OUT 6u         // top-k: an output position computed from the counts >= k

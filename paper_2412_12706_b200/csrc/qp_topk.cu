@@ -7,6 +7,7 @@
 // first among equals" without sorting.  Integer work only: results are exact.
 #include <cooperative_groups.h>
 
+#include "qp_checked.cuh"
 #include "qp_common.cuh"
 
 namespace qp {
@@ -140,7 +141,7 @@ topk_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid
       const unsigned tot_g = __shfl_sync(0xffffffffu, sg, 31), tot_e = __shfl_sync(0xffffffffu, se, 31);
       const unsigned pre_g = __shfl_sync(0xffffffffu, sg - wg, warp), pre_e = __shfl_sync(0xffffffffu, se - we, warp);
       const unsigned pg = run_g + pre_g + __popc(bg & lt_mask), pe = run_e + pre_e + __popc(be & lt_mask);
-      if (gt || (eq && pe < need)) out[pg + min(pe, need)] = j;
+      if ((gt || (eq && pe < need)) && QP_IN_RANGE(pg + min(pe, need), k, QP_SITE_TOPK_OUT)) out[pg + min(pe, need)] = j;
       run_g += tot_g;
       run_e += tot_e;
       __syncthreads();                                      // warp_gt / warp_eq are rewritten by the next chunk
@@ -281,7 +282,7 @@ topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __
     const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
     const unsigned pg = row_g[q] + cnt_g[q][warp] + __popc(bg & lt_mask);
     const unsigned pe = row_e[q] + cnt_e[q][warp] + __popc(be & lt_mask);
-    if (gt || (eq && pe < need)) out[pg + min(pe, need)] = j;
+    if ((gt || (eq && pe < need)) && QP_IN_RANGE(pg + min(pe, need), k, QP_SITE_TOPK_OUT)) out[pg + min(pe, need)] = j;
   }
 }
 
@@ -468,7 +469,7 @@ topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, cons
     const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
     const unsigned pg = base_g + row_g[q] + cnt_g[q][warp] + __popc(bg & lt_mask);
     const unsigned pe = base_e + row_e[q] + cnt_e[q][warp] + __popc(be & lt_mask);
-    if (gt || (eq && pe < need)) out[pg + min(pe, need)] = seg0 + i;
+    if ((gt || (eq && pe < need)) && QP_IN_RANGE(pg + min(pe, need), k, QP_SITE_TOPK_OUT)) out[pg + min(pe, need)] = seg0 + i;
   }
   cluster.sync();                                                // no CTA leaves while another may still read its totals
 }
@@ -560,5 +561,9 @@ cudaError_t launch_head_budgets(const float* scores, int Bt, int Hkv, int L, int
   head_budget_kernel<<<Bt, 64, Hkv * sizeof(int), st>>>(kept_flat, (int)k_total, Hkv, P, L, w, n_mean, unit, n_heads);
   return cudaGetLastError();
 }
+
+#ifdef QP_CHECKED
+cudaError_t topk_check_read(unsigned int (&out)[4]) { return checked::read_and_clear(out); }
+#endif
 
 }  // namespace qp
