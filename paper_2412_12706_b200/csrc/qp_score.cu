@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(RM_ROWS * RM_SLICES)
 rowstat_merge_kernel(const float2* __restrict__ stat_partial, int blk0, int n_rb, int n_tiles, int R,
                      float2* __restrict__ rowstat) {
   __shared__ float2 part[RM_SLICES][RM_ROWS];
+  chain_enter();
   const int blk = blk0 + blockIdx.x / RM_PARTS, rb = blk % n_rb;
   const int rl = threadIdx.x % RM_ROWS, sl = threadIdx.x / RM_ROWS, row = (blockIdx.x % RM_PARTS) * RM_ROWS + rl;
   const float2* p = stat_partial + (size_t)blk * n_tiles * SC_RB + row;
@@ -65,6 +66,7 @@ constexpr int PK_THREADS = 256, PK_PER = 4, PK_OUT = PK_THREADS * PK_PER, PK_MAX
 __global__ void __launch_bounds__(PK_THREADS)
 pool_kernel(const float* __restrict__ votes_partial, int n_rb, int P, int pool, float* __restrict__ scores) {
   __shared__ float sv[PK_OUT + 2 * PK_MAX_HALO];
+  chain_enter();
   const int bh = blockIdx.y, j0 = blockIdx.x * PK_OUT, r = (pool - 1) / 2;
   const float* vp = votes_partial + (size_t)bh * n_rb * P;
   for (int i = threadIdx.x; i < PK_OUT + 2 * r; i += PK_THREADS) {
@@ -135,14 +137,15 @@ cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, c
     e = launch_score_sweep_tc(1, n_layers, Qwin, K, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st, bh0, cnt,
                               &n_splits);
     if (e != cudaSuccess) return e;
-    rowstat_merge_kernel<<<cnt * s.n_rb * RM_PARTS, RM_ROWS * RM_SLICES, 0, st>>>(stat_partial, bh0 * s.n_rb, s.n_rb,
-                                                                                 n_splits, R, rowstat);
+    e = launch_chained(rowstat_merge_kernel, dim3(cnt * s.n_rb * RM_PARTS), dim3(RM_ROWS * RM_SLICES), 0, st,
+                       (const float2*)stat_partial, bh0 * s.n_rb, s.n_rb, n_splits, R, rowstat);
+    if (e != cudaSuccess) return e;
     e = launch_score_sweep_tc(2, n_layers, Qwin, K, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st, bh0, cnt,
                               nullptr);
     if (e != cudaSuccess) return e;
   }
-  pool_kernel<<<dim3((P + PK_OUT - 1) / PK_OUT, BH), PK_THREADS, 0, st>>>(votes_partial, s.n_rb, P, d.pool, scores);
-  return cudaGetLastError();
+  return launch_chained(pool_kernel, dim3((P + PK_OUT - 1) / PK_OUT, BH), dim3(PK_THREADS), 0, st,
+                        (const float*)votes_partial, s.n_rb, P, d.pool, scores);
 }
 
 cudaError_t launch_window_scores(const void* Qwin, const void* K, const ScoreDims& d, float* scores, void* ws,

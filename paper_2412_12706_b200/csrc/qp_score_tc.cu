@@ -227,6 +227,7 @@ score_sweep_tc_kernel(const __grid_constant__ ScoreMaps<NL> maps, int bh0, int B
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+  chain_enter();
   // bh counts (layer, batch, KV head): the scratch arrays are laid out over all of them, the inputs are per layer
   const int split = blockIdx.x, rb = blockIdx.y, bh = bh0 + blockIdx.z, layer = bh / BH, bhl = bh % BH;
   const int b = bhl / Hkv, hk = bhl % Hkv, G = Hq / Hkv, P = L - w, R = G * w;
@@ -441,10 +442,9 @@ cudaError_t launch_tc(dim3 grid, int bh0, int BH, cudaStream_t st, const ScoreMa
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(score_sweep_tc_kernel<PASS, D, NL>, smem, done);
   if (e != cudaSuccess) return e;
-  score_sweep_tc_kernel<PASS, D, NL><<<grid, TC_THREADS, smem, st>>>(maps, bh0, BH, d.Hq, d.Hkv, d.L, d.w, s.n_rb, s.n_tiles,
-                                                                    per, (int)grid.x, scale_log2, stat_partial, rowstat,
-                                                                    votes_partial, error_word);
-  return cudaGetLastError();
+  return launch_chained(score_sweep_tc_kernel<PASS, D, NL>, grid, dim3(TC_THREADS), smem, st, maps, bh0, BH, d.Hq, d.Hkv, d.L,
+                        d.w, s.n_rb, s.n_tiles, per, (int)grid.x, scale_log2, stat_partial, rowstat, votes_partial,
+                        error_word);
 }
 
 template <int NL>

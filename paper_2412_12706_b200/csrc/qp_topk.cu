@@ -35,6 +35,7 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 template <int NL>
 __global__ void __launch_bounds__(TK_THREADS)
 topk_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid_constant__ TopkOut<NL> o) {
+  chain_enter();
   const int layer = blockIdx.x / BH, n_keep = o.n_keep[layer];
   const int P = L - w, k = n_keep - w;
   const int bh = blockIdx.x % BH, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -156,6 +157,7 @@ topk_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid
 template <int ITEMS, int NL>
 __global__ void __launch_bounds__(TK_THREADS)
 topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid_constant__ TopkOut<NL> o) {
+  chain_enter();
   const int layer = blockIdx.x / BH, n_keep = o.n_keep[layer];
   const int P = L - w, k = n_keep - w;
   const int bh = blockIdx.x % BH, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -296,6 +298,7 @@ constexpr int TKC_ITEMS = 16;
 template <int NL>
 __global__ void __cluster_dims__(TKC_CTAS, 1, 1) __launch_bounds__(TK_THREADS)
 topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid_constant__ TopkOut<NL> o) {
+  chain_enter();
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   const int head = blockIdx.x / TKC_CTAS, crank = (int)cluster.block_rank();
@@ -483,12 +486,12 @@ cudaError_t launch_topk(const float* scores, int blocks, int BH, int L, int w, c
   // a cluster per head also pays for prefixes of 8k to 32k positions when the heads alone would leave most SMs
   // idle (measured at 32k positions: 19.5 us against 24.8 us for 8 heads)
   const bool few_heads = blocks * TKC_CTAS <= sm_count();
-  if (P <= 8 * TK_THREADS) topk_reg_kernel<8, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
-  else if (P <= 32 * TK_THREADS && !few_heads) topk_reg_kernel<32, NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
+  if (P <= 8 * TK_THREADS) return launch_chained(topk_reg_kernel<8, NL>, dim3(blocks), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
+  else if (P <= 32 * TK_THREADS && !few_heads)
+    return launch_chained(topk_reg_kernel<32, NL>, dim3(blocks), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
   else if (P <= TKC_CTAS * TKC_ITEMS * TK_THREADS)
-    topk_cluster_kernel<NL><<<blocks * TKC_CTAS, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
-  else topk_kernel<NL><<<blocks, TK_THREADS, 0, st>>>(scores, L, w, BH, o);
-  return cudaGetLastError();
+    return launch_chained(topk_cluster_kernel<NL>, dim3(blocks * TKC_CTAS), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
+  return launch_chained(topk_kernel<NL>, dim3(blocks), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
 }
 }  // namespace
 
