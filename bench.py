@@ -59,7 +59,7 @@ NCU_TRAFFIC: dict = {
     "ratio": {"llama3-70b-32k-b4-4bit-pyramid": 1.049, "llama3-8b-32k-b8-2bit": 1.026, "llama3-8b-8k-b1-4bit": 1.036},
 }
 
-KERNELS_PER_COMPRESS = 6      # sweep 1, row-stat merge, sweep 2, pool, top-k, gather+quantize (+ one 4-byte memset)
+KERNELS_PER_COMPRESS = 5      # sweep 1, sweep 2 (folds the row statistics), pool, top-k, gather+quantize (+ one 4-byte memset)
 KERNELS_PER_DECODE_CALL = 2   # split-K attention, merge
 DECODE_KERNEL_SOURCES = ("qp_decode.cu", "qp_decode_mma.cu", "qp_decode_mma2.cu", "qp_decode_mma8.cu",
                          "qp_decode_mma16.cu", "qp_mma.cuh")

@@ -110,7 +110,7 @@ bool score_tc_supported(int D);
 cudaError_t launch_score_sweep_tc(int pass, int n_layers, const void* const* q, const void* const* k, const ScoreDims& d,
                                   const ScoreWorkspace& s, float scale_log2, float2* stat_partial, const float2* rowstat,
                                   float* votes_partial, int* error_word, cudaStream_t st, int bh0, int bh_count,
-                                  int* n_splits);
+                                  int* n_splits, int n_stat = 0);
 
 cudaError_t launch_select_topk(const float* scores, int BH, int L, int w, int n_keep, int32_t* kept, cudaStream_t st);
 // n_layers layers in one launch: scores [n_layers, BH, P]; kept[l] int32 [BH, n_keep[l]]

@@ -4,7 +4,8 @@
 // matrix; the logits are their product (a dense contraction: qp_score_tc.cu runs it on tcgen05).  The row
 // softmax needs every visible key of a row before any column can be normalised, hence two sweeps over K:
 //   sweep 1  per (run of key tiles, row) running (max, sum of exp) -> stat partials
-//   merge    per row: global max M and 1/Z
+//   merge    per row: global max M and 1/Z (folded by every block of sweep 2 for its own rows; a kernel of its own
+//            only when sweep 1 left more than 64 pairs per row)
 //   sweep 2  recompute the tile's logits, p = exp2(t - M)/Z, sum the tile's columns over the
 //            rows of the block                                     -> vote partials
 //   pool     sum the row blocks, zero-padded moving average of width `pool`.
@@ -137,11 +138,15 @@ cudaError_t launch_window_scores_layers(int n_layers, const void* const* Qwin, c
     e = launch_score_sweep_tc(1, n_layers, Qwin, K, d, s, scale_log2, stat_partial, nullptr, nullptr, err, st, bh0, cnt,
                               &n_splits);
     if (e != cudaSuccess) return e;
-    e = launch_chained(rowstat_merge_kernel, dim3(cnt * s.n_rb * RM_PARTS), dim3(RM_ROWS * RM_SLICES), 0, st,
-                       (const float2*)stat_partial, bh0 * s.n_rb, s.n_rb, n_splits, R, rowstat);
-    if (e != cudaSuccess) return e;
-    e = launch_score_sweep_tc(2, n_layers, Qwin, K, d, s, scale_log2, nullptr, rowstat, votes_partial, err, st, bh0, cnt,
-                              nullptr);
+    // the row statistics are folded inside sweep 2 unless sweep 1 left very many pairs per row
+    const bool fold_in_sweep = n_splits <= 64;
+    if (!fold_in_sweep) {
+      e = launch_chained(rowstat_merge_kernel, dim3(cnt * s.n_rb * RM_PARTS), dim3(RM_ROWS * RM_SLICES), 0, st,
+                         (const float2*)stat_partial, bh0 * s.n_rb, s.n_rb, n_splits, R, rowstat);
+      if (e != cudaSuccess) return e;
+    }
+    e = launch_score_sweep_tc(2, n_layers, Qwin, K, d, s, scale_log2, stat_partial, fold_in_sweep ? nullptr : rowstat,
+                              votes_partial, err, st, bh0, cnt, nullptr, n_splits);
     if (e != cudaSuccess) return e;
   }
   return launch_chained(pool_kernel, dim3((P + PK_OUT - 1) / PK_OUT, BH), dim3(PK_THREADS), 0, st,

@@ -271,7 +271,30 @@ score_sweep_tc_kernel(const __grid_constant__ ScoreMaps<NL> maps, int bh0, int B
     }
     cp_async_commit();
   }
-  if (PASS == 2 && tid < TC_M) sRow[tid] = rowstat[(size_t)(bh * n_rb + rb) * TC_M + tid];
+  if (PASS == 2 && tid < TC_M) {
+    if (rowstat) {
+      sRow[tid] = rowstat[(size_t)(bh * n_rb + rb) * TC_M + tid];
+    } else {
+      // sweep 1 left n_splits (max, sum) pairs per row: every block folds those of its 128 rows itself, in the same
+      // fixed order, instead of a kernel of its own between the sweeps (four loads in flight at a time)
+      const float2* p = stat_partial + (size_t)(bh * n_rb + rb) * n_splits * TC_M + tid;
+      float m = -INFINITY, z = 0.f;
+      for (int i0 = 0; i0 < n_splits; i0 += 4) {
+        float2 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = p[(size_t)min(i0 + i, n_splits - 1) * TC_M];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (i0 + i < n_splits && v[i].x != -INFINITY) {
+            const float mn = fmaxf(m, v[i].x);
+            z = z * exp2f(m - mn) + v[i].y * exp2f(v[i].x - mn);
+            m = mn;
+          }
+      }
+      const bool valid = rb * TC_M + tid < R;
+      sRow[tid] = make_float2(valid ? m : 0.f, valid ? __fdiv_rn(1.0f, z) : 0.f);
+    }
+  }
   cp_async_wait<0>();
   asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -437,20 +460,20 @@ cudaError_t key_map(CUtensorMap* map, const void* k, long long rows, int D) {
 template <int PASS, int D, int NL>
 cudaError_t launch_tc(dim3 grid, int bh0, int BH, cudaStream_t st, const ScoreMaps<NL>& maps, const ScoreDims& d,
                       const ScoreWorkspace& s, int per, float scale_log2, float2* stat_partial, const float2* rowstat,
-                      float* votes_partial, int* error_word) {
+                      float* votes_partial, int* error_word, int n_stat) {
   constexpr size_t smem = 3 * (size_t)TC_M * D * 2 + 1024;   // Q + two K stages + alignment slack
   static unsigned char done[64] = {};
   const cudaError_t e = allow_smem(score_sweep_tc_kernel<PASS, D, NL>, smem, done);
   if (e != cudaSuccess) return e;
   return launch_chained(score_sweep_tc_kernel<PASS, D, NL>, grid, dim3(TC_THREADS), smem, st, maps, bh0, BH, d.Hq, d.Hkv, d.L,
-                        d.w, s.n_rb, s.n_tiles, per, (int)grid.x, scale_log2, stat_partial, rowstat, votes_partial,
-                        error_word);
+                        d.w, s.n_rb, s.n_tiles, per, PASS == 1 ? (int)grid.x : n_stat, scale_log2, stat_partial, rowstat,
+                        votes_partial, error_word);
 }
 
 template <int NL>
 cudaError_t launch_sweep(int pass, int n_layers, const void* const* q, const void* const* k, int bh0, int bh_count,
                          const ScoreDims& d, const ScoreWorkspace& s, float scale_log2, float2* stat_partial,
-                         const float2* rowstat, float* votes_partial, int* error_word, cudaStream_t st, int* n_splits) {
+                         const float2* rowstat, float* votes_partial, int* error_word, cudaStream_t st, int* n_splits, int n_stat) {
   const int BH = d.Bt * d.Hkv;                          // (batch, KV head) pairs of one layer
   if ((long long)BH * d.L > 0x7fffffffLL - TC_N) return cudaErrorInvalidValue;   // row coordinates are 32-bit
   // the two sweeps of a call (and repeated calls on the same buffers) ask for the same maps: keep the last set
@@ -496,23 +519,24 @@ cudaError_t launch_sweep(int pass, int n_layers, const void* const* q, const voi
   if (n_splits) *n_splits = splits;
   const dim3 grid(splits, s.n_rb, bh_count);
   if (d.D == 128)
-    return pass == 1 ? launch_tc<1, 128, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
-                     : launch_tc<2, 128, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
-  return pass == 1 ? launch_tc<1, 64, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word)
-                   : launch_tc<2, 64, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word);
+    return pass == 1 ? launch_tc<1, 128, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word, n_stat)
+                     : launch_tc<2, 128, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word, n_stat);
+  return pass == 1 ? launch_tc<1, 64, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word, n_stat)
+                   : launch_tc<2, 64, NL>(grid, bh0, BH, st, maps, d, s, (int)per, scale_log2, stat_partial, rowstat, votes_partial, error_word, n_stat);
 }
 }  // namespace
 
 // s: the scratch layout for batch * n_layers batch entries (the layers are stacked along the batch dimension)
 // bh0, bh_count: the (layer, batch, KV head) triples this launch covers; *n_splits: blocks along the keys, i.e. the
-// (max, sum) pairs sweep 1 leaves per row in stat_partial [triple, row block, split, 128 rows]
+// (max, sum) pairs sweep 1 leaves per row in stat_partial [triple, row block, split, 128 rows]; sweep 2 with
+// rowstat == nullptr folds n_stat such pairs per row itself
 cudaError_t launch_score_sweep_tc(int pass, int n_layers, const void* const* q, const void* const* k, const ScoreDims& d,
                                   const ScoreWorkspace& s, float scale_log2, float2* stat_partial, const float2* rowstat,
                                   float* votes_partial, int* error_word, cudaStream_t st, int bh0, int bh_count,
-                                  int* n_splits) {
+                                  int* n_splits, int n_stat) {
 #define QP_SWEEP(NL) \
   return launch_sweep<NL>(pass, n_layers, q, k, bh0, bh_count, d, s, scale_log2, stat_partial, rowstat, votes_partial, \
-                          error_word, st, n_splits)
+                          error_word, st, n_splits, n_stat)
   if (n_layers == 1) QP_SWEEP(1);
   if (n_layers <= 8) QP_SWEEP(8);
   if (n_layers <= 32) QP_SWEEP(32);
