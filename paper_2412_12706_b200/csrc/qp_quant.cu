@@ -92,8 +92,14 @@ struct QuantTable {
 // (25 instructions per element under ncu against about 13 of arithmetic).
 // GROUP = 32 (the usual group) is compiled with the group's 32 elements held in registers between the min/max sweep
 // and the packing, and with vector stores of a group's words; GROUP = 0 takes the group size at run time.
+// Twelve blocks of 128 threads per SM (40 registers, a few spilled words): the kernel waits on its gathered rows, so
+// resident warps count for more than registers; measured with at least 1 / 10 / 12 / 14 blocks per SM for 8192 kept tokens
+// x 64 heads: 96.7 / 93.1 / 89.9 / 96.6 us at 2 bit, 99.0 / 96.5 / 92.7 / 98.7 us at 4 bit, 113.0 / 101.6 / 100.9 / 108.9 us at 8 bit.
+#ifndef QP_QUANT_MINB
+#define QP_QUANT_MINB 12
+#endif
 template <int BITS, int NL, int D, int GROUP, bool FILTER = false>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, QP_QUANT_MINB)
 gather_quant_kernel(const __grid_constant__ QuantTable<NL> tab, int g_rt) {
   const int g = GROUP > 0 ? GROUP : g_rt;
   extern __shared__ __align__(16) uint16_t sK[];   // [g][D] gathered key rows
