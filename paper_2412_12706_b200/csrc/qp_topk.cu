@@ -288,20 +288,21 @@ topk_reg_kernel(const float* __restrict__ scores, int L, int w, int BH, const __
   }
 }
 
-// The same selection for long prefixes (up to TKC_CTAS * TKC_ITEMS * 1024 positions) by a thread-block cluster per
+// The same selection for long prefixes (up to CTAS * TKC_ITEMS * 1024 positions; CTAS = 8, or 4 or 2 for mid head counts) by a
+// thread-block cluster per
 // (layer, batch, KV head): CTA c of the cluster holds the contiguous segment [c * S, (c + 1) * S) of the prefix in
 // registers, builds its own digit histogram in shared memory, and every CTA then sums the cluster's histograms
 // through distributed shared memory, so all of them take the same decision without any global traffic.
 constexpr int TKC_CTAS = 8;
 constexpr int TKC_ITEMS = 16;
 
-template <int NL>
-__global__ void __cluster_dims__(TKC_CTAS, 1, 1) __launch_bounds__(TK_THREADS)
+template <int NL, int CTAS>
+__global__ void __cluster_dims__(CTAS, 1, 1) __launch_bounds__(TK_THREADS)
 topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, const __grid_constant__ TopkOut<NL> o) {
   chain_enter();
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  const int head = blockIdx.x / TKC_CTAS, crank = (int)cluster.block_rank();
+  const int head = blockIdx.x / CTAS, crank = (int)cluster.block_rank();
   const int layer = head / BH, n_keep = o.n_keep[layer];
   const int P = L - w, k = n_keep - w;
   const int bh = head % BH, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -311,7 +312,7 @@ topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, cons
   if (crank == 0)
     for (int i = tid; i < w; i += TK_THREADS) out[k + i] = P + i;  // window tokens are always kept
   if (k >= P) {                                                    // keep everything (the whole cluster leaves)
-    for (int j = crank * TK_THREADS + tid; j < P; j += TKC_CTAS * TK_THREADS) out[j] = j;
+    for (int j = crank * TK_THREADS + tid; j < P; j += CTAS * TK_THREADS) out[j] = j;
     return;
   }
 
@@ -323,7 +324,7 @@ topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, cons
   __shared__ unsigned row_g[TKC_ITEMS], row_e[TKC_ITEMS];
   __shared__ unsigned tot_ge[2];                                 // this CTA's kept / equal totals
 
-  const int S = (P + TKC_CTAS - 1) / TKC_CTAS;                   // positions per CTA
+  const int S = (P + CTAS - 1) / CTAS;                   // positions per CTA
   const int seg0 = crank * S, seg_n = max(0, min(S, P - seg0));  // this CTA's segment
   uint32_t key[TKC_ITEMS];
 #pragma unroll
@@ -346,7 +347,7 @@ topk_cluster_kernel(const float* __restrict__ scores, int L, int w, int BH, cons
     if (tid < n_bins) {
       unsigned sum = 0;
 #pragma unroll
-      for (int c = 0; c < TKC_CTAS; ++c) sum += cluster.map_shared_rank(mine, c)[tid];
+      for (int c = 0; c < CTAS; ++c) sum += cluster.map_shared_rank(mine, c)[tid];
       ghist[tid] = sum;
     } else if (tid < 256) {
       ghist[tid] = 0;
@@ -486,11 +487,19 @@ cudaError_t launch_topk(const float* scores, int blocks, int BH, int L, int w, c
   // a cluster per head also pays for prefixes of 8k to 32k positions when the heads alone would leave most SMs
   // idle (measured at 32k positions: 19.5 us against 24.8 us for 8 heads)
   const bool few_heads = blocks * TKC_CTAS <= sm_count();
+  // between the two: a cluster of four or two per head while that still fits in one round of the SMs (measured at
+  // 32k positions: 32 heads 24.8 -> 16.7 us with four)
+  if (!few_heads && P > 8 * TK_THREADS) {
+    if (P <= 4 * TKC_ITEMS * TK_THREADS && blocks * 4 <= sm_count())
+      return launch_chained(topk_cluster_kernel<NL, 4>, dim3(blocks * 4), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
+    if (P <= 2 * TKC_ITEMS * TK_THREADS && blocks * 2 <= sm_count())
+      return launch_chained(topk_cluster_kernel<NL, 2>, dim3(blocks * 2), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
+  }
   if (P <= 8 * TK_THREADS) return launch_chained(topk_reg_kernel<8, NL>, dim3(blocks), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
   else if (P <= 32 * TK_THREADS && !few_heads)
     return launch_chained(topk_reg_kernel<32, NL>, dim3(blocks), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
   else if (P <= TKC_CTAS * TKC_ITEMS * TK_THREADS)
-    return launch_chained(topk_cluster_kernel<NL>, dim3(blocks * TKC_CTAS), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
+    return launch_chained(topk_cluster_kernel<NL, TKC_CTAS>, dim3(blocks * TKC_CTAS), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
   return launch_chained(topk_kernel<NL>, dim3(blocks), dim3(TK_THREADS), 0, st, scores, L, w, BH, o);
 }
 }  // namespace

@@ -70,12 +70,13 @@ def test_select_topk_bit_exact_with_ties(P, w, n):
 
 @pytest.mark.parametrize("P,w,n", [(5000, 32, 32 + 1000), (8192, 16, 16 + 4096), (20000, 32, 32 + 2048),
                                    (32736, 32, 8192), (12345, 8, 8 + 12000), (9000, 32, 32 + 1)])
-def test_select_topk_one_block_per_head_with_many_heads(P, w, n):
-    """With more heads than an eighth of the SMs every head is selected by one block from registers (12-bit digits):
+@pytest.mark.parametrize("Bt,Hkv", [(4, 6), (8, 6), (16, 10)])
+def test_select_topk_one_block_per_head_with_many_heads(P, w, n, Bt, Hkv):
+    """With more heads than an eighth of the SMs a head is selected by one block from registers, or above 8k positions by
+    a cluster of four (24 heads) or two (48 heads) while those fit in one round of the SMs, else by one block (160 heads):
     ties, constant rows, sorted rows, rows whose scores share their leading bits, denormals and zeros."""
     L = P + w
-    rng = np.random.default_rng(P * 7 + n)
-    Bt, Hkv = 4, 6
+    rng = np.random.default_rng(P * 7 + n + Bt)
     s = rng.random((Bt, Hkv, P)).astype(np.float32)
     s[0, 0] = np.round(s[0, 0] * 16) / 16
     s[0, 1] = 0.5
